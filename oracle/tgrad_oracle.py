@@ -1,0 +1,274 @@
+"""CPU oracle for the TensorGRaD optimizer step (Algorithm 1 of the paper).
+
+TEST INFRASTRUCTURE ONLY.  This file is a plain, slow, fp64 restatement of
+what the paper defines.  It shares no code with the CUDA library, is never
+imported by it, and must only be used by the tests, the smoke check and the
+benchmark's CPU-baseline leg.
+
+Every function names the passage it follows.  Contractions run in complex128,
+stored optimizer states are rounded to fp32 once per step (the paper keeps the
+optimizer states in full precision, Section 2.3), the top-k key is computed in
+fp32 exactly as the selection rule fixes it.
+
+Conventions where the paper is silent (each one is a stated reading, not a
+fact of the paper -- "parity unpinned" against the authors' own code for
+these): beta1/beta2/eps values, alpha on the low-rank part only (the
+reconstruction steps of Algorithm 1, not the equation of Section 2.2), bias correction with t+1,
+moments carried over unchanged across refreshes (slot-wise for the sparse
+ones), decoupled weight decay, fp16 storage of W/G in the mixed recipe.
+
+Sign convention: the caller passes grad = d(phi)/dW; Algorithm 1 defines
+G = -grad and W <- W + eta * Gtilde(G).  Every stage is odd in the sign of G
+(or even, for V), so the oracle evaluates the stages on grad and subtracts.
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------
+# Sparse part (Section 2.2, "Unstructured sparse gradient tensor")
+# --------------------------------------------------------------------------
+
+def magnitude_key(g: np.ndarray) -> np.ndarray:
+    """|g|^2 as fp32: fl(fl(re*re) + fl(im*im)), no fused multiply-add.
+
+    Top-k *magnitude* selection orders entries by |g|; squaring is monotone,
+    and this fp32 expression is the precision in which the decision is taken.
+    numpy rounds each float32 operation separately.
+    """
+    g = np.asarray(g)
+    re = np.ascontiguousarray(g.real, dtype=np.float32)
+    im = np.ascontiguousarray(g.imag, dtype=np.float32)
+    return (re * re) + (im * im)
+
+
+def sparse_indices_topk(g: np.ndarray, k: int) -> np.ndarray:
+    """SparseIndices(G, rho, top-k) of Algorithm 1, with k = ceil(rho I).
+
+    The k entries largest under (key descending, flat row-major index
+    ascending); returned as ascending flat indices (uint32).  A stable sort of
+    the negated key keeps equal keys in index order.
+    """
+    key = magnitude_key(g).reshape(-1)
+    if k < 0 or k > key.size:
+        raise ValueError("k out of range")
+    order = np.argsort(-key, kind="stable")
+    return np.sort(order[:k]).astype(np.uint32)
+
+
+def sparse_gather(g: np.ndarray, omega: np.ndarray) -> np.ndarray:
+    """Sparse(G, Omega): the values at the stored indices (the per-step
+    "create sparse tensor" statement of Algorithm 1)."""
+    return np.asarray(g).reshape(-1)[omega.astype(np.int64)].copy()
+
+
+def residual(g: np.ndarray, omega: np.ndarray) -> np.ndarray:
+    """R = G - Sparse(G, Omega): G with the entries at Omega set to zero
+    (Section 2.2 "Residual and composition"; the subtraction inside Algorithm 1)."""
+    r = np.array(g, copy=True, order="C")
+    r.reshape(-1)[omega.astype(np.int64)] = 0      # C-contiguous: reshape is a view
+    return r
+
+
+# --------------------------------------------------------------------------
+# Tensor algebra (Appendix "Tensor Operations and Notation")
+# --------------------------------------------------------------------------
+
+def unfold(x: np.ndarray, n: int) -> np.ndarray:
+    """Mode-n unfolding: mode-n fibres as columns, remaining indices ordered
+    first-index-fastest (Definition "Mode-k Unfolding")."""
+    return np.reshape(np.moveaxis(x, n, 0), (x.shape[n], -1), order="F")
+
+
+def mode_n_product(x: np.ndarray, u: np.ndarray, n: int) -> np.ndarray:
+    """(X x_n U)[.., j, ..] = sum_{i_n} X[.., i_n, ..] U[j, i_n]
+    (Definition "Mode-k Product"; U is J x I_n)."""
+    y = np.tensordot(u, x, axes=([1], [n]))      # new index j first
+    return np.moveaxis(y, 0, n)
+
+
+def tucker_compress(r: np.ndarray, factors: Sequence[np.ndarray]) -> np.ndarray:
+    """G_L = R x_1 U1^H ... x_N UN^H  (Section 2.2 low-rank compression,
+    the "low-rank compression" statement of Algorithm 1; complex tensors take conjugate transposes, Remark
+    "Real-Valued Analysis").  Modes are contracted in the order written."""
+    x = np.asarray(r, dtype=np.complex128)
+    for n, u in enumerate(factors):
+        x = mode_n_product(x, np.conj(np.asarray(u, dtype=np.complex128)).T, n)
+    return x
+
+
+def tucker_reconstruct(c: np.ndarray, factors: Sequence[np.ndarray]) -> np.ndarray:
+    """Gtilde_L = C x_1 U1 ... x_N UN (Section 2.2; the "reconstruct low-rank
+    part" statement of Algorithm 1)."""
+    x = np.asarray(c, dtype=np.complex128)
+    for n, u in enumerate(factors):
+        x = mode_n_product(x, np.asarray(u, dtype=np.complex128), n)
+    return x
+
+
+def mode_gram(r: np.ndarray, n: int) -> np.ndarray:
+    """A_n = R_(n) R_(n)^H (Hermitian PSD, I_n x I_n), complex128."""
+    m = unfold(np.asarray(r, dtype=np.complex128), n)
+    return m @ np.conj(m).T
+
+
+def canonical_phase(u: np.ndarray) -> np.ndarray:
+    """Multiply each column by the unit phase that makes its largest-modulus
+    component real and positive (first such row on ties)."""
+    u = np.array(u, copy=True)
+    for j in range(u.shape[1]):
+        col = u[:, j]
+        i = int(np.argmax(np.abs(col)))
+        a = col[i]
+        if a != 0:
+            u[:, j] = col * (np.conj(a) / np.abs(a))
+    return u
+
+
+def tucker_factors(r: np.ndarray, ranks: Sequence[int]) -> List[np.ndarray]:
+    """TuckerFactors(R, r) of Algorithm 1.
+
+    Each U^(n) holds the r_n leading left singular vectors of the mode-n
+    unfolding of R (the truncated-SVD stage of the decomposition described in
+    Appendix "Tensor Decomposition / Implementation"), obtained here as the
+    eigenvectors of the r_n largest eigenvalues of A_n = R_(n) R_(n)^H, in
+    descending eigenvalue order, phase-canonicalised, stored as complex64.
+    No refinement iterations are applied.
+    """
+    out = []
+    for n, rn in enumerate(ranks):
+        a = mode_gram(r, n)
+        w, v = np.linalg.eigh(a)                      # ascending eigenvalues
+        v = v[:, ::-1][:, :rn]
+        out.append(np.ascontiguousarray(canonical_phase(v).astype(np.complex64)))
+    return out
+
+
+# --------------------------------------------------------------------------
+# Adam in the compressed space (AdamUpdate of Algorithm 1; UPDATE block of Algorithm 3)
+# --------------------------------------------------------------------------
+
+def adam_update(x, m, v, beta1, beta2, eps, t):
+    """One Adam update of a compressed gradient x (complex) with first moment m
+    (complex64) and second moment v (float32).  Returns (N, m_new, v_new):
+
+        M <- b1 M + (1-b1) x          V <- b2 V + (1-b2) |x conj(x)|
+        N  = (M / (1-b1^(t+1))) / (sqrt(V / (1-b2^(t+1))) + eps)
+
+    t is the 0-based step counter, so the correction uses t+1.  The corrected
+    moments are temporaries: the stored ones are the un-corrected M and V,
+    rounded to fp32.
+    """
+    b1 = float(np.float32(beta1)); b2 = float(np.float32(beta2)); e = float(np.float32(eps))
+    x = np.asarray(x, dtype=np.complex128)
+    m_new = (b1 * np.asarray(m, dtype=np.complex128) + (1.0 - b1) * x).astype(np.complex64)
+    v_new = (b2 * np.asarray(v, dtype=np.float64)
+             + (1.0 - b2) * (x.real * x.real + x.imag * x.imag)).astype(np.float32)
+    c1 = float(np.float32(1.0 - b1 ** (t + 1)))
+    c2 = float(np.float32(1.0 - b2 ** (t + 1)))
+    n = (m_new.astype(np.complex128) / c1) / (np.sqrt(v_new.astype(np.float64) / c2) + e)
+    return n, m_new, v_new
+
+
+# --------------------------------------------------------------------------
+# The step (Algorithm 1)
+# --------------------------------------------------------------------------
+
+@dataclasses.dataclass
+class OracleConfig:
+    shape: Sequence[int]
+    ranks: Sequence[int]
+    k: int
+    T: int
+    lr: float = 1e-3
+    alpha: float = 1.0
+    lam: float = 1.0
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-8
+    weight_decay: float = 0.0
+    half_storage: bool = False      # W and G live as fp16 (re, im) pairs
+
+
+def _store_w(w: np.ndarray, half: bool) -> np.ndarray:
+    """Round a complex128 weight to its storage type and widen it back."""
+    if half:
+        re = w.real.astype(np.float16).astype(np.float64)
+        im = w.imag.astype(np.float16).astype(np.float64)
+        return re + 1j * im
+    return w.astype(np.complex64).astype(np.complex128)
+
+
+class OracleState:
+    """State of Algorithm 1 for one weight tensor (its initialisation statements)."""
+
+    def __init__(self, cfg: OracleConfig):
+        self.cfg = cfg
+        self.t = 0
+        p = tuple(int(r) for r in cfg.ranks)
+        self.omega: Optional[np.ndarray] = None
+        self.factors: Optional[List[np.ndarray]] = None
+        self.m_l = np.zeros(p, dtype=np.complex64)
+        self.v_l = np.zeros(p, dtype=np.float32)
+        self.m_s = np.zeros(cfg.k, dtype=np.complex64)
+        self.v_s = np.zeros(cfg.k, dtype=np.float32)
+        # last step's intermediates, kept for inspection by tests
+        self.core = None
+        self.n_l = None
+        self.g_s = None
+        self.n_s = None
+
+
+def oracle_refresh(st: OracleState, grad: np.ndarray) -> None:
+    """The `t mod T = 0` branch of Algorithm 1: new Omega, residual, new factors.  Moments are
+    left untouched (nothing in the loop resets them)."""
+    cfg = st.cfg
+    st.omega = sparse_indices_topk(grad, cfg.k)
+    st.factors = tucker_factors(residual(grad, st.omega), cfg.ranks)
+
+
+def oracle_step(st: OracleState, w: np.ndarray, grad: np.ndarray, refresh: Optional[bool] = None) -> np.ndarray:
+    """One pass of the loop body of Algorithm 1 for one tensor.
+
+    w, grad: complex arrays of cfg.shape holding values exactly representable
+    in the storage type.  Returns the new weight (complex64, or complex64
+    holding fp16-representable values for half storage).
+    refresh=None follows the schedule t mod T = 0; True/False overrides it.
+    """
+    cfg = st.cfg
+    do_refresh = (st.t % cfg.T == 0) if refresh is None else refresh
+    if do_refresh:
+        oracle_refresh(st, grad)
+    omega = st.omega.astype(np.int64)
+    # sparse values, residual, low-rank compression
+    g_s = sparse_gather(grad, st.omega).astype(np.complex64)
+    core = tucker_compress(residual(grad, st.omega), st.factors).astype(np.complex64)
+    # AdamUpdate on both compressed parts
+    n_s, st.m_s, st.v_s = adam_update(g_s, st.m_s, st.v_s, cfg.beta1, cfg.beta2, cfg.eps, st.t)
+    n_l, st.m_l, st.v_l = adam_update(core, st.m_l, st.v_l, cfg.beta1, cfg.beta2, cfg.eps, st.t)
+    n_s = n_s.astype(np.complex64); n_l = n_l.astype(np.complex64)
+    # reconstruction, scaled sparse add, weight update (signs flipped, see module docstring)
+    lr = float(np.float32(cfg.lr)); al = float(np.float32(cfg.alpha)); la = float(np.float32(cfg.lam))
+    wd = float(np.float32(cfg.weight_decay))
+    wn = np.asarray(w, dtype=np.complex128)
+    if wd != 0.0:
+        wn = wn * (1.0 - lr * wd)
+    d = tucker_reconstruct(n_l, st.factors)
+    wn = np.ascontiguousarray(_store_w(wn - (lr * al) * d, cfg.half_storage))
+    flat = wn.reshape(-1)                          # a view of the contiguous array
+    flat[omega] = _store_w(flat[omega] - (lr * la) * n_s.astype(np.complex128), cfg.half_storage)
+    st.core, st.n_l, st.g_s, st.n_s = core, n_l, g_s, n_s
+    st.t += 1
+    return wn.astype(np.complex64)
+
+
+def state_entries(shape, ranks, k):
+    """Optimizer-state entry counts (Appendix "Parameter Complexity Analysis"):
+    core-shaped moments, factor matrices, sparse indices and sparse moments."""
+    p = int(np.prod(ranks, dtype=np.int64))
+    fac = int(sum(int(i) * int(r) for i, r in zip(shape, ranks)))
+    return {"m_l": p, "v_l": p, "factors": fac, "omega": int(k), "m_s": int(k), "v_s": int(k)}

@@ -1,0 +1,63 @@
+"""Shared test utilities: comparison metrics and brute-force references.
+
+Nothing here implements the optimizer; these are measuring sticks.
+"""
+import numpy as np
+
+
+def rel_err(a, b, floor_frac=1e-3):
+    """max_i |a_i - b_i| / max(|b_i|, tau), tau = floor_frac * rms(b).
+
+    Pure element-wise relative error is undefined where b crosses zero, so
+    entries smaller than a fraction of the array's rms are measured against
+    that floor.
+    """
+    a = np.asarray(a).reshape(-1).astype(np.complex128)
+    b = np.asarray(b).reshape(-1).astype(np.complex128)
+    if b.size == 0:
+        return 0.0
+    rms = np.sqrt(np.mean(np.abs(b) ** 2))
+    tau = floor_frac * rms
+    den = np.maximum(np.abs(b), tau if tau > 0 else 1.0)
+    return float(np.max(np.abs(a - b) / den))
+
+
+def fro_err(a, b):
+    a = np.asarray(a).reshape(-1).astype(np.complex128)
+    b = np.asarray(b).reshape(-1).astype(np.complex128)
+    nb = np.linalg.norm(b)
+    return float(np.linalg.norm(a - b) / (nb if nb > 0 else 1.0))
+
+
+def max_sin_angle(u, v):
+    """Largest principal-angle sine between span(u) and span(v) (both with
+    orthonormal columns): || (I - v v^H) u ||_2."""
+    u = np.asarray(u, dtype=np.complex128)
+    v = np.asarray(v, dtype=np.complex128)
+    resid = u - v @ (np.conj(v).T @ u)
+    return float(np.linalg.norm(resid, 2))
+
+
+def ortho_defect(u):
+    u = np.asarray(u, dtype=np.complex128)
+    return float(np.max(np.abs(np.conj(u).T @ u - np.eye(u.shape[1]))))
+
+
+def brute_topk(g, k):
+    """Pure-Python top-k: sort all (key, index) pairs, key descending then
+    index ascending; key = fp32 re*re + im*im with separately rounded ops."""
+    flat = np.asarray(g).reshape(-1)
+    pairs = []
+    for i in range(flat.size):
+        re = np.float32(flat[i].real)
+        im = np.float32(flat[i].imag)
+        key = np.float32(np.float32(re * re) + np.float32(im * im))
+        pairs.append((-float(key), i))
+    pairs.sort()
+    return sorted(i for _, i in pairs[:k])
+
+
+def random_orthonormal(rng, n, r):
+    a = rng.standard_normal((n, r)) + 1j * rng.standard_normal((n, r))
+    q, _ = np.linalg.qr(a)
+    return q
