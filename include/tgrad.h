@@ -1,0 +1,186 @@
+/*
+ * tgrad.h -- C ABI of the B200 (sm_100a) TensorGRaD optimizer-step library.
+ *
+ * One state object per complex weight tensor W in C^{I_1 x ... x I_N}.  A step
+ * is Algorithm 1 of the paper ("Adam with Sparse and Low-Rank Gradient
+ * Compression"): the gradient is split into an unstructured sparse part
+ * (magnitude top-k index set Omega, Section 2.2 "Unstructured sparse gradient
+ * tensor") and a low-rank Tucker part (factor matrices U^(n), Section 2.2
+ * "Low-rank gradient tensor decomposition"); Adam runs on the k sparse values
+ * and on the Tucker core; the core is expanded back through the U^(n), the
+ * sparse update is scatter-added, and W is updated in place.
+ *
+ * Conventions
+ *  - All tensors are dense, row-major (last index fastest).  TGRAD_C64 stores
+ *    each entry as two fp32 (re, im); TGRAD_C32H as two IEEE fp16 (re, im)
+ *    (the paper's mixed-precision recipe, Section 2.3: weights and gradients in
+ *    half precision, every optimizer state in fp32).
+ *  - The caller passes grad = d(phi)/dW.  Algorithm 1 is written for
+ *    G = -grad and W <- W + eta*Gtilde(G); the library evaluates the same
+ *    stages on grad and subtracts, which is bit-identical.
+ *  - Pointers named d_* are DEVICE pointers, everything else is host memory.
+ *  - The library never allocates or frees device memory and never creates
+ *    streams.  The caller owns: the weight, the gradient, one persistent
+ *    block (Omega, U^(n), moments, status words) and one workspace block
+ *    (scratch; contents need not survive between calls, but the same
+ *    workspace must not be used by two states concurrently).  Sizes come
+ *    from tgrad_state_bytes().  Both blocks must be 256-byte aligned.
+ *  - All device work is enqueued asynchronously on the given stream
+ *    (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *  - Argument errors are detected on the host before anything is enqueued and
+ *    leave every buffer untouched.  Conditions found on the device (Jacobi
+ *    sweep cap reached, non-finite gradient seen by the selection) set sticky
+ *    bits that tgrad_query_status() reads.  Nothing aborts or traps.
+ *  - A state is not thread-safe; distinct states may be used from distinct
+ *    threads.
+ */
+#ifndef TGRAD_H_
+#define TGRAD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tgrad_state tgrad_state;   /* opaque host handle; owns no device memory */
+
+typedef enum {
+  TGRAD_OK = 0,
+  TGRAD_ERR_INVALID_ARG = 1,
+  TGRAD_ERR_UNSUPPORTED = 2,
+  TGRAD_ERR_BUFFER_TOO_SMALL = 3,
+  TGRAD_ERR_CUDA = 4,
+  TGRAD_ERR_NO_CONVERGE = 5,
+  TGRAD_ERR_NONFINITE = 6,
+  TGRAD_ERR_BAD_STATE = 7
+} tgrad_status;
+
+/* sticky device flags reported by tgrad_query_status() */
+#define TGRAD_FLAG_NO_CONVERGE 1   /* the Jacobi eigensolver hit jacobi_max_sweeps */
+#define TGRAD_FLAG_NONFINITE   2   /* a NaN/Inf magnitude was seen while selecting Omega */
+
+typedef enum {
+  TGRAD_C64 = 0,   /* interleaved 2 x fp32 */
+  TGRAD_C32H = 1   /* interleaved 2 x IEEE fp16 */
+} tgrad_dtype;
+
+#define TGRAD_MAX_NDIM 8
+
+/* Hyper-parameters of Algorithm 1 (its "Require" line) plus storage options. */
+typedef struct {
+  int32_t ndim;                     /* N, 3 <= ndim <= TGRAD_MAX_NDIM                          */
+  int64_t dims[TGRAD_MAX_NDIM];     /* I_1..I_N, row-major; prod(dims) < 2^32                   */
+  int32_t ranks[TGRAD_MAX_NDIM];    /* Tucker ranks, 1 <= r_n <= I_n                            */
+  int64_t k;                        /* |Omega| = ceil(rho*I), computed exactly by the caller    */
+  int32_t T;                        /* subspace change frequency, >= 1                          */
+  float lr;                         /* eta                                                      */
+  float alpha;                      /* scale of the reconstructed low-rank update               */
+  float lambda;                     /* scale of the sparse update                               */
+  float beta1, beta2, eps;          /* Adam decay rates and epsilon                             */
+  float weight_decay;               /* decoupled decay W <- (1 - eta*wd) W before the update    */
+  int32_t wg_dtype;                 /* tgrad_dtype of W and grad; all states are fp32           */
+  int32_t auto_refresh;             /* 1: tgrad_step refreshes Omega and U^(n) when t % T == 0  */
+  int32_t jacobi_max_sweeps;        /* sweep cap of the eigensolver (0 -> default 30)           */
+  float jacobi_tol;                 /* off-diagonal tolerance relative to max diag (0 -> 1e-6)  */
+} tgrad_config;
+
+/* Selectors for tgrad_export_state / tgrad_import_state.  FACTOR_BASE + n is
+ * U^(n+1), an I_n x r_n row-major complex64 matrix. */
+enum {
+  TGRAD_WHAT_OMEGA = 1,        /* k x uint32, strictly ascending flat indices */
+  TGRAD_WHAT_M_L = 2,          /* prod(r_n) x complex64, row-major core order */
+  TGRAD_WHAT_V_L = 3,          /* prod(r_n) x fp32                            */
+  TGRAD_WHAT_M_S = 4,          /* k x complex64, slot j <-> Omega[j]          */
+  TGRAD_WHAT_V_S = 5,          /* k x fp32                                    */
+  TGRAD_WHAT_CORE = 6,         /* last step's compressed gradient (export only; workspace) */
+  TGRAD_WHAT_N_L = 7,          /* last step's normalised core update (export only)         */
+  TGRAD_WHAT_N_S = 8,          /* last step's normalised sparse update (export only)       */
+  TGRAD_WHAT_GRAM_BASE = 32,   /* + n: A_n = R_(n) R_(n)^H of the last refresh, I_n x I_n complex64 (export only) */
+  TGRAD_WHAT_FACTOR_BASE = 64  /* + n */
+};
+
+/* Sizes of the two caller-owned device blocks for a configuration.
+ * Counts follow the state inventory of Algorithm 1 (its initialisation
+ * statements) and of the appendix "Parameter Complexity Analysis":
+ * prod(r_n) core-shaped entries for each low-rank moment, sum I_n r_n factor
+ * entries, k indices and k entries for each sparse moment. */
+tgrad_status tgrad_state_bytes(const tgrad_config* cfg, size_t* persistent_bytes, size_t* workspace_bytes);
+
+/* Algorithm 1 initialisation: t <- 0, M_L, V_L, M_S, V_S <- 0 (enqueued on
+ * the stream).  Omega and U^(n) are undefined until the first refresh.
+ * Returns a host handle in *out that refers to, but does not own, the two
+ * device blocks. */
+tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_t persistent_bytes,
+                              void* d_workspace, size_t workspace_bytes, void* cuda_stream, tgrad_state** out);
+
+/* One pass of the loop body of Algorithm 1 for one tensor: (refresh if
+ * auto_refresh and t mod T == 0), sparse gather, residual, Tucker compression
+ * (chained mode-n products with U^(n)H, Section 2.2), AdamUpdate on the sparse
+ * values and on the core, reconstruction scaled by alpha, scaled sparse add,
+ * W <- W - eta*Gtilde, t <- t+1.
+ * d_weight: in/out, prod(dims) entries of wg_dtype.  d_grad: input of the same
+ * shape and dtype; it is restored to its input value before the call's work
+ * completes, but is written temporarily during a refresh.
+ * Returns TGRAD_ERR_BAD_STATE if no refresh has happened yet and auto_refresh
+ * is 0. */
+tgrad_status tgrad_step(tgrad_state* st, void* d_weight, void* d_grad, void* cuda_stream);
+
+/* The `t mod T = 0` branch of Algorithm 1 on the supplied gradient:
+ * Omega <- magnitude top-k of grad (key = fp32 re*re + im*im without fused
+ * multiply-add, ties to the lower flat index, stored ascending);
+ * R <- grad with Omega zeroed; U^(n) <- eigenvectors of the r_n largest
+ * eigenvalues of R_(n) R_(n)^H (Jacobi), descending, each column scaled by the
+ * unit phase that makes its largest-modulus component real positive.
+ * Moments are not touched.  d_grad is modified while the call's work runs and
+ * restored at its end. */
+tgrad_status tgrad_refresh_subspace(tgrad_state* st, void* d_grad, void* cuda_stream);
+
+/* Batched variants over a list of layers: semantically n independent calls
+ * (the tensors of an FNO's spectral layers are independent).  Arrays are HOST
+ * arrays of handles / device pointers. */
+tgrad_status tgrad_step_batched(tgrad_state* const* states, void* const* d_weights, void* const* d_grads,
+                                int32_t n_tensors, void* cuda_stream);
+tgrad_status tgrad_refresh_subspace_batched(tgrad_state* const* states, void* const* d_grads, int32_t n_tensors,
+                                            void* cuda_stream);
+
+/* Synchronises the stream, then reports the sticky flags (TGRAD_FLAG_*), the
+ * step counter t and the number of Jacobi sweeps the last refresh used per
+ * mode (sweeps may be NULL; otherwise ndim int32). */
+tgrad_status tgrad_query_status(tgrad_state* st, void* cuda_stream, int32_t* sticky_flags, int64_t* t,
+                                int32_t* sweeps);
+
+/* Checkpoint / inspection: copy one state component to or from HOST memory.
+ * `bytes` must equal the component's size exactly.  Both calls synchronise the
+ * stream.  tgrad_set_step sets the counter t (host side). */
+tgrad_status tgrad_export_state(tgrad_state* st, int32_t what, void* host_dst, size_t bytes, void* cuda_stream);
+tgrad_status tgrad_import_state(tgrad_state* st, int32_t what, const void* host_src, size_t bytes,
+                                void* cuda_stream);
+tgrad_status tgrad_set_step(tgrad_state* st, int64_t t);
+
+/* Frees the host handle only. */
+tgrad_status tgrad_destroy_state(tgrad_state* st);
+
+const char* tgrad_status_string(tgrad_status s);
+
+/* Kernels launched by this library since it was loaded (host-side counter). */
+int64_t tgrad_launch_count(void);
+
+/* Optional per-stage device timing of tgrad_step (CUDA events recorded on the
+ * caller's stream between the stages of a non-refresh step).  Stages, in
+ * order: 0 trailing-mode compression fused with the sparse gather/Adam
+ * (streams grad), 1 remaining mode products of the compression, 2 Adam on the
+ * core, 3 leading mode products of the reconstruction, 4 trailing-mode
+ * reconstruction fused with the weight update and sparse add (streams W).
+ * tgrad_get_stage_times synchronises the stream and returns, for the steps
+ * since the last call (at most the 64 most recent), the summed milliseconds
+ * per stage in ms_sum[5] and the number of steps in *n_steps. */
+#define TGRAD_NUM_STAGES 5
+tgrad_status tgrad_set_stage_timing(tgrad_state* st, int32_t enable);
+tgrad_status tgrad_get_stage_times(tgrad_state* st, void* cuda_stream, float* ms_sum, int32_t* n_steps);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TGRAD_H_ */

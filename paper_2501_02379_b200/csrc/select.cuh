@@ -1,0 +1,244 @@
+// Magnitude top-k selection of the sparse index set Omega
+// (SparseIndices with the top-k strategy, Section 2.2 "Unstructured sparse
+// gradient tensor"): radix select on the fp32 bit pattern of |g|^2, then an
+// ordered compaction that writes Omega ascending.  Ties at the threshold key
+// go to the lower flat index.  Everything is integer work after the key, and
+// no result depends on the order in which atomics land.
+#pragma once
+#include "common.cuh"
+
+namespace tg {
+
+struct SelState {
+  uint32_t prefix;   // key bits fixed so far (high bits)
+  uint32_t krem;     // rank still to resolve inside the current prefix bucket
+  uint32_t thr;      // final threshold key (valid after the last pass)
+  uint32_t take_eq;  // how many entries with key == thr belong to Omega
+};
+
+// three passes over the 32 key bits: 11 + 11 + 10
+__host__ __device__ inline int sel_bits(int pass) { return pass == 2 ? 10 : 11; }
+__host__ __device__ inline int sel_shift(int pass) { return pass == 0 ? 21 : (pass == 1 ? 10 : 0); }
+constexpr int kSelMaxBins = 2048;
+constexpr int kChunk = 2048;        // elements per compaction block
+constexpr int kChunkThreads = 256;  // 8 consecutive elements per thread
+
+__global__ void sel_init_kernel(SelState* st, uint32_t k) {
+  st->prefix = 0u; st->krem = k; st->thr = 0u; st->take_eq = 0u;
+}
+
+// Histogram of the current digit over all entries whose higher bits equal the
+// prefix chosen so far.
+template <class S>
+__global__ void __launch_bounds__(512) sel_hist_kernel(const void* __restrict__ g, uint32_t n, int pass,
+                                                      const SelState* __restrict__ st, uint32_t* __restrict__ hist,
+                                                      int* __restrict__ flags) {
+  __shared__ uint32_t sh[kSelMaxBins];
+  const int bits = sel_bits(pass), shift = sel_shift(pass);
+  const uint32_t nb = 1u << bits;
+  for (uint32_t i = threadIdx.x; i < nb; i += blockDim.x) sh[i] = 0u;
+  __syncthreads();
+  const uint32_t prefix = st->prefix;
+  const uint32_t hi_mask = (pass == 0) ? 0u : (0xffffffffu << (shift + bits));
+  bool bad = false;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  // block-uniform loop bound, so every warp stays converged for the warp votes below
+  for (uint64_t b0 = (uint64_t)blockIdx.x * blockDim.x; b0 < n; b0 += stride) {
+    const uint64_t i = b0 + threadIdx.x;
+    const bool valid = i < n;
+    uint32_t key = valid ? mag_key(S::load(g, i)) : 0u;
+    if (pass == 0 && (key & 0x7f800000u) == 0x7f800000u) bad = true;
+    bool in = valid && (key & hi_mask) == prefix;
+    uint32_t d = (key >> shift) & (nb - 1u);
+    // warp-aggregated shared atomics: gradients crowd into a few exponent bins
+    unsigned act = __ballot_sync(0xffffffffu, in);
+    if (in) {
+      unsigned peers = __match_any_sync(act, d);
+      if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&sh[d], (uint32_t)__popc(peers));
+    }
+  }
+  __syncthreads();
+  for (uint32_t i = threadIdx.x; i < nb; i += blockDim.x) {
+    uint32_t c = sh[i];
+    if (c) atomicAdd(&hist[i], c);
+  }
+  if (bad) atomicOr(flags, 2);
+}
+
+// Walk the histogram from the largest digit down until the cumulative count
+// reaches the wanted rank; fix that digit in the prefix.
+__global__ void __launch_bounds__(1024) sel_pick_kernel(const uint32_t* __restrict__ hist, int pass, SelState* st) {
+  __shared__ uint32_t sc[kSelMaxBins];
+  __shared__ uint32_t wsum[32];
+  const int bits = sel_bits(pass), shift = sel_shift(pass);
+  const int nb = 1 << bits;
+  const int t = threadIdx.x;
+  // reversed order: position p <-> digit nb-1-p; two consecutive positions per thread
+  uint32_t a0 = (2 * t < nb) ? hist[nb - 1 - 2 * t] : 0u;
+  uint32_t a1 = (2 * t + 1 < nb) ? hist[nb - 2 - 2 * t] : 0u;
+  uint32_t s = a0 + a1, incl = s;
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+    if ((t & 31) >= o) incl += v;
+  }
+  if ((t & 31) == 31) wsum[t >> 5] = incl;
+  __syncthreads();
+  if (t < 32) {
+    uint32_t w = wsum[t], wi = w;
+    for (int o = 1; o < 32; o <<= 1) {
+      uint32_t v = __shfl_up_sync(0xffffffffu, wi, o);
+      if (t >= o) wi += v;
+    }
+    wsum[t] = wi - w;   // exclusive
+  }
+  __syncthreads();
+  uint32_t excl = wsum[t >> 5] + incl - s;
+  if (2 * t < nb) sc[2 * t] = excl + a0;            // inclusive cumulative counts, descending digits
+  if (2 * t + 1 < nb) sc[2 * t + 1] = excl + a0 + a1;
+  __syncthreads();
+  const uint32_t krem = st->krem;
+  __syncthreads();   // everyone has read krem before the one matching thread rewrites it
+  for (int p = t; p < nb; p += blockDim.x) {
+    uint32_t cur = sc[p], prev = p ? sc[p - 1] : 0u;
+    if (prev < krem && krem <= cur) {               // exactly one p satisfies this when krem >= 1
+      uint32_t d = (uint32_t)(nb - 1 - p);
+      uint32_t np = st->prefix | (d << shift);
+      st->prefix = np;
+      st->krem = krem - prev;
+      if (pass == 2) { st->thr = np; st->take_eq = krem - prev; }
+    }
+  }
+}
+
+// Per block of kChunk consecutive entries: how many keys lie above / at the threshold.
+template <class S>
+__global__ void __launch_bounds__(kChunkThreads) sel_count_kernel(const void* __restrict__ g, uint32_t n,
+                                                                  const SelState* __restrict__ st,
+                                                                  uint32_t* __restrict__ blk_gt,
+                                                                  uint32_t* __restrict__ blk_eq) {
+  __shared__ uint32_t sg[kChunkThreads / 32], se[kChunkThreads / 32];
+  const uint32_t thr = st->thr;
+  const uint32_t base = blockIdx.x * (uint32_t)kChunk;
+  uint32_t cg = 0, ce = 0;
+  // coalesced order here: only totals matter
+  for (int r = 0; r < kChunk / kChunkThreads; ++r) {
+    uint32_t i = base + r * kChunkThreads + threadIdx.x;
+    if (i < n) {
+      uint32_t key = mag_key(S::load(g, i));
+      cg += key > thr; ce += key == thr;
+    }
+  }
+  for (int o = 16; o; o >>= 1) { cg += __shfl_xor_sync(0xffffffffu, cg, o); ce += __shfl_xor_sync(0xffffffffu, ce, o); }
+  if ((threadIdx.x & 31) == 0) { sg[threadIdx.x >> 5] = cg; se[threadIdx.x >> 5] = ce; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t a = 0, b = 0;
+    for (int w = 0; w < kChunkThreads / 32; ++w) { a += sg[w]; b += se[w]; }
+    blk_gt[blockIdx.x] = a; blk_eq[blockIdx.x] = b;
+  }
+}
+
+// In-place exclusive scan of the per-block counts (single block).
+__global__ void __launch_bounds__(1024) sel_scan_kernel(uint32_t* __restrict__ blk_gt, uint32_t* __restrict__ blk_eq,
+                                                       uint32_t nblk) {
+  __shared__ uint32_t wg[32], we[32];
+  __shared__ uint32_t carry_g, carry_e;
+  const int t = threadIdx.x;
+  if (t == 0) { carry_g = 0; carry_e = 0; }
+  __syncthreads();
+  for (uint32_t base = 0; base < nblk; base += 1024) {
+    uint32_t i = base + t;
+    uint32_t g = (i < nblk) ? blk_gt[i] : 0u, e = (i < nblk) ? blk_eq[i] : 0u;
+    uint32_t ig = g, ie = e;
+    for (int o = 1; o < 32; o <<= 1) {
+      uint32_t vg = __shfl_up_sync(0xffffffffu, ig, o), ve = __shfl_up_sync(0xffffffffu, ie, o);
+      if ((t & 31) >= o) { ig += vg; ie += ve; }
+    }
+    if ((t & 31) == 31) { wg[t >> 5] = ig; we[t >> 5] = ie; }
+    __syncthreads();
+    if (t < 32) {
+      uint32_t a = wg[t], b = we[t], ia = a, ib = b;
+      for (int o = 1; o < 32; o <<= 1) {
+        uint32_t va = __shfl_up_sync(0xffffffffu, ia, o), vb = __shfl_up_sync(0xffffffffu, ib, o);
+        if (t >= o) { ia += va; ib += vb; }
+      }
+      wg[t] = ia - a; we[t] = ib - b;
+    }
+    __syncthreads();
+    uint32_t cg = carry_g, ce = carry_e;
+    uint32_t xg = cg + wg[t >> 5] + ig - g, xe = ce + we[t >> 5] + ie - e;
+    if (i < nblk) { blk_gt[i] = xg; blk_eq[i] = xe; }
+    __syncthreads();
+    if (t == 1023) { carry_g = xg + g; carry_e = xe + e; }
+    __syncthreads();
+  }
+}
+
+// Ordered compaction: entry i belongs to Omega iff key > thr, or key == thr and
+// fewer than take_eq equal keys precede it.  Its slot is the number of selected
+// entries before it, so Omega comes out strictly ascending.  The selected values
+// are saved to g_s (fp32 complex) for the residual/restore passes of the refresh.
+template <class S>
+__global__ void __launch_bounds__(kChunkThreads) sel_compact_kernel(const void* __restrict__ g, uint32_t n,
+                                                                    const SelState* __restrict__ st,
+                                                                    const uint32_t* __restrict__ blk_gt,
+                                                                    const uint32_t* __restrict__ blk_eq,
+                                                                    uint32_t* __restrict__ omega,
+                                                                    cf* __restrict__ g_s, uint32_t k) {
+  __shared__ uint32_t wsum[kChunkThreads / 32];
+  constexpr int EPT = kChunk / kChunkThreads;   // 8 consecutive entries per thread
+  const uint32_t thr = st->thr, take = st->take_eq;
+  const uint32_t base = blockIdx.x * (uint32_t)kChunk + threadIdx.x * EPT;
+  cf v[EPT];
+  uint32_t key[EPT];
+  uint32_t cnt = 0;   // packed: eq count in the high half, gt count in the low half
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    uint32_t i = base + e;
+    if (i < n) { v[e] = S::load(g, i); key[e] = mag_key(v[e]); } else { v[e] = make_float2(0.f, 0.f); key[e] = 0u; }
+    bool valid = i < n;
+    cnt += (valid && key[e] > thr) ? 1u : 0u;
+    cnt += (valid && key[e] == thr) ? 0x10000u : 0u;
+  }
+  uint32_t incl = cnt;
+  const int t = threadIdx.x;
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t u = __shfl_up_sync(0xffffffffu, incl, o);
+    if ((t & 31) >= o) incl += u;
+  }
+  if ((t & 31) == 31) wsum[t >> 5] = incl;
+  __syncthreads();
+  uint32_t woff = 0;
+  for (int w = 0; w < (t >> 5); ++w) woff += wsum[w];
+  uint32_t excl = woff + incl - cnt;
+  uint32_t gt_before = blk_gt[blockIdx.x] + (excl & 0xffffu);
+  uint32_t eq_before = blk_eq[blockIdx.x] + (excl >> 16);
+#pragma unroll
+  for (int e = 0; e < EPT; ++e) {
+    uint32_t i = base + e;
+    if (i >= n) break;
+    bool isgt = key[e] > thr, iseq = key[e] == thr;
+    bool sel = isgt || (iseq && eq_before < take);
+    if (sel) {
+      uint32_t pos = gt_before + (eq_before < take ? eq_before : take);
+      if (pos < k) { omega[pos] = i; g_s[pos] = v[e]; }
+    }
+    gt_before += isgt; eq_before += iseq;
+  }
+}
+
+// R = G - Sparse(G, Omega): zero the entries at Omega in place ...
+template <class S>
+__global__ void scatter_zero_kernel(void* __restrict__ g, const uint32_t* __restrict__ omega, uint32_t k) {
+  uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < k) S::store(g, omega[j], make_float2(0.f, 0.f));
+}
+// ... and put the saved values back once the factor matrices are computed.
+template <class S>
+__global__ void scatter_restore_kernel(void* __restrict__ g, const uint32_t* __restrict__ omega,
+                                       const cf* __restrict__ g_s, uint32_t k) {
+  uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < k) S::store(g, omega[j], g_s[j]);
+}
+
+}  // namespace tg

@@ -1,0 +1,609 @@
+// Host side of the C ABI: state layout, argument checks, stage scheduling on the
+// caller's stream.  Every step of the path runs in the kernels of this library;
+// there is no CPU or library fallback.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "../../include/tgrad.h"
+#include "common.cuh"
+#include "gram.cuh"
+#include "jacobi.cuh"
+#include "modeprod.cuh"
+#include "select.cuh"
+#include "tail.cuh"
+
+using namespace tg;
+
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+
+constexpr int kStages = 5;   // proj_tail, proj_chain, adam_core, back_chain, back_tail
+constexpr int kTimingRing = 64;
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+struct Layout {
+  // persistent block
+  size_t p_flags, p_omega, p_factor[TGRAD_MAX_NDIM], p_ml, p_vl, p_ms, p_vs, p_total;
+  // workspace block
+  size_t w_ns, w_gs, w_core, w_nl, w_bufa, w_bufb, w_sel, w_hist, w_blk, w_gram[TGRAD_MAX_NDIM], w_jac[TGRAD_MAX_NDIM],
+      w_v[TGRAD_MAX_NDIM], w_partial, w_total;
+  uint64_t numel, P, tsize;   // entries, core entries, entries of the tail-contracted tensor
+  uint32_t nblk;              // compaction blocks
+  int gram_splits[TGRAD_MAX_NDIM];
+  uint32_t gram_chunks[TGRAD_MAX_NDIM], gram_cps[TGRAD_MAX_NDIM];
+};
+
+struct TailPlan {
+  int rpl, rbp, nwarps, grid;
+  size_t smem_proj, smem_back;
+};
+
+tgrad_status validate(const tgrad_config* c) {
+  if (!c) return TGRAD_ERR_INVALID_ARG;
+  if (c->ndim < 2 || c->ndim > TGRAD_MAX_NDIM) return TGRAD_ERR_INVALID_ARG;
+  long double tot = 1;
+  for (int n = 0; n < c->ndim; ++n) {
+    if (c->dims[n] < 1) return TGRAD_ERR_INVALID_ARG;
+    if (c->ranks[n] < 1 || c->ranks[n] > c->dims[n]) return TGRAD_ERR_INVALID_ARG;
+    tot *= (long double)c->dims[n];
+  }
+  if (c->k < 0 || (long double)c->k > tot) return TGRAD_ERR_INVALID_ARG;
+  if (c->T < 1) return TGRAD_ERR_INVALID_ARG;
+  if (c->wg_dtype != TGRAD_C64 && c->wg_dtype != TGRAD_C32H) return TGRAD_ERR_INVALID_ARG;
+  if (!(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps >= 0.f))
+    return TGRAD_ERR_INVALID_ARG;
+  if (c->jacobi_max_sweeps < 0 || c->jacobi_tol < 0.f) return TGRAD_ERR_INVALID_ARG;
+  // limits of this implementation
+  if (c->ndim < 3) return TGRAD_ERR_UNSUPPORTED;             // the matrix case is not built
+  if (tot >= 4294967296.0L) return TGRAD_ERR_UNSUPPORTED;    // flat indices are uint32
+  for (int n = 0; n < c->ndim; ++n)
+    if (c->dims[n] > JAC_MAX_N) return TGRAD_ERR_UNSUPPORTED;
+  if (c->ranks[c->ndim - 1] > 32) return TGRAD_ERR_UNSUPPORTED;
+  return TGRAD_OK;
+}
+
+int pick_rbp(int rb) { return rb <= 4 ? 4 : rb <= 8 ? 8 : rb <= 16 ? 16 : 32; }
+
+void plan_gram(const tgrad_config* c, int n, int sm, uint32_t& chunks, uint32_t& cps, int& splits) {
+  uint64_t O = 1, C = 1;
+  for (int m = 0; m < n; ++m) O *= c->dims[m];
+  for (int m = n + 1; m < c->ndim; ++m) C *= c->dims[m];
+  uint64_t total = (C == 1) ? (O + GR_KT - 1) / GR_KT : O * ((C + GR_KT - 1) / GR_KT);
+  int T = (int)((c->dims[n] + GR_T - 1) / GR_T);
+  int tiles = T * (T + 1) / 2;
+  uint64_t want = (uint64_t)(4 * sm + tiles - 1) / tiles;
+  if (want < 1) want = 1;
+  if (want > 256) want = 256;
+  if (want > total) want = total;
+  uint64_t per = (total + want - 1) / want;
+  chunks = (uint32_t)total; cps = (uint32_t)per; splits = (int)((total + per - 1) / per);
+}
+
+tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
+  tgrad_status s = validate(c);
+  if (s != TGRAD_OK) return s;
+  const int N = c->ndim;
+  uint64_t numel = 1, P = 1;
+  for (int n = 0; n < N; ++n) { numel *= (uint64_t)c->dims[n]; P *= (uint64_t)c->ranks[n]; }
+  L.numel = numel; L.P = P;
+  uint64_t S = numel / ((uint64_t)c->dims[N - 1] * c->dims[N - 2]);
+  L.tsize = S * c->ranks[N - 1] * c->ranks[N - 2];
+  const uint64_t k = (uint64_t)c->k;
+  size_t o = 0;
+  L.p_flags = o; o = align_up(o + 64 * sizeof(int));
+  L.p_omega = o; o = align_up(o + k * 4);
+  for (int n = 0; n < N; ++n) { L.p_factor[n] = o; o = align_up(o + (size_t)c->dims[n] * c->ranks[n] * 8); }
+  L.p_ml = o; o = align_up(o + P * 8);
+  L.p_vl = o; o = align_up(o + P * 4);
+  L.p_ms = o; o = align_up(o + k * 8);
+  L.p_vs = o; o = align_up(o + k * 4);
+  L.p_total = o;
+  o = 0;
+  L.w_ns = o; o = align_up(o + k * 8);
+  L.w_gs = o; o = align_up(o + k * 8);
+  L.w_core = o; o = align_up(o + P * 8);
+  L.w_nl = o; o = align_up(o + P * 8);
+  L.w_bufa = o; o = align_up(o + L.tsize * 8);
+  L.w_bufb = o; o = align_up(o + L.tsize * 8);
+  L.w_sel = o; o = align_up(o + sizeof(SelState));
+  L.w_hist = o; o = align_up(o + 3 * kSelMaxBins * 4);
+  L.nblk = (uint32_t)((numel + kChunk - 1) / kChunk);
+  L.w_blk = o; o = align_up(o + (size_t)2 * L.nblk * 4);
+  size_t partial = 0;
+  for (int n = 0; n < N; ++n) {
+    size_t sq = (size_t)c->dims[n] * c->dims[n] * 8;
+    L.w_gram[n] = o; o = align_up(o + sq);   // A_n, kept for inspection
+    L.w_jac[n] = o; o = align_up(o + sq);    // working copy the solver diagonalises
+    L.w_v[n] = o; o = align_up(o + sq);      // accumulated rotations
+    plan_gram(c, n, sm, L.gram_chunks[n], L.gram_cps[n], L.gram_splits[n]);
+    size_t pb = sq * L.gram_splits[n];
+    if (pb > partial) partial = pb;
+  }
+  L.w_partial = o; o = align_up(o + partial);
+  L.w_total = o;
+  return TGRAD_OK;
+}
+
+}  // namespace
+
+struct tgrad_state {
+  tgrad_config cfg;
+  Layout L;
+  char* dp;
+  char* dw;
+  int64_t t;
+  bool have_subspace;
+  int sm_count;
+  TailPlan tail;
+  // optional per-stage timing
+  bool timing;
+  int timing_steps;
+  cudaEvent_t ev[kTimingRing][kStages + 1];
+};
+
+namespace {
+
+#define TG_LAUNCH_CHECK()                                  \
+  do {                                                     \
+    g_launches.fetch_add(1, std::memory_order_relaxed);    \
+    if (cudaPeekAtLastError() != cudaSuccess) return TGRAD_ERR_CUDA; \
+  } while (0)
+
+template <class S, int RPL, int RBP>
+tgrad_status tail_attr(const TailPlan& tp) {
+  if (cudaFuncSetAttribute(proj_tail_kernel<S, RPL, RBP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)tp.smem_proj) != cudaSuccess) return TGRAD_ERR_CUDA;
+  if (cudaFuncSetAttribute(back_tail_kernel<S, RPL, RBP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)tp.smem_back) != cudaSuccess) return TGRAD_ERR_CUDA;
+  return TGRAD_OK;
+}
+
+template <class S, int RPL, int RBP>
+tgrad_status tail_launch(bool back, const TailPlan& tp, void* ptr, const TailParams& p, cudaStream_t st) {
+  if (back) back_tail_kernel<S, RPL, RBP><<<tp.grid, tp.nwarps * 32, tp.smem_back, st>>>(ptr, p);
+  else proj_tail_kernel<S, RPL, RBP><<<tp.grid, tp.nwarps * 32, tp.smem_proj, st>>>(ptr, p);
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
+}
+
+// op: 0 = set attributes, 1 = proj, 2 = back
+template <class S>
+tgrad_status tail_dispatch(int op, const TailPlan& tp, void* ptr, const TailParams& p, cudaStream_t st) {
+#define TG_CASE(RPL_, RBP_)                                                     \
+  if (tp.rpl == RPL_ && tp.rbp == RBP_) {                                       \
+    if (op == 0) return tail_attr<S, RPL_, RBP_>(tp);                           \
+    return tail_launch<S, RPL_, RBP_>(op == 2, tp, ptr, p, st);                 \
+  }
+  TG_CASE(1, 4) TG_CASE(2, 4) TG_CASE(4, 4) TG_CASE(1, 8) TG_CASE(2, 8) TG_CASE(1, 16) TG_CASE(1, 32)
+#undef TG_CASE
+  return TGRAD_ERR_UNSUPPORTED;
+}
+
+tgrad_status tail_any(const tgrad_state* s, int op, void* ptr, const TailParams& p, cudaStream_t st) {
+  return s->cfg.wg_dtype == TGRAD_C64 ? tail_dispatch<StoreC64>(op, s->tail, ptr, p, st)
+                                      : tail_dispatch<StoreC32H>(op, s->tail, ptr, p, st);
+}
+
+tgrad_status plan_tail(tgrad_state* s) {
+  const tgrad_config& c = s->cfg;
+  const int N = c.ndim;
+  const int A = (int)c.dims[N - 2], B = (int)c.dims[N - 1], ra = c.ranks[N - 2], rb = c.ranks[N - 1];
+  TailPlan& tp = s->tail;
+  tp.rbp = pick_rbp(rb);
+  int rows = (A + 31) / 32, cap = 16 / tp.rbp; if (cap < 1) cap = 1;
+  int rpl = rows < cap ? rows : cap;
+  tp.rpl = rpl >= 4 ? 4 : rpl >= 2 ? 2 : 1;
+  const int Bs = B | 1, ras = ra | 1;
+  const size_t kMax = 227 * 1024;
+  int nw = 0;
+  const int cand[4] = {8, 4, 2, 1};
+  const size_t lim[3] = {56 * 1024, 113 * 1024, kMax};
+  for (int li = 0; li < 3 && !nw; ++li)
+    for (int ci = (li == 0 ? 0 : 1); ci < 4; ++ci) {
+      size_t a = tail_smem_bytes(A, B, Bs, ra, ras, tp.rbp, cand[ci], false);
+      size_t b = tail_smem_bytes(A, B, Bs, ra, ras, tp.rbp, cand[ci], true);
+      if ((a > b ? a : b) <= lim[li]) { nw = cand[ci]; break; }
+    }
+  if (!nw) return TGRAD_ERR_UNSUPPORTED;   // a trailing A x B slab does not fit in shared memory
+  tp.nwarps = nw;
+  tp.smem_proj = tail_smem_bytes(A, B, Bs, ra, ras, tp.rbp, nw, false);
+  tp.smem_back = tail_smem_bytes(A, B, Bs, ra, ras, tp.rbp, nw, true);
+  size_t sm = tp.smem_proj > tp.smem_back ? tp.smem_proj : tp.smem_back;
+  int per_sm = (int)(kMax / (sm + 1024)); if (per_sm < 1) per_sm = 1;
+  int by_threads = 2048 / (nw * 32); if (per_sm > by_threads) per_sm = by_threads;
+  if (per_sm > 16) per_sm = 16;
+  uint64_t S = s->L.numel / ((uint64_t)A * B);
+  uint64_t need = (S + nw - 1) / nw;
+  uint64_t g = (uint64_t)s->sm_count * per_sm;
+  tp.grid = (int)(need < g ? need : g);
+  TailParams dummy; memset(&dummy, 0, sizeof(dummy));
+  return tail_any(s, 0, nullptr, dummy, 0);
+}
+
+AdamScalars adam_scalars(const tgrad_config& c, int64_t t) {
+  AdamScalars a;
+  a.beta1 = c.beta1; a.beta2 = c.beta2;
+  a.omb1 = 1.0f - c.beta1; a.omb2 = 1.0f - c.beta2;
+  float c1 = (float)(1.0 - std::pow((double)c.beta1, (double)(t + 1)));
+  float c2 = (float)(1.0 - std::pow((double)c.beta2, (double)(t + 1)));
+  a.inv_c1 = 1.0f / c1; a.inv_c2 = 1.0f / c2;
+  a.eps = c.eps;
+  return a;
+}
+
+template <class S>
+tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
+  const tgrad_config& c = s->cfg;
+  const Layout& L = s->L;
+  const int N = c.ndim;
+  const uint32_t n = (uint32_t)L.numel, k = (uint32_t)c.k;
+  int* flags = reinterpret_cast<int*>(s->dp + L.p_flags);
+  uint32_t* omega = reinterpret_cast<uint32_t*>(s->dp + L.p_omega);
+  cf* g_s = reinterpret_cast<cf*>(s->dw + L.w_gs);
+  if (k > 0) {
+    SelState* sel = reinterpret_cast<SelState*>(s->dw + L.w_sel);
+    uint32_t* hist = reinterpret_cast<uint32_t*>(s->dw + L.w_hist);
+    uint32_t* blk_gt = reinterpret_cast<uint32_t*>(s->dw + L.w_blk);
+    uint32_t* blk_eq = blk_gt + L.nblk;
+    if (cudaMemsetAsync(hist, 0, 3 * kSelMaxBins * 4, st) != cudaSuccess) return TGRAD_ERR_CUDA;
+    sel_init_kernel<<<1, 1, 0, st>>>(sel, k); TG_LAUNCH_CHECK();
+    uint64_t want = ((uint64_t)n + 511) / 512;
+    int hgrid = (int)(want < (uint64_t)s->sm_count * 8 ? want : (uint64_t)s->sm_count * 8);
+    for (int pass = 0; pass < 3; ++pass) {
+      sel_hist_kernel<S><<<hgrid, 512, 0, st>>>(d_grad, n, pass, sel, hist + pass * kSelMaxBins, flags);
+      TG_LAUNCH_CHECK();
+      sel_pick_kernel<<<1, 1024, 0, st>>>(hist + pass * kSelMaxBins, pass, sel); TG_LAUNCH_CHECK();
+    }
+    sel_count_kernel<S><<<L.nblk, kChunkThreads, 0, st>>>(d_grad, n, sel, blk_gt, blk_eq); TG_LAUNCH_CHECK();
+    sel_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, L.nblk); TG_LAUNCH_CHECK();
+    sel_compact_kernel<S><<<L.nblk, kChunkThreads, 0, st>>>(d_grad, n, sel, blk_gt, blk_eq, omega, g_s, k);
+    TG_LAUNCH_CHECK();
+    scatter_zero_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, k); TG_LAUNCH_CHECK();
+  }
+  cf* partial = reinterpret_cast<cf*>(s->dw + L.w_partial);
+  JacobiParams jp; memset(&jp, 0, sizeof(jp));
+  for (int m = 0; m < N; ++m) {
+    uint64_t O = 1, C = 1;
+    for (int q = 0; q < m; ++q) O *= c.dims[q];
+    for (int q = m + 1; q < N; ++q) C *= c.dims[q];
+    const int In = (int)c.dims[m];
+    const int T = (In + GR_T - 1) / GR_T;
+    cf* A = reinterpret_cast<cf*>(s->dw + L.w_gram[m]);
+    dim3 grid(T * T, L.gram_splits[m]);
+    gram_partial_kernel<S><<<grid, 256, 0, st>>>(d_grad, In, (uint32_t)O, (uint32_t)C, L.gram_chunks[m],
+                                                 L.gram_cps[m], partial);
+    TG_LAUNCH_CHECK();
+    gram_reduce_kernel<<<(In * In + 255) / 256, 256, 0, st>>>(partial, L.gram_splits[m], In, A); TG_LAUNCH_CHECK();
+    jp.mode[m].A = reinterpret_cast<cf*>(s->dw + L.w_jac[m]);
+    jp.mode[m].V = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
+    jp.mode[m].U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
+    jp.mode[m].n = In; jp.mode[m].r = c.ranks[m];
+    if (cudaMemcpyAsync(s->dw + L.w_jac[m], A, (size_t)In * In * 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return TGRAD_ERR_CUDA;
+  }
+  if (k > 0) { scatter_restore_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, g_s, k); TG_LAUNCH_CHECK(); }
+  jp.max_sweeps = c.jacobi_max_sweeps > 0 ? c.jacobi_max_sweeps : 30;
+  jp.tol = c.jacobi_tol > 0.f ? c.jacobi_tol : 1e-6f;
+  jp.flags = flags;
+  jacobi_kernel<<<N, JAC_THREADS, 0, st>>>(jp); TG_LAUNCH_CHECK();
+  s->have_subspace = true;
+  return TGRAD_OK;
+}
+
+tgrad_status do_refresh(tgrad_state* s, void* d_grad, cudaStream_t st) {
+  return s->cfg.wg_dtype == TGRAD_C64 ? refresh_impl<StoreC64>(s, d_grad, st) : refresh_impl<StoreC32H>(s, d_grad, st);
+}
+
+tgrad_status mode_product(bool conj_t, const cf* in, cf* out, const cf* U, uint64_t O, int M, int K, uint64_t C,
+                          int r_n, cudaStream_t st) {
+  dim3 grid((unsigned)((C + MP_BC - 1) / MP_BC), (unsigned)((M + MP_BM - 1) / MP_BM), (unsigned)O);
+  if (conj_t) mode_product_kernel<true><<<grid, 256, 0, st>>>(in, out, U, M, K, (int)C, r_n);
+  else mode_product_kernel<false><<<grid, 256, 0, st>>>(in, out, U, M, K, (int)C, r_n);
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
+}
+
+#define TG_TRY(x) do { tgrad_status _s = (x); if (_s != TGRAD_OK) return _s; } while (0)
+#define TG_MARK(i) do { if (evs) cudaEventRecord(evs[i], st); } while (0)
+
+tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t st) {
+  const tgrad_config& c = s->cfg;
+  const Layout& L = s->L;
+  const int N = c.ndim;
+  if (c.auto_refresh && (s->t % c.T) == 0) TG_TRY(do_refresh(s, d_grad, st));
+  if (!s->have_subspace) return TGRAD_ERR_BAD_STATE;
+  cudaEvent_t* evs = s->timing ? s->ev[s->timing_steps % kTimingRing] : nullptr;
+
+  const int A = (int)c.dims[N - 2], B = (int)c.dims[N - 1], ra = c.ranks[N - 2], rb = c.ranks[N - 1];
+  TailParams p; memset(&p, 0, sizeof(p));
+  p.A = A; p.B = B; p.Bs = B | 1; p.ra = ra; p.rb = rb; p.ras = ra | 1;
+  p.E = (uint32_t)((uint64_t)A * B); p.nslab = (uint32_t)(L.numel / p.E);
+  p.Ua = reinterpret_cast<const cf*>(s->dp + L.p_factor[N - 2]);
+  p.Ub = reinterpret_cast<const cf*>(s->dp + L.p_factor[N - 1]);
+  p.omega = reinterpret_cast<const uint32_t*>(s->dp + L.p_omega);
+  p.k = (int)c.k;
+  p.m_s = reinterpret_cast<cf*>(s->dp + L.p_ms);
+  p.v_s = reinterpret_cast<float*>(s->dp + L.p_vs);
+  p.n_s = reinterpret_cast<cf*>(s->dw + L.w_ns);
+  p.g_s = reinterpret_cast<cf*>(s->dw + L.w_gs);
+  p.adam = adam_scalars(c, s->t);
+  p.s_low = (float)((double)c.lr * (double)c.alpha);
+  p.s_sparse = (float)((double)c.lr * (double)c.lambda);
+  p.decay = (float)(1.0 - (double)c.lr * (double)c.weight_decay);
+  cf* bufa = reinterpret_cast<cf*>(s->dw + L.w_bufa);
+  cf* bufb = reinterpret_cast<cf*>(s->dw + L.w_bufb);
+  cf* core = reinterpret_cast<cf*>(s->dw + L.w_core);
+  cf* n_l = reinterpret_cast<cf*>(s->dw + L.w_nl);
+
+  // low-rank compression: trailing two modes while streaming G, then modes N-2 .. 1
+  TG_MARK(0);
+  p.t = bufa;
+  TG_TRY(tail_any(s, 1, d_grad, p, st));
+  TG_MARK(1);
+  {
+    cf* cur = bufa; cf* nxt = bufb;
+    uint64_t C = (uint64_t)ra * rb;
+    for (int m = N - 3; m >= 0; --m) {
+      uint64_t O = 1;
+      for (int q = 0; q < m; ++q) O *= c.dims[q];
+      cf* dst = (m == 0) ? core : nxt;
+      TG_TRY(mode_product(true, cur, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[m]), O, c.ranks[m],
+                          (int)c.dims[m], C, c.ranks[m], st));
+      C *= c.ranks[m];
+      cf* tmp = cur; cur = nxt; nxt = tmp;
+    }
+  }
+  TG_MARK(2);
+  adam_core_kernel<<<(unsigned)((L.P + 255) / 256), 256, 0, st>>>(
+      core, reinterpret_cast<cf*>(s->dp + L.p_ml), reinterpret_cast<float*>(s->dp + L.p_vl), n_l, (uint32_t)L.P, p.adam);
+  TG_LAUNCH_CHECK();
+  TG_MARK(3);
+  // reconstruction: modes 1 .. N-2 on the small tensor, trailing two while streaming W
+  const cf* tprime;
+  {
+    const cf* cur = n_l;
+    cf* bufs[2] = {bufa, bufb};
+    int which = ((N - 2) & 1) ? 0 : 1;          // make the last product land in bufa
+    uint64_t O = 1;
+    for (int m = 0; m <= N - 3; ++m) {
+      uint64_t C = (uint64_t)ra * rb;
+      for (int q = m + 1; q <= N - 3; ++q) C *= c.ranks[q];
+      cf* dst = bufs[which];
+      TG_TRY(mode_product(false, cur, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[m]), O, (int)c.dims[m],
+                          c.ranks[m], C, c.ranks[m], st));
+      O *= c.dims[m];
+      cur = dst; which ^= 1;
+    }
+    tprime = cur;
+  }
+  TG_MARK(4);
+  p.t = const_cast<cf*>(tprime);
+  TG_TRY(tail_any(s, 2, d_weight, p, st));
+  TG_MARK(5);
+  if (s->timing) s->timing_steps++;
+  s->t += 1;
+  return TGRAD_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+tgrad_status tgrad_state_bytes(const tgrad_config* cfg, size_t* persistent_bytes, size_t* workspace_bytes) {
+  if (!persistent_bytes || !workspace_bytes) return TGRAD_ERR_INVALID_ARG;
+  Layout L;
+  tgrad_status s = compute_layout(cfg, L, 148);
+  if (s != TGRAD_OK) return s;
+  *persistent_bytes = L.p_total;
+  *workspace_bytes = L.w_total;
+  return TGRAD_OK;
+}
+
+tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_t persistent_bytes, void* d_workspace,
+                              size_t workspace_bytes, void* cuda_stream, tgrad_state** out) {
+  if (!out) return TGRAD_ERR_INVALID_ARG;
+  *out = nullptr;
+  Layout L;
+  tgrad_status s = compute_layout(cfg, L, 148);
+  if (s != TGRAD_OK) return s;
+  if (!d_persistent || !d_workspace) return TGRAD_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_persistent) & 255) || (reinterpret_cast<uintptr_t>(d_workspace) & 255))
+    return TGRAD_ERR_INVALID_ARG;
+  if (persistent_bytes < L.p_total || workspace_bytes < L.w_total) return TGRAD_ERR_BUFFER_TOO_SMALL;
+  tgrad_state* st = new (std::nothrow) tgrad_state;
+  if (!st) return TGRAD_ERR_INVALID_ARG;
+  memset(st, 0, sizeof(*st));
+  st->cfg = *cfg; st->L = L;
+  st->dp = static_cast<char*>(d_persistent); st->dw = static_cast<char*>(d_workspace);
+  st->t = 0; st->have_subspace = false;
+  int dev = 0, sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
+  st->sm_count = sm;
+  s = plan_tail(st);
+  if (s != TGRAD_OK) { delete st; return s; }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  // Algorithm 1 initialisation: zero moments (and flags, Omega, factors for determinism)
+  if (cudaMemsetAsync(d_persistent, 0, L.p_total, stream) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
+  *out = st;
+  return TGRAD_OK;
+}
+
+tgrad_status tgrad_step(tgrad_state* st, void* d_weight, void* d_grad, void* cuda_stream) {
+  if (!st || !d_weight || !d_grad) return TGRAD_ERR_INVALID_ARG;
+  if (!aligned16(d_weight) || !aligned16(d_grad)) return TGRAD_ERR_INVALID_ARG;
+  return do_step(st, d_weight, d_grad, static_cast<cudaStream_t>(cuda_stream));
+}
+
+tgrad_status tgrad_refresh_subspace(tgrad_state* st, void* d_grad, void* cuda_stream) {
+  if (!st || !d_grad) return TGRAD_ERR_INVALID_ARG;
+  if (!aligned16(d_grad)) return TGRAD_ERR_INVALID_ARG;
+  return do_refresh(st, d_grad, static_cast<cudaStream_t>(cuda_stream));
+}
+
+tgrad_status tgrad_step_batched(tgrad_state* const* states, void* const* d_weights, void* const* d_grads,
+                                int32_t n_tensors, void* cuda_stream) {
+  if (n_tensors < 0 || (n_tensors > 0 && (!states || !d_weights || !d_grads))) return TGRAD_ERR_INVALID_ARG;
+  for (int i = 0; i < n_tensors; ++i) {
+    if (!states[i] || !d_weights[i] || !d_grads[i]) return TGRAD_ERR_INVALID_ARG;
+    if (!aligned16(d_weights[i]) || !aligned16(d_grads[i])) return TGRAD_ERR_INVALID_ARG;
+    if (!states[i]->have_subspace && !(states[i]->cfg.auto_refresh && states[i]->t % states[i]->cfg.T == 0))
+      return TGRAD_ERR_BAD_STATE;
+  }
+  for (int i = 0; i < n_tensors; ++i)
+    TG_TRY(do_step(states[i], d_weights[i], d_grads[i], static_cast<cudaStream_t>(cuda_stream)));
+  return TGRAD_OK;
+}
+
+tgrad_status tgrad_refresh_subspace_batched(tgrad_state* const* states, void* const* d_grads, int32_t n_tensors,
+                                            void* cuda_stream) {
+  if (n_tensors < 0 || (n_tensors > 0 && (!states || !d_grads))) return TGRAD_ERR_INVALID_ARG;
+  for (int i = 0; i < n_tensors; ++i)
+    if (!states[i] || !d_grads[i] || !aligned16(d_grads[i])) return TGRAD_ERR_INVALID_ARG;
+  for (int i = 0; i < n_tensors; ++i) TG_TRY(do_refresh(states[i], d_grads[i], static_cast<cudaStream_t>(cuda_stream)));
+  return TGRAD_OK;
+}
+
+tgrad_status tgrad_query_status(tgrad_state* st, void* cuda_stream, int32_t* sticky_flags, int64_t* t, int32_t* sweeps) {
+  if (!st) return TGRAD_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int host[1 + TGRAD_MAX_NDIM];
+  if (cudaMemcpyAsync(host, st->dp + st->L.p_flags, sizeof(host), cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return TGRAD_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return TGRAD_ERR_CUDA;
+  if (sticky_flags) *sticky_flags = host[0];
+  if (t) *t = st->t;
+  if (sweeps) for (int n = 0; n < st->cfg.ndim; ++n) sweeps[n] = host[1 + n];
+  return TGRAD_OK;
+}
+
+static tgrad_status locate(tgrad_state* st, int32_t what, bool for_import, char** ptr, size_t* bytes) {
+  const tgrad_config& c = st->cfg; const Layout& L = st->L;
+  const size_t k = (size_t)c.k, P = (size_t)L.P;
+  switch (what) {
+    case TGRAD_WHAT_OMEGA: *ptr = st->dp + L.p_omega; *bytes = k * 4; return TGRAD_OK;
+    case TGRAD_WHAT_M_L: *ptr = st->dp + L.p_ml; *bytes = P * 8; return TGRAD_OK;
+    case TGRAD_WHAT_V_L: *ptr = st->dp + L.p_vl; *bytes = P * 4; return TGRAD_OK;
+    case TGRAD_WHAT_M_S: *ptr = st->dp + L.p_ms; *bytes = k * 8; return TGRAD_OK;
+    case TGRAD_WHAT_V_S: *ptr = st->dp + L.p_vs; *bytes = k * 4; return TGRAD_OK;
+    default: break;
+  }
+  if (what >= TGRAD_WHAT_FACTOR_BASE && what < TGRAD_WHAT_FACTOR_BASE + c.ndim) {
+    int n = what - TGRAD_WHAT_FACTOR_BASE;
+    *ptr = st->dp + L.p_factor[n]; *bytes = (size_t)c.dims[n] * c.ranks[n] * 8; return TGRAD_OK;
+  }
+  if (for_import) return TGRAD_ERR_INVALID_ARG;
+  switch (what) {
+    case TGRAD_WHAT_CORE: *ptr = st->dw + L.w_core; *bytes = P * 8; return TGRAD_OK;
+    case TGRAD_WHAT_N_L: *ptr = st->dw + L.w_nl; *bytes = P * 8; return TGRAD_OK;
+    case TGRAD_WHAT_N_S: *ptr = st->dw + L.w_ns; *bytes = k * 8; return TGRAD_OK;
+    default: break;
+  }
+  if (what >= TGRAD_WHAT_GRAM_BASE && what < TGRAD_WHAT_GRAM_BASE + c.ndim) {
+    int n = what - TGRAD_WHAT_GRAM_BASE;
+    *ptr = st->dw + L.w_gram[n]; *bytes = (size_t)c.dims[n] * c.dims[n] * 8; return TGRAD_OK;
+  }
+  return TGRAD_ERR_INVALID_ARG;
+}
+
+tgrad_status tgrad_export_state(tgrad_state* st, int32_t what, void* host_dst, size_t bytes, void* cuda_stream) {
+  if (!st || (!host_dst && bytes)) return TGRAD_ERR_INVALID_ARG;
+  char* p; size_t nb;
+  tgrad_status s = locate(st, what, false, &p, &nb);
+  if (s != TGRAD_OK) return s;
+  if (bytes != nb) return TGRAD_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (nb && cudaMemcpyAsync(host_dst, p, nb, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return TGRAD_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return TGRAD_ERR_CUDA;
+  return TGRAD_OK;
+}
+
+tgrad_status tgrad_import_state(tgrad_state* st, int32_t what, const void* host_src, size_t bytes, void* cuda_stream) {
+  if (!st || (!host_src && bytes)) return TGRAD_ERR_INVALID_ARG;
+  char* p; size_t nb;
+  tgrad_status s = locate(st, what, true, &p, &nb);
+  if (s != TGRAD_OK) return s;
+  if (bytes != nb) return TGRAD_ERR_BUFFER_TOO_SMALL;
+  if (what == TGRAD_WHAT_OMEGA) {   // Omega must be strictly ascending and in range
+    const uint32_t* om = static_cast<const uint32_t*>(host_src);
+    const size_t k = (size_t)st->cfg.k;
+    for (size_t j = 0; j < k; ++j) {
+      if ((uint64_t)om[j] >= st->L.numel) return TGRAD_ERR_INVALID_ARG;
+      if (j && om[j] <= om[j - 1]) return TGRAD_ERR_INVALID_ARG;
+    }
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (nb && cudaMemcpyAsync(p, host_src, nb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return TGRAD_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return TGRAD_ERR_CUDA;
+  if (what == TGRAD_WHAT_OMEGA || what >= TGRAD_WHAT_FACTOR_BASE) st->have_subspace = true;
+  return TGRAD_OK;
+}
+
+tgrad_status tgrad_set_step(tgrad_state* st, int64_t t) {
+  if (!st || t < 0) return TGRAD_ERR_INVALID_ARG;
+  st->t = t;
+  return TGRAD_OK;
+}
+
+tgrad_status tgrad_set_stage_timing(tgrad_state* st, int32_t enable) {
+  if (!st) return TGRAD_ERR_INVALID_ARG;
+  if (enable && !st->ev[0][0]) {
+    for (int i = 0; i < kTimingRing; ++i)
+      for (int j = 0; j <= kStages; ++j)
+        if (cudaEventCreate(&st->ev[i][j]) != cudaSuccess) return TGRAD_ERR_CUDA;
+  }
+  st->timing = enable != 0;
+  st->timing_steps = 0;
+  return TGRAD_OK;
+}
+
+tgrad_status tgrad_get_stage_times(tgrad_state* st, void* cuda_stream, float* ms_sum, int32_t* n_steps) {
+  if (!st || !ms_sum || !n_steps) return TGRAD_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return TGRAD_ERR_CUDA;
+  int n = st->timing_steps < kTimingRing ? st->timing_steps : kTimingRing;
+  for (int j = 0; j < kStages; ++j) ms_sum[j] = 0.f;
+  for (int i = 0; i < n; ++i)
+    for (int j = 0; j < kStages; ++j) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, st->ev[i][j], st->ev[i][j + 1]) != cudaSuccess) return TGRAD_ERR_CUDA;
+      ms_sum[j] += ms;
+    }
+  *n_steps = n;
+  st->timing_steps = 0;
+  return TGRAD_OK;
+}
+
+tgrad_status tgrad_destroy_state(tgrad_state* st) {
+  if (!st) return TGRAD_ERR_INVALID_ARG;
+  if (st->ev[0][0])
+    for (int i = 0; i < kTimingRing; ++i)
+      for (int j = 0; j <= kStages; ++j)
+        if (st->ev[i][j]) cudaEventDestroy(st->ev[i][j]);
+  delete st;
+  return TGRAD_OK;
+}
+
+const char* tgrad_status_string(tgrad_status s) {
+  switch (s) {
+    case TGRAD_OK: return "ok";
+    case TGRAD_ERR_INVALID_ARG: return "invalid argument";
+    case TGRAD_ERR_UNSUPPORTED: return "unsupported configuration";
+    case TGRAD_ERR_BUFFER_TOO_SMALL: return "buffer size mismatch";
+    case TGRAD_ERR_CUDA: return "CUDA error";
+    case TGRAD_ERR_NO_CONVERGE: return "eigensolver did not converge";
+    case TGRAD_ERR_NONFINITE: return "non-finite gradient";
+    case TGRAD_ERR_BAD_STATE: return "state has no subspace yet";
+    default: return "unknown status";
+  }
+}
+
+int64_t tgrad_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

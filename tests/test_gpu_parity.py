@@ -1,0 +1,170 @@
+"""GPU-vs-oracle parity through the C ABI (run with -m gpu on a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tgrad_oracle as orc
+from paper_2501_02379_b200 import binding as B
+from paper_2501_02379_b200 import synth
+from tests import helpers as H
+from tests.parity import Pair, to_device, from_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name", ["tiny4", "small4", "small5", "ragged4"])
+def test_trajectory_small(name):
+    wl = synth.WORKLOADS[name]
+    p = Pair(wl)
+    for t in range(wl.steps):
+        p.step(t)
+    print(name, p.report)
+
+
+def test_trajectory_cfg1_full():
+    wl = synth.WORKLOADS["cfg1"]
+    p = Pair(wl)
+    for t in range(wl.steps):
+        p.step(t)
+    print("cfg1", p.report)
+
+
+def test_alpha_lambda_weight_decay():
+    wl = synth.WORKLOADS["small4"]
+    p = Pair(wl, alpha=0.25, lam=0.5, weight_decay=0.1, lr=1e-2)
+    for t in range(wl.T + 2):
+        p.step(t)
+
+
+def test_k_zero_lowrank_only():
+    import dataclasses
+    wl = dataclasses.replace(synth.WORKLOADS["small4"], rho=(0, 1), outlier_frac=(0, 1))
+    assert wl.k == 0
+    p = Pair(wl)
+    for t in range(wl.T + 1):
+        p.step(t)
+
+
+def test_topk_ties_bit_exact():
+    # tie-heavy quantised gradients, all-equal magnitudes, k in {1, I-1, I}
+    shape = (12, 10, 8, 5)
+    n = int(np.prod(shape))
+    for seed, k in [(0, 137), (1, 1), (2, n - 1), (3, n), (4, 2048), (5, 2049)]:
+        g = synth.quantised_ties(shape, 3, seed)
+        cfg = B.make_config(shape, (4, 3, 3, 2), k, 4, auto_refresh=False)
+        st = B.TgradState(cfg)
+        st.refresh_subspace(to_device(g, False))
+        assert np.array_equal(st.export(B.WHAT_OMEGA), orc.sparse_indices_topk(g, k)), (seed, k)
+    g = np.full(shape, 1 - 2j, dtype=np.complex64)
+    cfg = B.make_config(shape, (4, 3, 3, 2), 777, 4, auto_refresh=False)
+    st = B.TgradState(cfg)
+    st.refresh_subspace(to_device(g, False))
+    assert np.array_equal(st.export(B.WHAT_OMEGA), np.arange(777, dtype=np.uint32))
+
+
+def test_topk_multi_block_ragged():
+    # several compaction blocks plus a ragged tail, ties across block borders
+    shape = (37, 11, 9, 7)
+    g = synth.quantised_ties(shape, 40, 11)
+    n = g.size
+    for k in (1, 5000, n // 2):
+        cfg = B.make_config(shape, (4, 3, 3, 2), k, 4, auto_refresh=False)
+        st = B.TgradState(cfg)
+        st.refresh_subspace(to_device(g, False))
+        assert np.array_equal(st.export(B.WHAT_OMEGA), orc.sparse_indices_topk(g, k)), k
+
+
+def test_half_storage_small():
+    import dataclasses
+    wl = dataclasses.replace(synth.WORKLOADS["ragged4"], half_storage=True)
+    p = Pair(wl)
+    for t in range(wl.T + 2):
+        p.step(t)
+    print("half", p.report)
+
+
+def test_auto_refresh_matches_explicit():
+    wl = synth.WORKLOADS["small4"]
+    src = synth.GradientSource(wl)
+    outs = []
+    for auto in (True, False):
+        cfg = B.make_config(wl.shape, wl.ranks, wl.k, wl.T, auto_refresh=auto)
+        st = B.TgradState(cfg)
+        w = to_device(src.weight(), False)
+        for t in range(wl.T + 2):
+            g = to_device(src.gradient(t), False)
+            if not auto and t % wl.T == 0:
+                st.refresh_subspace(g)
+            st.step(w, g)
+        outs.append((from_device(w, False), st.export(B.WHAT_M_L), st.export(B.WHAT_OMEGA)))
+    for a, b in zip(outs[0], outs[1]):
+        assert np.array_equal(a, b)
+
+
+def test_export_import_resume_bitwise():
+    wl = synth.WORKLOADS["small4"]
+    src = synth.GradientSource(wl)
+    total = 2 * wl.T + 3
+    cut = wl.T + 1
+    cfg = B.make_config(wl.shape, wl.ranks, wl.k, wl.T)
+    a = B.TgradState(cfg)
+    wa = to_device(src.weight(), False)
+    snap = None
+    for t in range(total):
+        if t == cut:
+            snap = {w: a.export(w) for w in (B.WHAT_OMEGA, B.WHAT_M_L, B.WHAT_V_L, B.WHAT_M_S, B.WHAT_V_S)}
+            snap["factors"] = a.factors()
+            snap["w"] = wa.clone()
+        a.step(wa, to_device(src.gradient(t), False))
+    b = B.TgradState(B.make_config(wl.shape, wl.ranks, wl.k, wl.T))
+    for w in (B.WHAT_OMEGA, B.WHAT_M_L, B.WHAT_V_L, B.WHAT_M_S, B.WHAT_V_S):
+        b.import_(w, snap[w])
+    for n, u in enumerate(snap["factors"]):
+        b.import_(B.WHAT_FACTOR_BASE + n, u)
+    b.set_step(cut)
+    wb = snap["w"]
+    for t in range(cut, total):
+        b.step(wb, to_device(src.gradient(t), False))
+    assert torch.equal(wa, wb)
+    for w in (B.WHAT_OMEGA, B.WHAT_M_L, B.WHAT_V_L, B.WHAT_M_S, B.WHAT_V_S):
+        assert np.array_equal(a.export(w), b.export(w))
+    assert a.query_status()[1] == b.query_status()[1] == total
+
+
+def test_batched_matches_single():
+    wl = synth.WORKLOADS["small4"]
+    srcs = [synth.GradientSource(wl, i) for i in range(3)]
+    single, batched = [], []
+    for mode in ("single", "batched"):
+        sts = [B.TgradState(B.make_config(wl.shape, wl.ranks, wl.k, wl.T)) for _ in srcs]
+        ws = [to_device(s.weight(), False) for s in srcs]
+        for t in range(wl.T + 1):
+            gs = [to_device(s.gradient(t), False) for s in srcs]
+            if mode == "single":
+                for st, w, g in zip(sts, ws, gs):
+                    st.step(w, g)
+            else:
+                B.step_batched(sts, ws, gs)
+        (single if mode == "single" else batched).extend(ws)
+    for a, b in zip(single, batched):
+        assert torch.equal(a, b)
+
+
+def test_nonfinite_sets_flag():
+    wl = synth.WORKLOADS["small4"]
+    g = synth.GradientSource(wl).gradient(0)
+    g.reshape(-1)[5] = np.nan
+    st = B.TgradState(B.make_config(wl.shape, wl.ranks, wl.k, wl.T, auto_refresh=False))
+    st.refresh_subspace(to_device(g, False))
+    flags, _, _ = st.query_status()
+    assert flags & B.FLAG_NONFINITE
+
+
+def test_jacobi_cap_sets_flag_not_hang():
+    wl = synth.WORKLOADS["small4"]
+    g = synth.GradientSource(wl).gradient(0)
+    st = B.TgradState(B.make_config(wl.shape, wl.ranks, wl.k, wl.T, auto_refresh=False, jacobi_max_sweeps=1,
+                                    jacobi_tol=1e-12))
+    st.refresh_subspace(to_device(g, False))
+    flags, _, sweeps = st.query_status()
+    assert flags & B.FLAG_NO_CONVERGE and max(sweeps) == 1
