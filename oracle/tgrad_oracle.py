@@ -168,10 +168,18 @@ def adam_update(x, m, v, beta1, beta2, eps, t):
     m_new = (b1 * np.asarray(m, dtype=np.complex128) + (1.0 - b1) * x).astype(np.complex64)
     v_new = (b2 * np.asarray(v, dtype=np.float64)
              + (1.0 - b2) * (x.real * x.real + x.imag * x.imag)).astype(np.float32)
+    n = adam_direction(m_new, v_new, beta1, beta2, eps, t)
+    return n, m_new, v_new
+
+
+def adam_direction(m, v, beta1, beta2, eps, t):
+    """N = (M / (1-b1^(t+1))) / (sqrt(V / (1-b2^(t+1))) + eps): the bias-corrected,
+    normalised update computed from stored (un-corrected) moments (last three
+    statements of the UPDATE block of Algorithm 3)."""
+    b1 = float(np.float32(beta1)); b2 = float(np.float32(beta2)); e = float(np.float32(eps))
     c1 = float(np.float32(1.0 - b1 ** (t + 1)))
     c2 = float(np.float32(1.0 - b2 ** (t + 1)))
-    n = (m_new.astype(np.complex128) / c1) / (np.sqrt(v_new.astype(np.float64) / c2) + e)
-    return n, m_new, v_new
+    return (np.asarray(m, dtype=np.complex128) / c1) / (np.sqrt(np.asarray(v, dtype=np.float64) / c2) + e)
 
 
 # --------------------------------------------------------------------------

@@ -46,7 +46,6 @@ struct TailParams {
   int k;
   cf* m_s; float* v_s;   // sparse moments (proj)
   cf* n_s;               // normalised sparse update: written by proj, read by back
-  cf* g_s;               // gathered sparse values (proj writes them for inspection)
   cf* t;                 // proj: out T[s][ra][rb];  back: in T'[s][ra][rb]
   AdamScalars adam;
   float s_low, s_sparse; // eta*alpha, eta*lambda
@@ -119,7 +118,7 @@ __global__ void __launch_bounds__(256) proj_tail_kernel(const void* __restrict__
         xs[si] = make_float2(0.f, 0.f);
         cf m = p.m_s[j]; float v = p.v_s[j];
         cf n = adam_apply(x, m, v, p.adam);
-        p.m_s[j] = m; p.v_s[j] = v; p.n_s[j] = n; p.g_s[j] = x;
+        p.m_s[j] = m; p.v_s[j] = v; p.n_s[j] = n;
       }
       __syncwarp();
     }

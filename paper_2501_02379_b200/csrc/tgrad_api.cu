@@ -330,7 +330,6 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   p.m_s = reinterpret_cast<cf*>(s->dp + L.p_ms);
   p.v_s = reinterpret_cast<float*>(s->dp + L.p_vs);
   p.n_s = reinterpret_cast<cf*>(s->dw + L.w_ns);
-  p.g_s = reinterpret_cast<cf*>(s->dw + L.w_gs);
   p.adam = adam_scalars(c, s->t);
   p.s_low = (float)((double)c.lr * (double)c.alpha);
   p.s_sparse = (float)((double)c.lr * (double)c.lambda);
