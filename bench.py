@@ -23,7 +23,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2501_02379_b200 import synth  # noqa: E402
+from paper_2501_02379_b200 import replicas, synth  # noqa: E402
 
 METRIC = "tgrad_step effective HBM GB/s"
 FALLBACK_HBM_GBS = 6650.0
@@ -208,7 +208,7 @@ def run_ours(args, wl):
 
     # replicas only: every rank owns independent tensors (layers); no data-path collective
     n_t = wl.n_tensors
-    srcs = [synth.GradientSource(wl, rank * n_t + i) for i in range(n_t)]
+    srcs = [synth.GradientSource(wl, i) for i in replicas.tensor_ids_for_rank(rank, world, n_t)]
     ring = args.ring
     grads_host = [[s.gradient(r) for r in range(ring)] for s in srcs]
     if half:
@@ -253,10 +253,7 @@ def run_ours(args, wl):
     sampler.active = False
     launches = B.launch_count() - l0
     ms = e0.elapsed_time(e1)
-    if dist is not None:
-        tt = torch.tensor([ms], device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = float(tt.item())
+    ms = replicas.max_over_ranks(ms, dist, "cuda")
     flags = [s.query_status()[0] for s in states]
 
     # ---- per-stage device times of non-refresh steps (events on the launching stream) ----
@@ -315,10 +312,7 @@ def run_ours(args, wl):
     e7.record(stream)
     barrier()
     e2e_ms = e6.elapsed_time(e7)
-    if dist is not None:
-        tt = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
+    e2e_ms = replicas.max_over_ranks(e2e_ms, dist, "cuda")
     sampler.stop()
 
     if rank != 0:
