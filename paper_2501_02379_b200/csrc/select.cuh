@@ -241,4 +241,14 @@ __global__ void scatter_restore_kernel(void* __restrict__ g, const uint32_t* __r
   if (j < k) S::store(g, omega[j], g_s[j]);
 }
 
+// slab_ptr[s] = number of Omega entries below s*E (s = 0..nslab): the ascending index list is
+// thereby grouped by slab, and the streaming kernels find their slab's entries with two loads.
+__global__ void slab_ptr_kernel(const uint32_t* __restrict__ omega, uint32_t k, uint32_t E, uint32_t nslab,
+                                uint32_t* __restrict__ slab_ptr) {
+  uint32_t s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s > nslab) return;
+  uint64_t key = (uint64_t)s * E;
+  slab_ptr[s] = (s == nslab) ? k : (uint32_t)lower_bound_u32(omega, (int)k, (uint32_t)key);
+}
+
 }  // namespace tg

@@ -43,6 +43,7 @@ struct TailParams {
   const cf* Ua;          // U^(N-1), A x ra row-major
   const cf* Ub;          // U^(N),   B x rb row-major
   const uint32_t* omega; // ascending flat indices
+  const uint32_t* slab_ptr; // slab_ptr[s] = first Omega slot of slab s (nslab + 1 entries)
   int k;
   cf* m_s; float* v_s;   // sparse moments (proj)
   cf* n_s;               // normalised sparse update: written by proj, read by back
@@ -108,8 +109,7 @@ __global__ void __launch_bounds__(256) proj_tail_kernel(const void* __restrict__
     __syncwarp();
     // ---- sparse part: gather, Adam, zero (residual) ----
     if (p.k > 0) {
-      int j0 = lower_bound_u32(p.omega, p.k, (uint32_t)gbase);
-      int j1 = lower_bound_u32(p.omega, p.k, (uint32_t)(gbase + E));
+      const int j0 = (int)p.slab_ptr[s], j1 = (int)p.slab_ptr[s + 1];
       for (int j = j0 + lane; j < j1; j += 32) {
         uint32_t loc = p.omega[j] - (uint32_t)gbase;
         uint32_t a = loc / B;
@@ -268,8 +268,7 @@ __global__ void __launch_bounds__(256) back_tail_kernel(void* __restrict__ w, Ta
     __syncwarp();
     // ---- scaled sparse add at Omega (on top of the dense update) ----
     if (p.k > 0) {
-      int j0 = lower_bound_u32(p.omega, p.k, (uint32_t)gbase);
-      int j1 = lower_bound_u32(p.omega, p.k, (uint32_t)(gbase + E));
+      const int j0 = (int)p.slab_ptr[s], j1 = (int)p.slab_ptr[s + 1];
       for (int j = j0 + lane; j < j1; j += 32) {
         uint32_t loc = p.omega[j] - (uint32_t)gbase;
         uint32_t a = loc / B;

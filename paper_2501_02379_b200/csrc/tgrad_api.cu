@@ -14,6 +14,7 @@
 #include "modeprod.cuh"
 #include "select.cuh"
 #include "tail.cuh"
+#include "tail_mma.cuh"
 
 using namespace tg;
 
@@ -28,7 +29,8 @@ inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
 struct Layout {
   // persistent block
-  size_t p_flags, p_omega, p_factor[TGRAD_MAX_NDIM], p_ml, p_vl, p_ms, p_vs, p_total;
+  size_t p_flags, p_omega, p_slab, p_factor[TGRAD_MAX_NDIM], p_ml, p_vl, p_ms, p_vs, p_total;
+  uint32_t nslab, E;          // slabs of the trailing two modes, entries per slab
   // workspace block
   size_t w_ns, w_gs, w_core, w_nl, w_bufa, w_bufb, w_sel, w_hist, w_blk, w_gram[TGRAD_MAX_NDIM], w_jac[TGRAD_MAX_NDIM],
       w_v[TGRAD_MAX_NDIM], w_partial, w_total;
@@ -41,6 +43,11 @@ struct Layout {
 struct TailPlan {
   int rpl, rbp, nwarps, grid;
   size_t smem_proj, smem_back;
+  // tensor-core fast path (complex64 storage, slab rows a multiple of 16)
+  bool mma;
+  int rat, rbt, nt;
+  TailMmaGeom gproj, gback;
+  int grid_proj, grid_back;
 };
 
 tgrad_status validate(const tgrad_config* c) {
@@ -97,6 +104,8 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
   size_t o = 0;
   L.p_flags = o; o = align_up(o + 64 * sizeof(int));
   L.p_omega = o; o = align_up(o + k * 4);
+  L.nslab = (uint32_t)S; L.E = (uint32_t)((uint64_t)c->dims[N - 1] * c->dims[N - 2]);
+  L.p_slab = o; o = align_up(o + ((size_t)S + 1) * 4);
   for (int n = 0; n < N; ++n) { L.p_factor[n] = o; o = align_up(o + (size_t)c->dims[n] * c->ranks[n] * 8); }
   L.p_ml = o; o = align_up(o + P * 8);
   L.p_vl = o; o = align_up(o + P * 4);
@@ -189,6 +198,58 @@ tgrad_status tail_any(const tgrad_state* s, int op, void* ptr, const TailParams&
                                       : tail_dispatch<StoreC32H>(op, s->tail, ptr, p, st);
 }
 
+template <int RAT, int RBT, int NT>
+tgrad_status mma_proj_op(int op, const TailPlan& tp, const void* g, const TailMmaParams& P, cudaStream_t st) {
+  if (op == 0) {
+    return cudaFuncSetAttribute(proj_tail_mma_kernel<RAT, RBT, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)tp.gproj.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
+  }
+  proj_tail_mma_kernel<RAT, RBT, NT><<<tp.grid_proj, tp.gproj.nwarps * 32, tp.gproj.total, st>>>(g, P);
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
+}
+template <int RAT, int RBT>
+tgrad_status mma_back_op(int op, const TailPlan& tp, void* w, const TailMmaParams& P, cudaStream_t st) {
+  if (op == 0) {
+    return cudaFuncSetAttribute(back_tail_mma_kernel<RAT, RBT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)tp.gback.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
+  }
+  back_tail_mma_kernel<RAT, RBT><<<tp.grid_back, tp.gback.nwarps * 32, tp.gback.total, st>>>(w, P);
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
+}
+// op: 0 = set attributes (both kernels), 1 = proj, 2 = back
+tgrad_status mma_dispatch(int op, const TailPlan& tp, void* ptr, const TailMmaParams& P, cudaStream_t st) {
+#define TG_MCASE(RAT_, RBT_)                                                                     \
+  if (tp.rat == RAT_ && tp.rbt == RBT_) {                                                        \
+    if (op == 0 || op == 2) {                                                                    \
+      tgrad_status r = mma_back_op<RAT_, RBT_>(op, tp, ptr, P, st);                              \
+      if (op == 2 || r != TGRAD_OK) return r;                                                    \
+    }                                                                                            \
+    if (tp.nt == 8) return mma_proj_op<RAT_, RBT_, 8>(op, tp, ptr, P, st);                       \
+    if (tp.nt == 4) return mma_proj_op<RAT_, RBT_, 4>(op, tp, ptr, P, st);                       \
+    if (tp.nt == 2) return mma_proj_op<RAT_, RBT_, 2>(op, tp, ptr, P, st);                       \
+    return TGRAD_ERR_UNSUPPORTED;                                                                \
+  }
+  TG_MCASE(1, 1) TG_MCASE(2, 1) TG_MCASE(4, 1) TG_MCASE(1, 2) TG_MCASE(2, 2) TG_MCASE(4, 2)
+#undef TG_MCASE
+  return TGRAD_ERR_UNSUPPORTED;
+}
+
+// Ring geometry of the fast path: as many warps as fit (at most 8), ring depth 2 for the
+// read-only kernel and 3 for the read-write one (deeper for small slabs).
+bool plan_mma_geom(int A, int B, int rat, int rbt, bool back, TailMmaGeom& out) {
+  const uint32_t kMax = 227 * 1024;
+  const int min_buf = back ? 3 : 2;
+  for (int nw = 8; nw >= 1; --nw) {
+    for (int nb = 4; nb >= min_buf; --nb) {
+      TailMmaGeom g = tail_mma_geom(A, B, rat, rbt, nw, nb);
+      if (g.total <= kMax) { out = g; return true; }
+    }
+  }
+  return false;
+}
+
 tgrad_status plan_tail(tgrad_state* s) {
   const tgrad_config& c = s->cfg;
   const int N = c.ndim;
@@ -222,7 +283,25 @@ tgrad_status plan_tail(tgrad_state* s) {
   uint64_t g = (uint64_t)s->sm_count * per_sm;
   tp.grid = (int)(need < g ? need : g);
   TailParams dummy; memset(&dummy, 0, sizeof(dummy));
-  return tail_any(s, 0, nullptr, dummy, 0);
+  tgrad_status r = tail_any(s, 0, nullptr, dummy, 0);
+  if (r != TGRAD_OK) return r;
+  // fast path
+  tp.mma = false;
+  const int nt = (A % 64 == 0) ? 8 : (A % 32 == 0) ? 4 : (A % 16 == 0) ? 2 : 0;
+  const int rat = (ra + 7) / 8, rbt = (rb + 7) / 8;
+  const bool rat_ok = rat == 1 || rat == 2 || rat == 4 || rat == 3;
+  if (c.wg_dtype == TGRAD_C64 && nt && rbt <= 2 && rat_ok && rat <= 4 && (((uint64_t)A * B * 8) % 16 == 0) &&
+      (uint64_t)A * B * 8 < (1u << 20)) {
+    tp.rat = rat == 3 ? 4 : rat; tp.rbt = rbt; tp.nt = nt;
+    if (plan_mma_geom(A, B, tp.rat, tp.rbt, false, tp.gproj) && plan_mma_geom(A, B, tp.rat, tp.rbt, true, tp.gback)) {
+      uint64_t gp = (S + tp.gproj.nwarps - 1) / tp.gproj.nwarps, gb2 = (S + tp.gback.nwarps - 1) / tp.gback.nwarps;
+      tp.grid_proj = (int)(gp < (uint64_t)s->sm_count ? gp : (uint64_t)s->sm_count);
+      tp.grid_back = (int)(gb2 < (uint64_t)s->sm_count ? gb2 : (uint64_t)s->sm_count);
+      TailMmaParams dm; memset(&dm, 0, sizeof(dm));
+      if (mma_dispatch(0, tp, nullptr, dm, 0) == TGRAD_OK) tp.mma = true;
+    }
+  }
+  return TGRAD_OK;
 }
 
 AdamScalars adam_scalars(const tgrad_config& c, int64_t t) {
@@ -234,6 +313,15 @@ AdamScalars adam_scalars(const tgrad_config& c, int64_t t) {
   a.inv_c1 = 1.0f / c1; a.inv_c2 = 1.0f / c2;
   a.eps = c.eps;
   return a;
+}
+
+tgrad_status build_slab_ptr(tgrad_state* s, cudaStream_t st) {
+  const Layout& L = s->L;
+  slab_ptr_kernel<<<(L.nslab + 1 + 255) / 256, 256, 0, st>>>(reinterpret_cast<const uint32_t*>(s->dp + L.p_omega),
+                                                              (uint32_t)s->cfg.k, L.E, L.nslab,
+                                                              reinterpret_cast<uint32_t*>(s->dp + L.p_slab));
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
 }
 
 template <class S>
@@ -264,6 +352,10 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
     sel_compact_kernel<S><<<L.nblk, kChunkThreads, 0, st>>>(d_grad, n, sel, blk_gt, blk_eq, omega, g_s, k);
     TG_LAUNCH_CHECK();
     scatter_zero_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, k); TG_LAUNCH_CHECK();
+  }
+  {
+    tgrad_status r = build_slab_ptr(s, st);
+    if (r != TGRAD_OK) return r;
   }
   cf* partial = reinterpret_cast<cf*>(s->dw + L.w_partial);
   JacobiParams jp; memset(&jp, 0, sizeof(jp));
@@ -326,6 +418,7 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   p.Ua = reinterpret_cast<const cf*>(s->dp + L.p_factor[N - 2]);
   p.Ub = reinterpret_cast<const cf*>(s->dp + L.p_factor[N - 1]);
   p.omega = reinterpret_cast<const uint32_t*>(s->dp + L.p_omega);
+  p.slab_ptr = reinterpret_cast<const uint32_t*>(s->dp + L.p_slab);
   p.k = (int)c.k;
   p.m_s = reinterpret_cast<cf*>(s->dp + L.p_ms);
   p.v_s = reinterpret_cast<float*>(s->dp + L.p_vs);
@@ -342,7 +435,13 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   // low-rank compression: trailing two modes while streaming G, then modes N-2 .. 1
   TG_MARK(0);
   p.t = bufa;
-  TG_TRY(tail_any(s, 1, d_grad, p, st));
+  TailMmaParams mp;
+  if (s->tail.mma) {
+    mp.p = p; mp.g = s->tail.gproj; mp.flags = reinterpret_cast<int*>(s->dp + L.p_flags);
+    TG_TRY(mma_dispatch(1, s->tail, d_grad, mp, st));
+  } else {
+    TG_TRY(tail_any(s, 1, d_grad, p, st));
+  }
   TG_MARK(1);
   {
     cf* cur = bufa; cf* nxt = bufb;
@@ -382,7 +481,12 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   }
   TG_MARK(4);
   p.t = const_cast<cf*>(tprime);
-  TG_TRY(tail_any(s, 2, d_weight, p, st));
+  if (s->tail.mma) {
+    mp.p = p; mp.g = s->tail.gback; mp.flags = reinterpret_cast<int*>(s->dp + L.p_flags);
+    TG_TRY(mma_dispatch(2, s->tail, d_weight, mp, st));
+  } else {
+    TG_TRY(tail_any(s, 2, d_weight, p, st));
+  }
   TG_MARK(5);
   if (s->timing) s->timing_steps++;
   s->t += 1;
@@ -541,6 +645,11 @@ tgrad_status tgrad_import_state(tgrad_state* st, int32_t what, const void* host_
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   if (nb && cudaMemcpyAsync(p, host_src, nb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return TGRAD_ERR_CUDA;
   if (cudaStreamSynchronize(stream) != cudaSuccess) return TGRAD_ERR_CUDA;
+  if (what == TGRAD_WHAT_OMEGA) {
+    tgrad_status r = build_slab_ptr(st, stream);
+    if (r != TGRAD_OK) return r;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return TGRAD_ERR_CUDA;
+  }
   if (what == TGRAD_WHAT_OMEGA || what >= TGRAD_WHAT_FACTOR_BASE) st->have_subspace = true;
   return TGRAD_OK;
 }

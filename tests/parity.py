@@ -16,7 +16,7 @@ from paper_2501_02379_b200 import synth
 from tests import helpers as H
 
 TOL_FLOAT = 1e-4       # max relative error, entries measured against max(|ref|, 2^-5 rms(ref)); see helpers.rel_err
-TOL_FRO = 2e-6         # and the whole array: ||a - b||_F / ||b||_F
+TOL_FRO = 5e-6         # and the whole array: ||a - b||_F / ||b||_F (split-TF32 products carry 2^-21 relative error)
 TOL_ANGLE = 1e-3       # largest principal-angle sine of a refreshed factor
 TOL_ORTHO = 1e-5       # max |U^H U - I|
 

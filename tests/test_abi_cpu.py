@@ -42,8 +42,9 @@ def test_state_bytes_counts_the_papers_inventory():
         pb, wb = B.state_bytes(cfg)
         p = int(np.prod(wl.ranks, dtype=np.int64))
         fac = sum(i * r for i, r in zip(wl.shape, wl.ranks))
-        need = 4 * wl.k + 8 * fac + 8 * p + 4 * p + 8 * wl.k + 4 * wl.k
-        assert need <= pb <= need + 256 * (6 + len(wl.shape)) + 512
+        slabs = wl.numel // (wl.shape[-1] * wl.shape[-2])
+        need = 4 * wl.k + 8 * fac + 8 * p + 4 * p + 8 * wl.k + 4 * wl.k + 4 * (slabs + 1)   # + per-slab offsets into Omega
+        assert need <= pb <= need + 256 * (7 + len(wl.shape)) + 512
         assert wb > 0 and pb % 256 == 0 and wb % 256 == 0
     # the paper's example (N=64, M=128, r=16): core-shaped moment + factors = 71,680 entries
     cfg = B.make_config((64, 64, 128, 128), (16, 16, 16, 16), 0, 10)
