@@ -76,8 +76,30 @@ __device__ __forceinline__ float tf32_hi(float x) {
 // lane = 4 g + t:  a0 (g, t)  a1 (g+8, t)  a2 (g, t+4)  a3 (g+8, t+4);  b0 (k=t, n=g)  b1 (k=t+4, n=g);
 // d0 (g, 2t)  d1 (g, 2t+1)  d2 (g+8, 2t)  d3 (g+8, 2t+1).
 __device__ __forceinline__ void mma_tf32(float (&d)[4], float a0, float a1, float a2, float a3, float b0, float b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(__float_as_uint(a0)), "r"(__float_as_uint(a1)), "r"(__float_as_uint(a2)), "r"(__float_as_uint(a3)),
+        "r"(__float_as_uint(b0)), "r"(__float_as_uint(b1)));
+}
+
+// The same MMA with operand a1 (resp. a1 and a3) negated inside the instruction sequence, so that the
+// negated copies of loop-invariant fragments do not occupy registers across the loop.
+__device__ __forceinline__ void mma_tf32_n1(float (&d)[4], float a0, float a1, float a2, float a3, float b0, float b1) {
+  asm(
+      "{\n\t.reg .b32 na1;\n\t"
+      "xor.b32 na1, %5, 0x80000000;\n\t"
+      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,na1,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n\t}"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(__float_as_uint(a0)), "r"(__float_as_uint(a1)), "r"(__float_as_uint(a2)), "r"(__float_as_uint(a3)),
+        "r"(__float_as_uint(b0)), "r"(__float_as_uint(b1)));
+}
+__device__ __forceinline__ void mma_tf32_n13(float (&d)[4], float a0, float a1, float a2, float a3, float b0, float b1) {
+  asm(
+      "{\n\t.reg .b32 na1, na3;\n\t"
+      "xor.b32 na1, %5, 0x80000000;\n\t"
+      "xor.b32 na3, %7, 0x80000000;\n\t"
+      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,na1,%6,na3}, {%8,%9}, {%0,%1,%2,%3};\n\t}"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(__float_as_uint(a0)), "r"(__float_as_uint(a1)), "r"(__float_as_uint(a2)), "r"(__float_as_uint(a3)),
         "r"(__float_as_uint(b0)), "r"(__float_as_uint(b1)));

@@ -14,7 +14,7 @@
 #include "modeprod.cuh"
 #include "select.cuh"
 #include "tail.cuh"
-#include "tail_mma.cuh"
+#include "tail_tc.cuh"
 
 using namespace tg;
 
@@ -43,10 +43,10 @@ struct Layout {
 struct TailPlan {
   int rpl, rbp, nwarps, grid;
   size_t smem_proj, smem_back;
-  // tensor-core fast path (complex64 storage, slab rows a multiple of 16)
-  bool mma;
-  int rat, rbt, nt;
-  TailMmaGeom gproj, gback;
+  // tensor-core fast path (complex64 storage, 16/32/64 slab rows, small trailing ranks)
+  bool tc;
+  int rat, ks, ntw;
+  TcGeom gproj, gback;
   int grid_proj, grid_back;
 };
 
@@ -198,56 +198,47 @@ tgrad_status tail_any(const tgrad_state* s, int op, void* ptr, const TailParams&
                                       : tail_dispatch<StoreC32H>(op, s->tail, ptr, p, st);
 }
 
-template <int RAT, int RBT, int NT>
-tgrad_status mma_proj_op(int op, const TailPlan& tp, const void* g, const TailMmaParams& P, cudaStream_t st) {
+template <int RAT, int KS, int NTW>
+tgrad_status tc_proj_op2(int op, const TailPlan& tp, const void* g, const TailTcParams& P, cudaStream_t st) {
   if (op == 0) {
-    return cudaFuncSetAttribute(proj_tail_mma_kernel<RAT, RBT, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(proj_tail_tc_kernel<RAT, KS, NTW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)tp.gproj.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
   }
-  proj_tail_mma_kernel<RAT, RBT, NT><<<tp.grid_proj, tp.gproj.nwarps * 32, tp.gproj.total, st>>>(g, P);
+  proj_tail_tc_kernel<RAT, KS, NTW><<<tp.grid_proj, PJ_THREADS, tp.gproj.total, st>>>(g, P);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
-template <int RAT, int RBT>
-tgrad_status mma_back_op(int op, const TailPlan& tp, void* w, const TailMmaParams& P, cudaStream_t st) {
+template <int RAT, int KS>
+tgrad_status tc_proj_op(int op, const TailPlan& tp, const void* g, const TailTcParams& P, cudaStream_t st) {
+  return tp.ntw == 2 ? tc_proj_op2<RAT, KS, 2>(op, tp, g, P, st) : tc_proj_op2<RAT, KS, 1>(op, tp, g, P, st);
+}
+template <int RAT>
+tgrad_status tc_back_op(int op, const TailPlan& tp, void* w, const TailTcParams& P, cudaStream_t st) {
   if (op == 0) {
-    return cudaFuncSetAttribute(back_tail_mma_kernel<RAT, RBT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(back_tail_tc_kernel<RAT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)tp.gback.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
   }
-  back_tail_mma_kernel<RAT, RBT><<<tp.grid_back, tp.gback.nwarps * 32, tp.gback.total, st>>>(w, P);
+  back_tail_tc_kernel<RAT><<<tp.grid_back, TC_THREADS, tp.gback.total, st>>>(w, P);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
 // op: 0 = set attributes (both kernels), 1 = proj, 2 = back
-tgrad_status mma_dispatch(int op, const TailPlan& tp, void* ptr, const TailMmaParams& P, cudaStream_t st) {
-#define TG_MCASE(RAT_, RBT_)                                                                     \
-  if (tp.rat == RAT_ && tp.rbt == RBT_) {                                                        \
+tgrad_status tc_dispatch(int op, const TailPlan& tp, void* ptr, const TailTcParams& P, cudaStream_t st) {
+#define TG_TCASE(RAT_)                                                                           \
+  if (tp.rat == RAT_) {                                                                          \
     if (op == 0 || op == 2) {                                                                    \
-      tgrad_status r = mma_back_op<RAT_, RBT_>(op, tp, ptr, P, st);                              \
+      tgrad_status r = tc_back_op<RAT_>(op, tp, ptr, P, st);                                     \
       if (op == 2 || r != TGRAD_OK) return r;                                                    \
     }                                                                                            \
-    if (tp.nt == 8) return mma_proj_op<RAT_, RBT_, 8>(op, tp, ptr, P, st);                       \
-    if (tp.nt == 4) return mma_proj_op<RAT_, RBT_, 4>(op, tp, ptr, P, st);                       \
-    if (tp.nt == 2) return mma_proj_op<RAT_, RBT_, 2>(op, tp, ptr, P, st);                       \
+    if (tp.ks == 4) return tc_proj_op<RAT_, 4>(op, tp, ptr, P, st);                              \
+    if (tp.ks == 5) return tc_proj_op<RAT_, 5>(op, tp, ptr, P, st);                              \
+    if (tp.ks == 8) return tc_proj_op<RAT_, 8>(op, tp, ptr, P, st);                              \
+    if (tp.ks == 9) return tc_proj_op<RAT_, 9>(op, tp, ptr, P, st);                              \
     return TGRAD_ERR_UNSUPPORTED;                                                                \
   }
-  TG_MCASE(1, 1) TG_MCASE(2, 1) TG_MCASE(4, 1) TG_MCASE(1, 2) TG_MCASE(2, 2) TG_MCASE(4, 2)
-#undef TG_MCASE
+  TG_TCASE(1) TG_TCASE(2)
+#undef TG_TCASE
   return TGRAD_ERR_UNSUPPORTED;
-}
-
-// Ring geometry of the fast path: as many warps as fit (at most 8), ring depth 2 for the
-// read-only kernel and 3 for the read-write one (deeper for small slabs).
-bool plan_mma_geom(int A, int B, int rat, int rbt, bool back, TailMmaGeom& out) {
-  const uint32_t kMax = 227 * 1024;
-  const int min_buf = back ? 3 : 2;
-  for (int nw = 8; nw >= 1; --nw) {
-    for (int nb = 4; nb >= min_buf; --nb) {
-      TailMmaGeom g = tail_mma_geom(A, B, rat, rbt, nw, nb);
-      if (g.total <= kMax) { out = g; return true; }
-    }
-  }
-  return false;
 }
 
 tgrad_status plan_tail(tgrad_state* s) {
@@ -286,19 +277,20 @@ tgrad_status plan_tail(tgrad_state* s) {
   tgrad_status r = tail_any(s, 0, nullptr, dummy, 0);
   if (r != TGRAD_OK) return r;
   // fast path
-  tp.mma = false;
-  const int nt = (A % 64 == 0) ? 8 : (A % 32 == 0) ? 4 : (A % 16 == 0) ? 2 : 0;
-  const int rat = (ra + 7) / 8, rbt = (rb + 7) / 8;
-  const bool rat_ok = rat == 1 || rat == 2 || rat == 4 || rat == 3;
-  if (c.wg_dtype == TGRAD_C64 && nt && rbt <= 2 && rat_ok && rat <= 4 && (((uint64_t)A * B * 8) % 16 == 0) &&
-      (uint64_t)A * B * 8 < (1u << 20)) {
-    tp.rat = rat == 3 ? 4 : rat; tp.rbt = rbt; tp.nt = nt;
-    if (plan_mma_geom(A, B, tp.rat, tp.rbt, false, tp.gproj) && plan_mma_geom(A, B, tp.rat, tp.rbt, true, tp.gback)) {
-      uint64_t gp = (S + tp.gproj.nwarps - 1) / tp.gproj.nwarps, gb2 = (S + tp.gback.nwarps - 1) / tp.gback.nwarps;
-      tp.grid_proj = (int)(gp < (uint64_t)s->sm_count ? gp : (uint64_t)s->sm_count);
-      tp.grid_back = (int)(gb2 < (uint64_t)s->sm_count ? gb2 : (uint64_t)s->sm_count);
-      TailMmaParams dm; memset(&dm, 0, sizeof(dm));
-      if (mma_dispatch(0, tp, nullptr, dm, 0) == TGRAD_OK) tp.mma = true;
+  tp.tc = false;
+  const int rat = (ra + 7) / 8, ksn = tc_ksteps(B);
+  const int ks = ksn <= 4 ? 4 : ksn == 5 ? 5 : ksn <= 8 ? 8 : ksn == 9 ? 9 : 0;
+  const double dec = 1.0 - (double)c.lr * (double)c.weight_decay;
+  if (c.wg_dtype == TGRAD_C64 && (A == 16 || A == 32 || A == 64) && rat <= 2 && rb <= 8 && ks && dec > 0.0) {
+    tp.rat = rat; tp.ks = ks; tp.ntw = (A == 64) ? 2 : 1;
+    const int pj_blocks = tp.ntw == 2 ? 3 : 4;                       // resident blocks per SM of the compression kernel
+    const uint32_t pj_smem = (227u * 1024u) / pj_blocks - 1024u;
+    if (proj_tc_geom(A, B, rat, (uint32_t)S, tp.ntw, pj_smem, tp.gproj) && tail_tc_geom(true, A, B, rat, (uint32_t)S, tp.gback)) {
+      const uint32_t cap = 2u * (uint32_t)s->sm_count, pcap = (uint32_t)pj_blocks * (uint32_t)s->sm_count;
+      tp.grid_proj = (int)(tp.gproj.ngroups < pcap ? tp.gproj.ngroups : pcap);
+      tp.grid_back = (int)(tp.gback.ngroups < cap ? tp.gback.ngroups : cap);
+      TailTcParams dm; memset(&dm, 0, sizeof(dm));
+      if (tc_dispatch(0, tp, nullptr, dm, 0) == TGRAD_OK) tp.tc = true;
     }
   }
   return TGRAD_OK;
@@ -435,10 +427,12 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   // low-rank compression: trailing two modes while streaming G, then modes N-2 .. 1
   TG_MARK(0);
   p.t = bufa;
-  TailMmaParams mp;
-  if (s->tail.mma) {
-    mp.p = p; mp.g = s->tail.gproj; mp.flags = reinterpret_cast<int*>(s->dp + L.p_flags);
-    TG_TRY(mma_dispatch(1, s->tail, d_grad, mp, st));
+  TailTcParams mp;
+  mp.flags = reinterpret_cast<int*>(s->dp + L.p_flags);
+  mp.s_sparse_pre = (float)((double)c.lr * (double)c.lambda / (1.0 - (double)c.lr * (double)c.weight_decay));
+  if (s->tail.tc) {
+    mp.p = p; mp.g = s->tail.gproj;
+    TG_TRY(tc_dispatch(1, s->tail, d_grad, mp, st));
   } else {
     TG_TRY(tail_any(s, 1, d_grad, p, st));
   }
@@ -481,9 +475,9 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   }
   TG_MARK(4);
   p.t = const_cast<cf*>(tprime);
-  if (s->tail.mma) {
-    mp.p = p; mp.g = s->tail.gback; mp.flags = reinterpret_cast<int*>(s->dp + L.p_flags);
-    TG_TRY(mma_dispatch(2, s->tail, d_weight, mp, st));
+  if (s->tail.tc) {
+    mp.p = p; mp.g = s->tail.gback;
+    TG_TRY(tc_dispatch(2, s->tail, d_weight, mp, st));
   } else {
     TG_TRY(tail_any(s, 2, d_weight, p, st));
   }
