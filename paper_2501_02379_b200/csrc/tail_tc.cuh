@@ -168,7 +168,20 @@ __global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_ker
       w[0] = h0.x; w[1] = h0.y; w[2] = -h0.y; w[3] = h1.x; w[4] = h1.y; w[5] = -h1.y;
       w[6] = l0.x; w[7] = l0.y; w[8] = -l0.y; w[9] = l1.x; w[10] = l1.y; w[11] = -l1.y;
     }
+  // ---- this thread's first two output floats of a group: which partial element each sums, where it goes ----
   const int out_per_slab = 2 * ra * rb, n_out = spi * out_per_slab;
+  int o_src[2], o_dst[2], o_q[2];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int o = tid + i * PJ_THREADS;
+    o_src[i] = -1; o_dst[i] = 0; o_q[i] = 0;
+    if (o < n_out) {
+      const int qo = o / out_per_slab, rem = o - qo * out_per_slab;
+      const int cidx = rem >> 1, ja = cidx / rb, jb = cidx - ja * rb;
+      o_src[i] = qo * tw * REDW + (ja * 8 + jb) * 2 + (rem & 1);
+      o_dst[i] = qo * out_per_slab + rem; o_q[i] = qo;
+    }
+  }
 
   if (tid == 0) {
     for (int i = 0; i < nbuf; ++i) mbar_init(&bars[i], 1);
@@ -194,21 +207,30 @@ __global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_ker
   // sums the partials of iteration `itp` (group up) in warp order and writes T
   auto reduce_out = [&](uint32_t up, uint32_t itp) {
     const float* rp = red + (size_t)(itp & 1) * PJ_WARPS * REDW;
-    for (int o = tid; o < n_out; o += PJ_THREADS) {
+    float* tg_ = reinterpret_cast<float*>(p.t) + (size_t)up * spi * out_per_slab;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      if (o_src[i] >= 0 && up * spi + o_q[i] < nslab) {
+        const float* src = rp + o_src[i];
+        float acc = src[0];
+        for (int w = 1; w < tw; ++w) acc += src[(size_t)w * REDW];
+        tg_[o_dst[i]] = acc;
+      }
+    }
+    for (int o = tid + 2 * PJ_THREADS; o < n_out; o += PJ_THREADS) {     // wide cores: more outputs than 2 per thread
       const int qo = o / out_per_slab, rem = o - qo * out_per_slab;
       const int cidx = rem >> 1, ja = cidx / rb, jb = cidx - ja * rb;
-      const uint32_t s = up * spi + qo;
-      if (s >= nslab) continue;
+      if (up * spi + qo >= nslab) continue;
       const float* src = rp + (size_t)(qo * tw) * REDW + ((ja * 8 + jb) * 2 + (rem & 1));
       float acc = src[0];
       for (int w = 1; w < tw; ++w) acc += src[(size_t)w * REDW];
-      reinterpret_cast<float*>(p.t)[(size_t)s * out_per_slab + rem] = acc;
+      tg_[o] = acc;
     }
   };
 
-  uint32_t it = 0;
+  uint32_t it = 0, phase = 0;
+  int buf = 0, pbuf = 0;      // ring slot of this iteration and of the previous one
   for (uint32_t u = blockIdx.x; u < ngroups; u += gstride, ++it) {
-    const int buf = (int)(it % nbuf);
     // bounds of the next group's entries: issued now, used at the end of this iteration
     int n0 = 0, n1 = 0;
     if (sparse && u + gstride < ngroups) {
@@ -216,7 +238,7 @@ __global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_ker
       uint32_t e = (un + 1) * spi; if (e > nslab) e = nslab;
       n0 = (int)p.slab_ptr[un * spi]; n1 = (int)p.slab_ptr[e];
     }
-    const bool ok = mbar_wait_bounded(&bars[buf], (it / nbuf) & 1);
+    const bool ok = mbar_wait_bounded(&bars[buf], phase);
     float* xg = reinterpret_cast<float*>(smem + (size_t)buf * G.grp_stride);
     // ---- sparse part, before the barrier: gather and zero (the residual); one entry of the group per thread ----
     const int jcur = b0 + tid;
@@ -243,16 +265,19 @@ __global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_ker
       // a copy did not arrive: record it, let the copies still in flight land (bounded), leave
       if (tid == 0) {
         atomicOr(P.flags, 4);
-        uint32_t ux = u + gstride;
-        for (int i = 1; i + 1 < nbuf && ux < ngroups; ++i, ux += gstride)
-          mbar_wait_bounded(&bars[(it + i) % nbuf], ((it + i) / nbuf) & 1, 1u << 16);
+        uint32_t ux = u + gstride, ph = phase;
+        int bx = buf;
+        for (int i = 1; i + 1 < nbuf && ux < ngroups; ++i, ux += gstride) {
+          if (++bx == nbuf) { bx = 0; ph ^= 1; }
+          mbar_wait_bounded(&bars[bx], ph, 1u << 16);
+        }
       }
       return;
     }
     // every warp is past its reads of the previous group: its ring buffer takes the group nbuf ahead
     if (it > 0 && tid == 0) {
       const uint32_t un = u + (uint32_t)(nbuf - 1) * gstride;
-      if (un < ngroups) tc_issue_load(gb, smem, G, bars, un, (int)((it - 1) % nbuf), nslab);
+      if (un < ngroups) tc_issue_load(gb, smem, G, bars, un, pbuf, nslab);
     }
     // ---- this group's contraction ----
     float d2[RAT][2][4];
@@ -324,6 +349,8 @@ __global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_ker
       const int j = b0 + tid;
       if (j < b1) { pom = p.omega[j]; pm = p.m_s[j]; pv = p.v_s[j]; }
     }
+    pbuf = buf;
+    if (++buf == nbuf) { buf = 0; phase ^= 1; }
   }
   if (it > 0) {
     __syncthreads();
@@ -416,9 +443,9 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
   }
   const bool decay = p.decay != 1.0f;
   const uint32_t row_bytes = 16u * (uint32_t)B * 8u;            // the 16 rows a warp owns
-  uint32_t it = 0;
+  uint32_t it = 0, phase = 0;
+  int buf = 0, lbuf = la % nbuf;      // ring slot of this iteration and of the group loaded `la` ahead
   for (uint32_t u = blockIdx.x; u < ngroups; u += gstride, ++it) {
-    const int buf = (int)(it % nbuf);
     const uint32_t s = u * spi + q;
     const bool active = s < nslab;
     if (lane == 0) bulk_wait_read<1>();     // this warp's store of two iterations ago has read its rows
@@ -432,7 +459,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
         tv[ks] = (active && ja < ra && gq < rb) ? __ldg(tin + (size_t)ja * rb + gq) : make_float2(0.f, 0.f);
       }
     }
-    const bool ok = mbar_wait_bounded(&bars[buf], (it / nbuf) & 1);
+    const bool ok = mbar_wait_bounded(&bars[buf], phase);
     float* wg = reinterpret_cast<float*>(smem + (size_t)buf * G.grp_stride);
     // ---- scaled sparse add at Omega, one entry of the group per thread ----
     if (sparse && ok) {
@@ -464,9 +491,12 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
     if (__syncthreads_or(!ok)) {
       if (tid == 0) {
         atomicOr(P.flags, 4);
-        uint32_t ux = u + gstride;
-        for (int i = 1; i < la && ux < ngroups; ++i, ux += gstride)
-          mbar_wait_bounded(&bars[(it + i) % nbuf], ((it + i) / nbuf) & 1, 1u << 16);
+        uint32_t ux = u + gstride, ph = phase;
+        int bx = buf;
+        for (int i = 1; i < la && ux < ngroups; ++i, ux += gstride) {
+          if (++bx == nbuf) { bx = 0; ph ^= 1; }
+          mbar_wait_bounded(&bars[bx], ph, 1u << 16);
+        }
       }
       if (lane == 0) bulk_wait_all<0>();
       return;
@@ -474,7 +504,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
     // every warp's store of iteration it-2 has been read (checked before the barrier): its buffer takes group it+la
     if (tid == 0) {
       const uint32_t un = u + (uint32_t)la * gstride;
-      if (un < ngroups) tc_issue_load(wb, smem, G, bars, un, (int)((it + la) % nbuf), nslab);
+      if (un < ngroups) tc_issue_load(wb, smem, G, bars, un, lbuf, nslab);
     }
     if (active) {
       float* ws = wg + (size_t)q * (2 * E);
@@ -539,6 +569,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
                                                                 (size_t)am * B * 8, row_bytes);
       bulk_commit();
     }
+    if (++buf == nbuf) { buf = 0; phase ^= 1; }
+    if (++lbuf == nbuf) lbuf = 0;
   }
   if (lane == 0) bulk_wait_all<0>();   // stores complete before the block's shared memory goes away
 }
