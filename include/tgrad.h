@@ -54,7 +54,8 @@ typedef enum {
   TGRAD_ERR_CUDA = 4,
   TGRAD_ERR_NO_CONVERGE = 5,
   TGRAD_ERR_NONFINITE = 6,
-  TGRAD_ERR_BAD_STATE = 7
+  TGRAD_ERR_BAD_STATE = 7,
+  TGRAD_ERR_TOO_LARGE = 8      /* tgrad_select_topk_noalloc: more entries than its built-in scratch covers */
 } tgrad_status;
 
 /* sticky device flags reported by tgrad_query_status() */
@@ -163,6 +164,44 @@ tgrad_status tgrad_set_step(tgrad_state* st, int64_t t);
 tgrad_status tgrad_destroy_state(tgrad_state* st);
 
 const char* tgrad_status_string(tgrad_status s);
+
+/* Magnitude top-k selection for callers that cannot allocate device memory.
+ * (The paper has no counterpart of this call; it computes the same Omega as
+ * the refresh, "Unstructured sparse gradient tensor" with the top-k strategy.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a
+ * framework's allocator callback or memory-pool hook (allocating there
+ * re-enters the allocator), in a process whose device memory was handed out
+ * in full at start-up, or in a latency-critical loop that must not take the
+ * driver's allocation lock.  The other entry points need a workspace block
+ * that somebody allocated; this one needs none.
+ *
+ * The scratch of the selection (radix histograms, threshold state, per-block
+ * counts) lives in a fixed array inside the library's device image, about
+ * 290 KB, which every GPU that loads the library holds until the process
+ * exits.  That fixes the largest input: numel <= TGRAD_NOALLOC_MAX_NUMEL,
+ * otherwise TGRAD_ERR_TOO_LARGE and nothing is enqueued.
+ *
+ * d_grad:   device, numel entries of wg_dtype (tgrad_dtype), read only.
+ * d_omega:  device, out, k x uint32: the flat indices of the k entries of
+ *           largest |g|^2 (fp32 re*re + im*im without fused multiply-add),
+ *           ties to the lower index, ascending.
+ * d_values: device, out, k x complex64: grad at those indices (widened to
+ *           fp32 if stored as fp16), i.e. Sparse(G, Omega) as index-value pairs.
+ * Work is enqueued on the stream; nothing is allocated or freed, on the
+ * device or by any library, and the stream is not synchronised.
+ *
+ * First call on a device: the library looks up the device address of its
+ * scratch array once per device (the device that is current at the call) and
+ * remembers it.  Make that first call outside any stream capture.
+ * Sharing: all calls on a device use the same scratch, which keeps what the
+ * last call left there; each call clears what it needs zeroed on its own
+ * stream first.  Two calls whose work overlaps on the GPU (different streams,
+ * or different threads and streams) race on it -- keep them on one stream or
+ * order them with events.  Non-finite inputs give an unspecified result. */
+#define TGRAD_NOALLOC_MAX_NUMEL (1ll << 26)
+tgrad_status tgrad_select_topk_noalloc(const void* d_grad, int64_t numel, int64_t k, int32_t wg_dtype,
+                                       uint32_t* d_omega, void* d_values, void* cuda_stream);
 
 /* Kernels launched by this library since it was loaded (host-side counter). */
 int64_t tgrad_launch_count(void);

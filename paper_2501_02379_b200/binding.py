@@ -19,6 +19,8 @@ NUM_STAGES = 5
 STAGE_NAMES = ["proj_tail", "proj_chain", "adam_core", "back_chain", "back_tail"]
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BUFFER_TOO_SMALL, ERR_CUDA, ERR_NO_CONVERGE, ERR_NONFINITE, ERR_BAD_STATE = range(8)
+ERR_TOO_LARGE = 8
+NOALLOC_MAX_NUMEL = 1 << 26
 FLAG_NO_CONVERGE, FLAG_NONFINITE = 1, 2
 C64, C32H = 0, 1
 WHAT_OMEGA, WHAT_M_L, WHAT_V_L, WHAT_M_S, WHAT_V_S, WHAT_CORE, WHAT_N_L, WHAT_N_S = 1, 2, 3, 4, 5, 6, 7, 8
@@ -54,7 +56,7 @@ EXPORTS = [
     "tgrad_state_bytes", "tgrad_init_state", "tgrad_step", "tgrad_refresh_subspace", "tgrad_step_batched",
     "tgrad_refresh_subspace_batched", "tgrad_query_status", "tgrad_export_state", "tgrad_import_state",
     "tgrad_set_step", "tgrad_destroy_state", "tgrad_status_string", "tgrad_launch_count",
-    "tgrad_set_stage_timing", "tgrad_get_stage_times",
+    "tgrad_set_stage_timing", "tgrad_get_stage_times", "tgrad_select_topk_noalloc",
 ]
 
 
@@ -85,6 +87,7 @@ def lib() -> C.CDLL:
         l.tgrad_launch_count.restype = C.c_int64
         l.tgrad_set_stage_timing.argtypes = [vp, C.c_int32]
         l.tgrad_get_stage_times.argtypes = [vp, vp, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+        l.tgrad_select_topk_noalloc.argtypes = [vp, C.c_int64, C.c_int64, C.c_int32, vp, vp, vp]
         for name in EXPORTS:
             if name not in ("tgrad_status_string", "tgrad_launch_count"):
                 getattr(l, name).restype = C.c_int
@@ -253,3 +256,14 @@ def refresh_subspace_batched(states: Sequence[TgradState], grads, stream=None):
     hs = (C.c_void_p * n)(*[s.handle for s in states])
     gs = (C.c_void_p * n)(*[g.data_ptr() for g in grads])
     _check(lib().tgrad_refresh_subspace_batched(hs, gs, n, _stream_ptr(stream)), "tgrad_refresh_subspace_batched")
+
+
+def select_topk_noalloc(grad, numel: int, k: int, omega_out, values_out, half_storage: bool = False, stream=None):
+    """Top-k index set and values of `grad` through the entry point that allocates nothing:
+    its scratch is a fixed array inside the library, so it serves callers that must not call
+    cudaMalloc (allocator hooks, fully pre-partitioned device memory).  `omega_out` (k x uint32)
+    and `values_out` (k x complex64 as float pairs) are device tensors the caller already owns.
+    Calls share that scratch: keep them on one stream."""
+    _check(lib().tgrad_select_topk_noalloc(grad.data_ptr(), int(numel), int(k), C32H if half_storage else C64,
+                                           omega_out.data_ptr() if k else None, values_out.data_ptr() if k else None,
+                                           _stream_ptr(stream)), "tgrad_select_topk_noalloc")

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "../../include/tgrad.h"
@@ -702,6 +703,7 @@ const char* tgrad_status_string(tgrad_status s) {
     case TGRAD_ERR_NO_CONVERGE: return "eigensolver did not converge";
     case TGRAD_ERR_NONFINITE: return "non-finite gradient";
     case TGRAD_ERR_BAD_STATE: return "state has no subspace yet";
+    case TGRAD_ERR_TOO_LARGE: return "input exceeds the built-in scratch of the allocation-free entry point";
     default: return "unknown status";
   }
 }
@@ -709,3 +711,85 @@ const char* tgrad_status_string(tgrad_status s) {
 int64_t tgrad_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free top-k selection.  Its scratch is a fixed array in the device image; the name
+// below is usable as an address in device code only -- host code asks the runtime for the
+// device address (once per device) and hands that to the kernels.
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr uint64_t kNaMaxNumel = (uint64_t)TGRAD_NOALLOC_MAX_NUMEL;
+constexpr uint32_t kNaMaxBlocks = (uint32_t)(kNaMaxNumel / kChunk);
+struct NoAllocScratch {
+  SelState sel;
+  int flags[4];
+  uint32_t hist[3 * kSelMaxBins];
+  uint32_t blk[2 * kNaMaxBlocks];
+};
+constexpr int kNaMaxDevices = 64;
+std::mutex g_na_mu;
+void* g_na_addr[kNaMaxDevices];
+int g_na_sm[kNaMaxDevices];
+}  // namespace
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+namespace {
+// Device address of the scratch array on the current device; looked up on the first call per device.
+tgrad_status noalloc_scratch(NoAllocScratch** out, int* sm_count) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TGRAD_ERR_CUDA;
+  if (dev < 0 || dev >= kNaMaxDevices) return TGRAD_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_na_mu);
+  if (!g_na_addr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) return TGRAD_ERR_CUDA;
+    int sm = 0;
+    if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm < 1) return TGRAD_ERR_CUDA;
+    g_na_addr[dev] = ptr; g_na_sm[dev] = sm;
+  }
+  *out = static_cast<NoAllocScratch*>(g_na_addr[dev]);
+  *sm_count = g_na_sm[dev];
+  return TGRAD_OK;
+}
+
+template <class S>
+tgrad_status select_noalloc_impl(const void* d_grad, uint32_t n, uint32_t k, uint32_t* d_omega, cf* d_values,
+                                 NoAllocScratch* sc, int sm, cudaStream_t st) {
+  const uint32_t nblk = (n + kChunk - 1) / kChunk;
+  uint32_t* blk_gt = sc->blk;
+  uint32_t* blk_eq = sc->blk + nblk;
+  // the histograms and the flag word must start at zero; everything else is overwritten before it is read
+  if (cudaMemsetAsync(sc->flags, 0, sizeof(sc->flags) + sizeof(sc->hist), st) != cudaSuccess) return TGRAD_ERR_CUDA;
+  sel_init_kernel<<<1, 1, 0, st>>>(&sc->sel, k); TG_LAUNCH_CHECK();
+  const uint64_t want = ((uint64_t)n + 511) / 512;
+  const int hgrid = (int)(want < (uint64_t)sm * 8 ? want : (uint64_t)sm * 8);
+  for (int pass = 0; pass < 3; ++pass) {
+    sel_hist_kernel<S><<<hgrid, 512, 0, st>>>(d_grad, n, pass, &sc->sel, sc->hist + pass * kSelMaxBins, sc->flags);
+    TG_LAUNCH_CHECK();
+    sel_pick_kernel<<<1, 1024, 0, st>>>(sc->hist + pass * kSelMaxBins, pass, &sc->sel); TG_LAUNCH_CHECK();
+  }
+  sel_count_kernel<S><<<nblk, kChunkThreads, 0, st>>>(d_grad, n, &sc->sel, blk_gt, blk_eq); TG_LAUNCH_CHECK();
+  sel_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, nblk); TG_LAUNCH_CHECK();
+  sel_compact_kernel<S><<<nblk, kChunkThreads, 0, st>>>(d_grad, n, &sc->sel, blk_gt, blk_eq, d_omega, d_values, k);
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
+}
+}  // namespace
+
+extern "C" tgrad_status tgrad_select_topk_noalloc(const void* d_grad, int64_t numel, int64_t k, int32_t wg_dtype,
+                                                  uint32_t* d_omega, void* d_values, void* cuda_stream) {
+  if (numel < 1 || k < 0 || k > numel) return TGRAD_ERR_INVALID_ARG;
+  if (wg_dtype != TGRAD_C64 && wg_dtype != TGRAD_C32H) return TGRAD_ERR_INVALID_ARG;
+  if ((uint64_t)numel > kNaMaxNumel) return TGRAD_ERR_TOO_LARGE;
+  if (!d_grad || (k > 0 && (!d_omega || !d_values))) return TGRAD_ERR_INVALID_ARG;
+  if (k == 0) return TGRAD_OK;
+  NoAllocScratch* sc = nullptr;
+  int sm = 0;
+  tgrad_status r = noalloc_scratch(&sc, &sm);
+  if (r != TGRAD_OK) return r;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  return wg_dtype == TGRAD_C64
+             ? select_noalloc_impl<StoreC64>(d_grad, (uint32_t)numel, (uint32_t)k, d_omega, static_cast<cf*>(d_values), sc, sm, st)
+             : select_noalloc_impl<StoreC32H>(d_grad, (uint32_t)numel, (uint32_t)k, d_omega, static_cast<cf*>(d_values), sc, sm, st);
+}
