@@ -34,7 +34,8 @@ struct Layout {
   uint32_t nslab, E;          // slabs of the trailing two modes, entries per slab
   // workspace block
   size_t w_ns, w_gs, w_core, w_nl, w_bufa, w_bufb, w_sel, w_hist, w_blk, w_gram[TGRAD_MAX_NDIM], w_jac[TGRAD_MAX_NDIM],
-      w_v[TGRAD_MAX_NDIM], w_partial, w_total;
+      w_v[TGRAD_MAX_NDIM], w_log[TGRAD_MAX_NDIM], w_lam[TGRAD_MAX_NDIM], w_partial, w_total;
+  bool jac_fast[TGRAD_MAX_NDIM];    // eigensolver with the matrix in shared memory and a rotation log
   uint64_t numel, P, tsize;   // entries, core entries, entries of the tail-contracted tensor
   uint32_t nblk;              // compaction blocks
   int gram_splits[TGRAD_MAX_NDIM];
@@ -130,6 +131,11 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
     L.w_gram[n] = o; o = align_up(o + sq);   // A_n, kept for inspection
     L.w_jac[n] = o; o = align_up(o + sq);    // working copy the solver diagonalises
     L.w_v[n] = o; o = align_up(o + sq);      // accumulated rotations
+    const int sweeps = c->jacobi_max_sweeps > 0 ? c->jacobi_max_sweeps : 30;
+    const size_t logb = jac_log_entries((int)c->dims[n], sweeps) * sizeof(float4);
+    L.jac_fast[n] = c->dims[n] <= JAC_SMEM_MAX_N && logb <= ((size_t)64 << 20);
+    L.w_log[n] = o; if (L.jac_fast[n]) o = align_up(o + logb);
+    L.w_lam[n] = o; o = align_up(o + (size_t)c->dims[n] * 4);
     plan_gram(c, n, sm, L.gram_chunks[n], L.gram_cps[n], L.gram_splits[n]);
     size_t pb = sq * L.gram_splits[n];
     if (pb > partial) partial = pb;
@@ -352,6 +358,9 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   }
   cf* partial = reinterpret_cast<cf*>(s->dw + L.w_partial);
   JacobiParams jp; memset(&jp, 0, sizeof(jp));
+  JacobiFastParams fp; memset(&fp, 0, sizeof(fp));
+  int nslow = 0;
+  size_t fast_smem = 0;
   for (int m = 0; m < N; ++m) {
     uint64_t O = 1, C = 1;
     for (int q = 0; q < m; ++q) O *= c.dims[q];
@@ -364,18 +373,41 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
                                                  L.gram_cps[m], partial);
     TG_LAUNCH_CHECK();
     gram_reduce_kernel<<<(In * In + 255) / 256, 256, 0, st>>>(partial, L.gram_splits[m], In, A); TG_LAUNCH_CHECK();
-    jp.mode[m].A = reinterpret_cast<cf*>(s->dw + L.w_jac[m]);
-    jp.mode[m].V = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
-    jp.mode[m].U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
-    jp.mode[m].n = In; jp.mode[m].r = c.ranks[m];
-    if (cudaMemcpyAsync(s->dw + L.w_jac[m], A, (size_t)In * In * 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-      return TGRAD_ERR_CUDA;
+    if (L.jac_fast[m]) {
+      JacobiFastMode& fm = fp.mode[fp.nmodes++];
+      fm.A = A;
+      fm.log = reinterpret_cast<float4*>(s->dw + L.w_log[m]);
+      fm.lam = reinterpret_cast<float*>(s->dw + L.w_lam[m]);
+      fm.V = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
+      fm.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
+      fm.n = In; fm.r = c.ranks[m]; fm.index = m; fm.row0 = fp.total_rows;
+      fp.total_rows += In;
+      const size_t sm = jac_sweeps_smem(In);
+      if (sm > fast_smem) fast_smem = sm;
+    } else {
+      JacobiMode& jm = jp.mode[nslow];
+      jp.index[nslow++] = m;
+      jm.A = reinterpret_cast<cf*>(s->dw + L.w_jac[m]);
+      jm.V = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
+      jm.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
+      jm.n = In; jm.r = c.ranks[m];
+      if (cudaMemcpyAsync(s->dw + L.w_jac[m], A, (size_t)In * In * 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return TGRAD_ERR_CUDA;
+    }
   }
   if (k > 0) { scatter_restore_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, g_s, k); TG_LAUNCH_CHECK(); }
-  jp.max_sweeps = c.jacobi_max_sweeps > 0 ? c.jacobi_max_sweeps : 30;
-  jp.tol = c.jacobi_tol > 0.f ? c.jacobi_tol : 1e-6f;
-  jp.flags = flags;
-  jacobi_kernel<<<N, JAC_THREADS, 0, st>>>(jp); TG_LAUNCH_CHECK();
+  const int max_sweeps = c.jacobi_max_sweeps > 0 ? c.jacobi_max_sweeps : 30;
+  const float tol = c.jacobi_tol > 0.f ? c.jacobi_tol : 1e-6f;
+  if (nslow) {
+    jp.max_sweeps = max_sweeps; jp.tol = tol; jp.flags = flags;
+    jacobi_kernel<<<nslow, JAC_THREADS, 0, st>>>(jp); TG_LAUNCH_CHECK();
+  }
+  if (fp.nmodes) {
+    fp.max_sweeps = max_sweeps; fp.tol = tol; fp.flags = flags;
+    jacobi_sweeps_kernel<<<fp.nmodes, JAC_THREADS, fast_smem, st>>>(fp); TG_LAUNCH_CHECK();
+    jacobi_vectors_kernel<<<(fp.total_rows + 7) / 8, 256, 0, st>>>(fp); TG_LAUNCH_CHECK();
+    jacobi_factors_kernel<<<fp.nmodes, JAC_THREADS, 0, st>>>(fp); TG_LAUNCH_CHECK();
+  }
   s->have_subspace = true;
   return TGRAD_OK;
 }
@@ -387,8 +419,8 @@ tgrad_status do_refresh(tgrad_state* s, void* d_grad, cudaStream_t st) {
 tgrad_status mode_product(bool conj_t, const cf* in, cf* out, const cf* U, uint64_t O, int M, int K, uint64_t C,
                           int r_n, cudaStream_t st) {
   dim3 grid((unsigned)((C + MP_BC - 1) / MP_BC), (unsigned)((M + MP_BM - 1) / MP_BM), (unsigned)O);
-  if (conj_t) mode_product_kernel<true><<<grid, 256, 0, st>>>(in, out, U, M, K, (int)C, r_n);
-  else mode_product_kernel<false><<<grid, 256, 0, st>>>(in, out, U, M, K, (int)C, r_n);
+  if (conj_t) mode_product_kernel<true><<<grid, MP_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
+  else mode_product_kernel<false><<<grid, MP_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
@@ -527,6 +559,8 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
   st->sm_count = sm;
   s = plan_tail(st);
   if (s != TGRAD_OK) { delete st; return s; }
+  if (cudaFuncSetAttribute(jacobi_sweeps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)jac_sweeps_smem(JAC_SMEM_MAX_N)) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   // Algorithm 1 initialisation: zero moments (and flags, Omega, factors for determinism)
   if (cudaMemsetAsync(d_persistent, 0, L.p_total, stream) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
