@@ -3,109 +3,193 @@
 // (TuckerFactors of Algorithm 1: leading left singular vectors of the mode-n
 // unfolding = leading eigenvectors of A_n).  The Gram matrix does not depend on
 // the column order of the unfolding, so the tensor is read in place as
-// [O][I_n][C] with C contiguous.
+// [O][I_n][C] with C contiguous and the contraction index k = (o, c) flattened.
 //
-// Only tile pairs on or above the diagonal are computed; split-K partial sums
-// go to scratch and are reduced in a fixed order (deterministic result).
+// Tensor cores, TF32 inputs, fp32 accumulation.  With rows as interleaved real
+// vectors X'[a] = (re, im, re, im, ...):
+//   Re A[a][b] = X'[a] . X'[b],   Im A[a][b] = X'[a] . Y'[b],  Y'[b] = (-im, re, -im, re, ...)
+// so one loaded fragment of row b serves both products.  A block owns a 64 x 64
+// tile of A (only tiles on or above the diagonal are computed), a warp 32 x 32
+// of it; K is split over blockIdx.y, partial sums go to scratch and are reduced
+// in a fixed order (deterministic result).
+// SPLIT = false: inputs rounded to TF32 once (relative error of an entry of A about
+// 2^-11.5 / sqrt(K) of the diagonal scale: used when K is large).  SPLIT = true:
+// x = hi + lo and the three products hi*hi, hi*lo, lo*hi (fp32-grade, for short K).
 #pragma once
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace tg {
 
-constexpr int GR_T = 64;     // output tile (rows a x cols b)
-constexpr int GR_KT = 16;    // K chunk
-constexpr int GR_LD = 66;    // padded tile row length in shared memory (keeps 16-byte alignment)
+constexpr int GR_T = 64;      // output tile (rows a x cols b)
+constexpr int GR_KT = 32;     // complex k per shared-memory chunk
+constexpr int GR_LD = 36;     // padded chunk row length: fragment loads (8 rows x 4 k) hit distinct banks
+constexpr int GR_THREADS = 128;
 
-template <class S>
-__global__ void __launch_bounds__(256) gram_partial_kernel(const void* __restrict__ g, int In, uint32_t O, uint32_t C,
-                                                           uint32_t chunks_total, uint32_t chunks_per_split,
-                                                           cf* __restrict__ partial) {
+__device__ __forceinline__ float gr_tf32(float x) { return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xffffe000u); }
+
+constexpr size_t GR_SMEM = 2 * 2 * GR_T * GR_LD * sizeof(cf);      // two stages of (Xa, Xb)
+
+template <class S, bool SPLIT>
+__global__ void __launch_bounds__(GR_THREADS) gram_partial_kernel(const void* __restrict__ g, int In, uint32_t O, uint32_t C,
+                                                                  uint32_t chunks_total, uint32_t chunks_per_split,
+                                                                  cf* __restrict__ partial) {
   const int T = (In + GR_T - 1) / GR_T;
   const int ta = blockIdx.x / T, tb = blockIdx.x % T;
   if (ta > tb) return;
-  __shared__ __align__(16) cf Xa[GR_KT][GR_LD];
-  __shared__ __align__(16) cf Xb[GR_KT][GR_LD];
-  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  extern __shared__ __align__(16) unsigned char gsm[];
+  typedef cf Tile[GR_T][GR_LD];
+  Tile* XA = reinterpret_cast<Tile*>(gsm);            // [2]
+  Tile* XBs = XA + 2;                                 // [2]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t = lane & 3;
+  const int wm = warp >> 1, wn = warp & 1;           // 2 x 2 warps of 32 x 32
   const int a0 = ta * GR_T, b0 = tb * GR_T;
-  const uint32_t cpo = (C + GR_KT - 1) / GR_KT;   // chunks per o when C > 1
+  const bool diag = ta == tb;
+  const uint32_t K32 = O * C;                        // the tensor has fewer than 2^32 entries
   uint32_t ch0 = blockIdx.y * chunks_per_split;
   uint32_t ch1 = ch0 + chunks_per_split; if (ch1 > chunks_total) ch1 = chunks_total;
-  cf acc[4][4];
+  // which 16-row / 8-column sub-tiles of this warp hold any row of A
+  bool mok[2], nok[4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int mt = 0; mt < 2; ++mt) mok[mt] = a0 + wm * 32 + mt * 16 < In;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = make_float2(0.f, 0.f);
+  for (int nt = 0; nt < 4; ++nt) nok[nt] = b0 + wn * 32 + nt * 8 < In;
+  float are[2][4][4], aim[2][4][4];
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { are[mt][nt][i] = 0.f; aim[mt][nt][i] = 0.f; }
+  // loader mapping (fixed per thread): lanes along k when rows are runs of k -- a thread keeps one k of
+  // the chunk and walks 16 rows; along the rows when C == 1 -- it keeps one row and walks 16 k
+  const bool along_k = C > 1;
+  const int ld_kc = along_k ? (tid % GR_KT) : 0, ld_row = along_k ? (tid / GR_KT) : (tid % GR_T);
+  const int ld_k2 = along_k ? 0 : (tid / GR_T);
+  const unsigned char* gb = static_cast<const unsigned char*>(g);
 
-  for (uint32_t ch = ch0; ch < ch1; ++ch) {
-    if (C == 1) {
-      // last mode: K index is o itself, rows of the tile are contiguous in memory
-      const uint32_t o0 = ch * GR_KT;
-      for (int i = tid; i < GR_KT * GR_T; i += 256) {
-        int aa = i % GR_T, kk = i / GR_T;
-        uint32_t o = o0 + kk;
-        cf va = make_float2(0.f, 0.f), vb = va;
-        if (o < O) {
-          if (a0 + aa < In) va = S::load(g, (size_t)o * In + a0 + aa);
-          if (b0 + aa < In) vb = S::load(g, (size_t)o * In + b0 + aa);
+  // chunk ch -> stage st: asynchronous 8-byte copies for fp32 storage (zero-filled outside the tensor),
+  // loads through registers with widening for fp16 storage
+  auto load_chunk = [&](uint32_t ch, int st) {
+    const uint32_t kk0 = ch * GR_KT;
+    cf (*xa)[GR_LD] = XA[st];
+    cf (*xb)[GR_LD] = XBs[st];
+    if (along_k) {
+      const uint32_t kk = kk0 + ld_kc;
+      const bool kok = kk < K32;
+      const uint32_t o = kok ? kk / C : 0, c = kok ? kk - o * C : 0;
+      const size_t base = (size_t)o * In * C + c;
+#pragma unroll 4
+      for (int i = 0; i < GR_T / (GR_THREADS / GR_KT); ++i) {
+        const int row = ld_row + i * (GR_THREADS / GR_KT);
+        const bool va = kok && a0 + row < In, vb = kok && b0 + row < In;
+        if (S::kBytes == 8) {
+          cp_async8(&xa[row][ld_kc], va ? gb + (base + (size_t)(a0 + row) * C) * 8 : gb, va ? 8u : 0u);
+          if (!diag) cp_async8(&xb[row][ld_kc], vb ? gb + (base + (size_t)(b0 + row) * C) * 8 : gb, vb ? 8u : 0u);
+        } else {
+          xa[row][ld_kc] = va ? S::load(g, base + (size_t)(a0 + row) * C) : make_float2(0.f, 0.f);
+          if (!diag) xb[row][ld_kc] = vb ? S::load(g, base + (size_t)(b0 + row) * C) : make_float2(0.f, 0.f);
         }
-        Xa[kk][aa] = va; Xb[kk][aa] = vb;
       }
     } else {
-      const uint32_t o = ch / cpo, c0 = (ch - o * cpo) * GR_KT;
-      for (int i = tid; i < GR_KT * GR_T; i += 256) {
-        int kk = i % GR_KT, aa = i / GR_KT;
-        uint32_t c = c0 + kk;
-        cf va = make_float2(0.f, 0.f), vb = va;
-        if (c < C) {
-          if (a0 + aa < In) va = S::load(g, ((size_t)o * In + a0 + aa) * C + c);
-          if (b0 + aa < In) vb = S::load(g, ((size_t)o * In + b0 + aa) * C + c);
+#pragma unroll 4
+      for (int i = 0; i < GR_KT / (GR_THREADS / GR_T); ++i) {
+        const int kc = ld_k2 + i * (GR_THREADS / GR_T);
+        const uint32_t kk = kk0 + kc;
+        const bool va = kk < K32 && a0 + ld_row < In, vb = kk < K32 && b0 + ld_row < In;
+        if (S::kBytes == 8) {
+          cp_async8(&xa[ld_row][kc], va ? gb + ((size_t)kk * In + a0 + ld_row) * 8 : gb, va ? 8u : 0u);
+          if (!diag) cp_async8(&xb[ld_row][kc], vb ? gb + ((size_t)kk * In + b0 + ld_row) * 8 : gb, vb ? 8u : 0u);
+        } else {
+          xa[ld_row][kc] = va ? S::load(g, (size_t)kk * In + a0 + ld_row) : make_float2(0.f, 0.f);
+          if (!diag) xb[ld_row][kc] = vb ? S::load(g, (size_t)kk * In + b0 + ld_row) : make_float2(0.f, 0.f);
         }
-        Xa[kk][aa] = va; Xb[kk][aa] = vb;
       }
     }
-    __syncthreads();
+    cp_async_commit();
+  };
+
+  if (ch0 < ch1) load_chunk(ch0, 0);
+  int st = 0;
+  for (uint32_t ch = ch0; ch < ch1; ++ch, st ^= 1) {
+    cp_async_wait<0>();
+    __syncthreads();                                   // chunk ch has landed; everyone is done with stage st^1
+    if (ch + 1 < ch1) load_chunk(ch + 1, st ^ 1);
+    const cf (*Xa)[GR_LD] = XA[st];
+    const cf (*XB)[GR_LD] = diag ? XA[st] : XBs[st];
 #pragma unroll
-    for (int kk = 0; kk < GR_KT; ++kk) {
-      float4 p0 = *reinterpret_cast<const float4*>(&Xa[kk][ty * 4]);
-      float4 p1 = *reinterpret_cast<const float4*>(&Xa[kk][ty * 4 + 2]);
-      float4 q0 = *reinterpret_cast<const float4*>(&Xb[kk][tx * 4]);
-      float4 q1 = *reinterpret_cast<const float4*>(&Xb[kk][tx * 4 + 2]);
-      cf a[4] = {make_float2(p0.x, p0.y), make_float2(p0.z, p0.w), make_float2(p1.x, p1.y), make_float2(p1.z, p1.w)};
-      cf b[4] = {make_float2(q0.x, q0.y), make_float2(q0.z, q0.w), make_float2(q1.x, q1.y), make_float2(q1.z, q1.w)};
+    for (int ks = 0; ks < GR_KT / 4; ++ks) {
+      const int kc = ks * 4 + t;
+      // A fragments: (row g, re), (row g+8, re), (row g, im), (row g+8, im)
+      float ah[2][4], al[2][4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int mt = 0; mt < 2; ++mt) {
+        const cf x0 = Xa[wm * 32 + mt * 16 + gq][kc], x1 = Xa[wm * 32 + mt * 16 + gq + 8][kc];
+        ah[mt][0] = gr_tf32(x0.x); ah[mt][1] = gr_tf32(x1.x); ah[mt][2] = gr_tf32(x0.y); ah[mt][3] = gr_tf32(x1.y);
+        if (SPLIT) { al[mt][0] = x0.x - ah[mt][0]; al[mt][1] = x1.x - ah[mt][1]; al[mt][2] = x0.y - ah[mt][2]; al[mt][3] = x1.y - ah[mt][3]; }
+      }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) cfma_conj(acc[i][j], a[i], b[j]);
+      for (int nt = 0; nt < 4; ++nt) {
+        if (!nok[nt]) continue;
+        const cf y = XB[wn * 32 + nt * 8 + gq][kc];
+        const float yh0 = gr_tf32(y.x), yh1 = gr_tf32(y.y);
+        const float yl0 = y.x - yh0, yl1 = y.y - yh1;
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          if (!mok[mt]) continue;
+          mma_tf32(are[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], yh0, yh1);
+          mma_tf32(aim[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], -yh1, yh0);
+          if (SPLIT) {
+            mma_tf32(are[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], yl0, yl1);
+            mma_tf32(aim[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], -yl1, yl0);
+            mma_tf32(are[mt][nt], al[mt][0], al[mt][1], al[mt][2], al[mt][3], yh0, yh1);
+            mma_tf32(aim[mt][nt], al[mt][0], al[mt][1], al[mt][2], al[mt][3], -yh1, yh0);
+          }
+        }
+      }
     }
-    __syncthreads();
   }
+  // accumulator (row g | g+8, col 2t | 2t+1) -> partial[split][a][b]
   cf* out = partial + (size_t)blockIdx.y * In * In;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    int a = a0 + ty * 4 + i;
-    if (a >= In) continue;
+  for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      int b = b0 + tx * 4 + j;
-      if (b < In) out[(size_t)a * In + b] = acc[i][j];
-    }
-  }
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int a = a0 + wm * 32 + mt * 16 + gq + (i >> 1) * 8, b = b0 + wn * 32 + nt * 8 + 2 * t + (i & 1);
+        if (a < In && b < In) out[(size_t)a * In + b] = make_float2(are[mt][nt][i], aim[mt][nt][i]);
+      }
 }
 
-// Sum the split-K partials in split order; mirror the upper triangle.
-__global__ void gram_reduce_kernel(const cf* __restrict__ partial, int splits, int In, cf* __restrict__ A) {
-  int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= In * In) return;
-  int a = idx / In, b = idx % In;
-  if (a > b) return;
+// Sum the split-K partials, always in the same order (four interleaved running sums per entry, then
+// those four in order): deterministic.  Mirrors the upper triangle.
+constexpr int GRR_E = 64, GRR_G = 4;     // entries per block, split groups
+__global__ void __launch_bounds__(GRR_E * GRR_G) gram_reduce_kernel(const cf* __restrict__ partial, int splits, int In,
+                                                                   cf* __restrict__ A) {
+  __shared__ cf part[GRR_G][GRR_E];
+  const int e = threadIdx.x % GRR_E, sg = threadIdx.x / GRR_E;
+  const int idx = blockIdx.x * GRR_E + e;
+  const int n2 = In * In;
+  const int a = idx < n2 ? idx / In : 0, b = idx < n2 ? idx - a * In : 0;
+  const bool live = idx < n2 && a <= b;
   float sx = 0.f, sy = 0.f;
-  for (int s = 0; s < splits; ++s) {
-    cf v = partial[(size_t)s * In * In + idx];
-    sx += v.x; sy += v.y;
+  if (live) {
+    const cf* p = partial + idx;
+#pragma unroll 4
+    for (int s = sg; s < splits; s += GRR_G) {
+      cf v = p[(size_t)s * n2];
+      sx += v.x; sy += v.y;
+    }
   }
-  if (a == b) { A[idx] = make_float2(sx, 0.f); return; }
-  A[idx] = make_float2(sx, sy);
-  A[(size_t)b * In + a] = make_float2(sx, -sy);
+  part[sg][e] = make_float2(sx, sy);
+  __syncthreads();
+  if (sg == 0 && live) {
+    for (int q = 1; q < GRR_G; ++q) { sx += part[q][e].x; sy += part[q][e].y; }
+    if (a == b) { A[idx] = make_float2(sx, 0.f); return; }
+    A[idx] = make_float2(sx, sy);
+    A[(size_t)b * In + a] = make_float2(sx, -sy);
+  }
 }
 
 }  // namespace tg

@@ -220,6 +220,17 @@ __device__ __forceinline__ void jac_pair(int m, int stage, int tb, int& p, int& 
   if (p > q) { int t = p; p = q; q = t; }
 }
 
+// One Newton step of (x, y) towards x^2 + y^2 = 1.  The defect e = 1 - x^2 - y^2 is formed without
+// rounding (products split into rounded part and exact remainder; the two subtractions are exact
+// because x^2 + y^2 is already within a few ulp of 1), so the step leaves only the unbiased final
+// rounding of x and y: the accumulated eigenvectors then lose orthonormality like a random walk.
+__device__ __forceinline__ void jac_unit(float& x, float& y) {
+  const float p = x * x, ep = fmaf(x, x, -p), q = y * y, eq = fmaf(y, y, -q);
+  const float hi = fmaxf(p, q), lo = fminf(p, q);
+  const float e = ((1.f - hi) - lo) - (ep + eq);
+  x = fmaf(0.5f * e, x, x); y = fmaf(0.5f * e, y, y);
+}
+
 // Rotation that annihilates the (p, q) entry b of the Hermitian 2 x 2 block [[a, b], [conj(b), d]], in fp32.
 // c and s (and the phase g = conj(b)/|b|) get one Newton step towards c^2 + s^2 = 1 (|g| = 1): what keeps the
 // accumulated eigenvectors orthonormal over thousands of rotations is that normalisation, not the angle.
@@ -227,12 +238,10 @@ __device__ __forceinline__ void jac_rotation(float a, float d, cf b, float absb,
   const float tau = (d - a) / (2.f * absb);
   const float t = copysignf(1.f, tau) / (fabsf(tau) + sqrtf(fmaf(tau, tau, 1.f)));
   float c = rsqrtf(fmaf(t, t, 1.f)), s = t * c;
-  float e = fmaf(-c, c, fmaf(-s, s, 1.f));
-  c = fmaf(0.5f * e, c, c); s = fmaf(0.5f * e, s, s);
+  jac_unit(c, s);
   const float inv = 1.f / absb;
   float gx = b.x * inv, gy = -b.y * inv;
-  e = fmaf(-gx, gx, fmaf(-gy, gy, 1.f));
-  gx = fmaf(0.5f * e, gx, gx); gy = fmaf(0.5f * e, gy, gy);
+  jac_unit(gx, gy);
   R.c = c; R.s = s; R.gx = gx; R.gy = gy;
   R.npp = a - t * absb; R.nqq = d + t * absb;
 }

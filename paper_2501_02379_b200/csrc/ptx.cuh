@@ -65,6 +65,14 @@ __device__ __forceinline__ void bulk_wait_all() {
 // make generic-proxy writes to shared memory visible to the async proxy (before a bulk store)
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// 8-byte asynchronous copy global -> shared (Ampere-style cp.async); src_bytes = 0 writes zeros instead
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gmem_src, uint32_t src_bytes) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // fp32 -> tf32 (round to nearest); the result is an fp32 bit pattern with the low 13 mantissa bits zero
 __device__ __forceinline__ float tf32_hi(float x) {
   uint32_t r;

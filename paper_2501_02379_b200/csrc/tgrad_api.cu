@@ -82,12 +82,12 @@ void plan_gram(const tgrad_config* c, int n, int sm, uint32_t& chunks, uint32_t&
   uint64_t O = 1, C = 1;
   for (int m = 0; m < n; ++m) O *= c->dims[m];
   for (int m = n + 1; m < c->ndim; ++m) C *= c->dims[m];
-  uint64_t total = (C == 1) ? (O + GR_KT - 1) / GR_KT : O * ((C + GR_KT - 1) / GR_KT);
+  uint64_t total = (O * C + GR_KT - 1) / GR_KT;      // the contraction index (o, c) is flattened
   int T = (int)((c->dims[n] + GR_T - 1) / GR_T);
   int tiles = T * (T + 1) / 2;
-  uint64_t want = (uint64_t)(4 * sm + tiles - 1) / tiles;
+  uint64_t want = (uint64_t)(6 * sm + tiles - 1) / tiles;
   if (want < 1) want = 1;
-  if (want > 256) want = 256;
+  if (want > 1024) want = 1024;
   if (want > total) want = total;
   uint64_t per = (total + want - 1) / want;
   chunks = (uint32_t)total; cps = (uint32_t)per; splits = (int)((total + per - 1) / per);
@@ -369,10 +369,15 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
     const int T = (In + GR_T - 1) / GR_T;
     cf* A = reinterpret_cast<cf*>(s->dw + L.w_gram[m]);
     dim3 grid(T * T, L.gram_splits[m]);
-    gram_partial_kernel<S><<<grid, 256, 0, st>>>(d_grad, In, (uint32_t)O, (uint32_t)C, L.gram_chunks[m],
-                                                 L.gram_cps[m], partial);
+    // long contractions average the TF32 input rounding away; short ones get the split-precision products
+    if (O * C >= 16384)
+      gram_partial_kernel<S, false><<<grid, GR_THREADS, GR_SMEM, st>>>(d_grad, In, (uint32_t)O, (uint32_t)C, L.gram_chunks[m],
+                                                                 L.gram_cps[m], partial);
+    else
+      gram_partial_kernel<S, true><<<grid, GR_THREADS, GR_SMEM, st>>>(d_grad, In, (uint32_t)O, (uint32_t)C, L.gram_chunks[m],
+                                                                L.gram_cps[m], partial);
     TG_LAUNCH_CHECK();
-    gram_reduce_kernel<<<(In * In + 255) / 256, 256, 0, st>>>(partial, L.gram_splits[m], In, A); TG_LAUNCH_CHECK();
+    gram_reduce_kernel<<<(In * In + GRR_E - 1) / GRR_E, GRR_E * GRR_G, 0, st>>>(partial, L.gram_splits[m], In, A); TG_LAUNCH_CHECK();
     if (L.jac_fast[m]) {
       JacobiFastMode& fm = fp.mode[fp.nmodes++];
       fm.A = A;
@@ -559,6 +564,13 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
   st->sm_count = sm;
   s = plan_tail(st);
   if (s != TGRAD_OK) { delete st; return s; }
+  {
+    cudaError_t e1 = cudaFuncSetAttribute(gram_partial_kernel<StoreC64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GR_SMEM);
+    cudaError_t e2 = cudaFuncSetAttribute(gram_partial_kernel<StoreC64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GR_SMEM);
+    cudaError_t e3 = cudaFuncSetAttribute(gram_partial_kernel<StoreC32H, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GR_SMEM);
+    cudaError_t e4 = cudaFuncSetAttribute(gram_partial_kernel<StoreC32H, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GR_SMEM);
+    if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
+  }
   if (cudaFuncSetAttribute(jacobi_sweeps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)jac_sweeps_smem(JAC_SMEM_MAX_N)) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
