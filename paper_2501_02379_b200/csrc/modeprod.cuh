@@ -114,14 +114,21 @@ __global__ void __launch_bounds__(MP_THREADS) mode_product_kernel(const cf* __re
   }
 }
 
-// AdamUpdate of Algorithm 1 on the Tucker core: moments in place, N_L out.
-__global__ void adam_core_kernel(const cf* __restrict__ core, cf* __restrict__ m_l, float* __restrict__ v_l,
-                                 cf* __restrict__ n_l, uint32_t n, AdamScalars a) {
+// AdamUpdate of Algorithm 1 on the Tucker core (entries [0, n)) and, when the streaming kernel only
+// gathered them, on the ks sparse values (entries [n, n + ks)): moments in place, N_L / N_S out.
+__global__ void adam_kernel(const cf* __restrict__ core, cf* __restrict__ m_l, float* __restrict__ v_l,
+                            cf* __restrict__ n_l, uint32_t n, const cf* __restrict__ g_s, cf* __restrict__ m_s,
+                            float* __restrict__ v_s, cf* __restrict__ n_s, uint32_t ks, AdamScalars a) {
   uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) {
     cf m = m_l[i]; float v = v_l[i];
     cf r = adam_apply(core[i], m, v, a);
     m_l[i] = m; v_l[i] = v; n_l[i] = r;
+  } else if (i - n < ks) {
+    i -= n;
+    cf m = m_s[i]; float v = v_s[i];
+    cf r = adam_apply(g_s[i], m, v, a);
+    m_s[i] = m; v_s[i] = v; n_s[i] = r;
   }
 }
 

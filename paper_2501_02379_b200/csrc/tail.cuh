@@ -46,6 +46,7 @@ struct TailParams {
   const uint32_t* slab_ptr; // slab_ptr[s] = first Omega slot of slab s (nslab + 1 entries)
   int k;
   cf* m_s; float* v_s;   // sparse moments (proj)
+  cf* g_s;               // gathered sparse values (fast path: their Adam update runs in the Adam kernel)
   cf* n_s;               // normalised sparse update: written by proj, read by back
   cf* t;                 // proj: out T[s][ra][rb];  back: in T'[s][ra][rb]
   AdamScalars adam;

@@ -195,13 +195,13 @@ __global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_ker
   // ---- sparse side, software-pipelined: the next group's entry bounds and first entries are fetched one group ahead ----
   const bool sparse = p.k > 0;
   int b0 = 0, b1 = 0;
-  uint32_t pom = 0; cf pm = make_float2(0.f, 0.f); float pv = 0.f;
+  uint32_t pom = 0;
   if (sparse) {
     const uint32_t u = blockIdx.x;
     uint32_t e = (u + 1) * spi; if (e > nslab) e = nslab;
     b0 = (int)p.slab_ptr[u * spi]; b1 = (int)p.slab_ptr[e];
     const int j = b0 + tid;
-    if (j < b1) { pom = p.omega[j]; pm = p.m_s[j]; pv = p.v_s[j]; }
+    if (j < b1) pom = p.omega[j];
   }
 
   // sums the partials of iteration `itp` (group up) in warp order and writes T
@@ -242,22 +242,18 @@ __global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_ker
     float* xg = reinterpret_cast<float*>(smem + (size_t)buf * G.grp_stride);
     // ---- sparse part, before the barrier: gather and zero (the residual); one entry of the group per thread ----
     const int jcur = b0 + tid;
-    const bool have = sparse && ok && jcur < b1;
-    cf xsp = make_float2(0.f, 0.f);
     if (sparse && ok) {
+      // the gathered values go to the sparse-value buffer; their Adam update runs with the core's
       const uint32_t base = u * (uint32_t)spi * E;
-      if (have) {
+      if (jcur < b1) {
         cf* xp = reinterpret_cast<cf*>(xg) + (pom - base);
-        xsp = *xp;
+        p.g_s[jcur] = *xp;
         *xp = make_float2(0.f, 0.f);
       }
       for (int j = jcur + PJ_THREADS; j < b1; j += PJ_THREADS) {   // more entries than threads: not prefetched
         cf* xp = reinterpret_cast<cf*>(xg) + (p.omega[j] - base);
-        cf x = *xp;
+        p.g_s[j] = *xp;
         *xp = make_float2(0.f, 0.f);
-        cf m = p.m_s[j]; float v = p.v_s[j];
-        cf n = adam_apply(x, m, v, p.adam);
-        p.m_s[j] = m; p.v_s[j] = v; p.n_s[j] = n;
       }
       fence_async_smem();      // the zeroed entries were written through the generic proxy; a later bulk copy overwrites them
     }
@@ -338,16 +334,12 @@ __global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_ker
         rw[4 * (8 * mt + gq) + t] = make_float4(d2[mt][0][0] + d2[mt][1][0], d2[mt][0][2] + d2[mt][1][2],
                                                 d2[mt][0][1] + d2[mt][1][1], d2[mt][0][3] + d2[mt][1][3]);
     }
-    // ---- off the critical path: the previous group's T, this group's sparse Adam, the next group's entries ----
+    // ---- off the critical path: the previous group's T, the next group's entries ----
     if (it > 0) reduce_out(u - gstride, it - 1);
     if (sparse) {
-      if (have) {
-        cf n = adam_apply(xsp, pm, pv, p.adam);
-        p.m_s[jcur] = pm; p.v_s[jcur] = pv; p.n_s[jcur] = n;
-      }
       b0 = n0; b1 = n1;
       const int j = b0 + tid;
-      if (j < b1) { pom = p.omega[j]; pm = p.m_s[j]; pv = p.v_s[j]; }
+      if (j < b1) pom = p.omega[j];
     }
     pbuf = buf;
     if (++buf == nbuf) { buf = 0; phase ^= 1; }

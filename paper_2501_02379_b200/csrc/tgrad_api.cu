@@ -453,6 +453,7 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   p.m_s = reinterpret_cast<cf*>(s->dp + L.p_ms);
   p.v_s = reinterpret_cast<float*>(s->dp + L.p_vs);
   p.n_s = reinterpret_cast<cf*>(s->dw + L.w_ns);
+  p.g_s = reinterpret_cast<cf*>(s->dw + L.w_gs);
   p.adam = adam_scalars(c, s->t);
   p.s_low = (float)((double)c.lr * (double)c.alpha);
   p.s_sparse = (float)((double)c.lr * (double)c.lambda);
@@ -489,9 +490,13 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
     }
   }
   TG_MARK(2);
-  adam_core_kernel<<<(unsigned)((L.P + 255) / 256), 256, 0, st>>>(
-      core, reinterpret_cast<cf*>(s->dp + L.p_ml), reinterpret_cast<float*>(s->dp + L.p_vl), n_l, (uint32_t)L.P, p.adam);
-  TG_LAUNCH_CHECK();
+  {
+    const uint32_t ks = s->tail.tc ? (uint32_t)c.k : 0u;      // the general streaming kernel updates the sparse moments itself
+    adam_kernel<<<(unsigned)((L.P + ks + 255) / 256), 256, 0, st>>>(
+        core, reinterpret_cast<cf*>(s->dp + L.p_ml), reinterpret_cast<float*>(s->dp + L.p_vl), n_l, (uint32_t)L.P,
+        p.g_s, p.m_s, p.v_s, p.n_s, ks, p.adam);
+    TG_LAUNCH_CHECK();
+  }
   TG_MARK(3);
   // reconstruction: modes 1 .. N-2 on the small tensor, trailing two while streaming W
   const cf* tprime;
