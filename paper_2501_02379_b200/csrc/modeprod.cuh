@@ -15,24 +15,27 @@
 // current one is being multiplied.
 #pragma once
 #include "common.cuh"
+#include "ptx.cuh"
 #include "tail.cuh"
 
 namespace tg {
 
-constexpr int MP_BM = 32, MP_BC = 64, MP_BK = 16, MP_THREADS = 128;
+constexpr int MP_BM = 32, MP_BK = 16, MP_THREADS = 128;
 
-template <bool CONJ_T>
+// MP_BC = 64 (4 x 4 micro-tile) or 32 (4 x 2: twice the blocks, for products with few tiles)
+template <bool CONJ_T, int MP_BC>
 __global__ void __launch_bounds__(MP_THREADS) mode_product_kernel(const cf* __restrict__ in, cf* __restrict__ out,
                                                                   const cf* __restrict__ U, int M, int K, int C, int r_n) {
   __shared__ __align__(16) cf As[2][MP_BK][MP_BM];
   __shared__ __align__(16) cf Bs[2][MP_BK][MP_BC];
   const int tid = threadIdx.x;
-  const int tm = tid >> 4, tc = tid & 15;          // 8 x 16 threads: 4 rows (m) x 4 cols (c) each
+  constexpr int NC = MP_BC / 16;                   // columns per thread
+  const int tm = tid >> 4, tc = tid & 15;          // 8 x 16 threads: 4 rows (m) x NC cols (c) each
   const int m0 = blockIdx.y * MP_BM, c0 = blockIdx.x * MP_BC;
   const size_t o = blockIdx.z;
   const cf* inb = in + o * (size_t)K * C;
   constexpr int A_PER = MP_BK * MP_BM / MP_THREADS;   // 4
-  constexpr int B_PER = MP_BK * MP_BC / MP_THREADS;   // 8
+  constexpr int B_PER = MP_BK * MP_BC / MP_THREADS;   // 8 or 4
   cf ra[A_PER], rb[B_PER];
 
   auto fetch = [&](int k0) {
@@ -74,11 +77,11 @@ __global__ void __launch_bounds__(MP_THREADS) mode_product_kernel(const cf* __re
     }
   };
 
-  cf acc[4][4];
+  cf acc[4][NC];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = make_float2(0.f, 0.f);
+    for (int j = 0; j < NC; ++j) acc[i][j] = make_float2(0.f, 0.f);
 
   fetch(0);
   stash(0);
@@ -89,13 +92,13 @@ __global__ void __launch_bounds__(MP_THREADS) mode_product_kernel(const cf* __re
     if (more) fetch(k0 + MP_BK);
 #pragma unroll
     for (int kk = 0; kk < MP_BK; ++kk) {
-      cf a[4], b[4];
+      cf a[4], b[NC];
       load_row_bcast<4>(&As[buf][kk][tm * 4], a);
-      load_row_bcast<4>(&Bs[buf][kk][tc * 4], b);
+      load_row_bcast<NC>(&Bs[buf][kk][tc * NC], b);
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) cfma(acc[i][j], a[i], b[j]);
+        for (int j = 0; j < NC; ++j) cfma(acc[i][j], a[i], b[j]);
     }
     if (more) stash(buf ^ 1);
     __syncthreads();
@@ -107,8 +110,8 @@ __global__ void __launch_bounds__(MP_THREADS) mode_product_kernel(const cf* __re
     const int m = m0 + tm * 4 + i;
     if (m >= M) continue;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int c = c0 + tc * 4 + j;
+    for (int j = 0; j < NC; ++j) {
+      const int c = c0 + tc * NC + j;
       if (c < C) outb[(size_t)m * C + c] = acc[i][j];
     }
   }
@@ -129,6 +132,219 @@ __global__ void adam_kernel(const cf* __restrict__ core, cf* __restrict__ m_l, f
     cf m = m_s[i]; float v = v_s[i];
     cf r = adam_apply(g_s[i], m, v, a);
     m_s[i] = m; v_s[i] = v; n_s[i] = r;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same product on the tensor cores, split-precision TF32 (hi*hi + lo*hi + hi*lo, fp32
+// accumulation).  Real formulation with the rows of the output doubled instead of its columns:
+//   [out_re; out_im][m][c] = [[Ar, -Ai], [Ai, Ar]][m][k] . [Xr; Xi][k][c]
+// so that one 8-byte load of the complex entry X[k][c] is a whole B fragment (k = t <-> (k, re),
+// k = t+4 <-> (k, im), n = g <-> c) and one complex entry of Aop a whole A fragment
+// (rows g <-> (m, re), g+8 <-> (m, im)).  One MMA = 8 m x 8 c x 4 k complex.
+// A block of 4 warps owns 32 (m) x 32 NT (c); a warp 32 x 8 NT.  X tiles arrive by 8-byte
+// asynchronous copies, double buffered; the Aop tile is stored already split.
+// ---------------------------------------------------------------------------------------------
+constexpr int MT_BM = 32, MT_BK = 16, MT_THREADS = 128;
+constexpr int MT_LDA = 20;                       // float4 per row of the A tile: conflict-free fragment loads
+
+__device__ __forceinline__ void mt_split(float x, float& hi, float& lo) {
+  hi = __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xffffe000u);
+  lo = x - hi;
+}
+
+template <bool CONJ_T, int NT>
+__global__ void __launch_bounds__(MT_THREADS) mode_product_tc_kernel(const cf* __restrict__ in, cf* __restrict__ out,
+                                                                     const cf* __restrict__ U, int M, int K, int C, int r_n) {
+  constexpr int BC = 32 * NT, LDX = BC + 4;      // X tile row length: rows 4 slots apart in the 16 bank pairs
+  __shared__ __align__(16) float4 As[2][MT_BM][MT_LDA];   // (re.hi, im.hi, re.lo, im.lo) of Aop[m][k]
+  __shared__ __align__(16) cf Xs[2][MT_BK][LDX];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t = lane & 3;
+  const int m0 = blockIdx.y * MT_BM, c0 = blockIdx.x * BC;
+  const size_t o = blockIdx.z;
+  const cf* inb = in + o * (size_t)K * C;
+  const unsigned char* inbytes = reinterpret_cast<const unsigned char*>(inb);
+
+  cf ra[MT_BK * MT_BM / MT_THREADS];
+  auto fetch_a = [&](int k0) {
+#pragma unroll
+    for (int i = 0; i < MT_BK * MT_BM / MT_THREADS; ++i) {
+      const int idx = tid + i * MT_THREADS;
+      int kk, mm;
+      if (CONJ_T) { mm = idx % MT_BM; kk = idx / MT_BM; } else { kk = idx % MT_BK; mm = idx / MT_BK; }
+      const int m = m0 + mm, k = k0 + kk;
+      cf v = make_float2(0.f, 0.f);
+      if (m < M && k < K) {
+        if (CONJ_T) { cf u = U[(size_t)k * r_n + m]; v = make_float2(u.x, -u.y); }
+        else v = U[(size_t)m * r_n + k];
+      }
+      ra[i] = v;
+    }
+  };
+  auto stash_a = [&](int buf) {
+#pragma unroll
+    for (int i = 0; i < MT_BK * MT_BM / MT_THREADS; ++i) {
+      const int idx = tid + i * MT_THREADS;
+      int kk, mm;
+      if (CONJ_T) { mm = idx % MT_BM; kk = idx / MT_BM; } else { kk = idx % MT_BK; mm = idx / MT_BK; }
+      float4 q;
+      mt_split(ra[i].x, q.x, q.z); mt_split(ra[i].y, q.y, q.w);
+      As[buf][mm][kk] = q;
+    }
+  };
+  auto load_x = [&](int k0, int buf) {
+#pragma unroll
+    for (int i = 0; i < MT_BK * BC / MT_THREADS; ++i) {
+      const int idx = tid + i * MT_THREADS;
+      const int cc = idx % BC, kk = idx / BC;
+      const int c = c0 + cc, k = k0 + kk;
+      const bool v = c < C && k < K;
+      cp_async8(&Xs[buf][kk][cc], v ? inbytes + ((size_t)k * C + c) * 8 : inbytes, v ? 8u : 0u);
+    }
+    cp_async_commit();
+  };
+
+  // a warp covers all 4 m-tiles (32 rows = 4 x 8 complex m) and NT column tiles: accumulators [4][NT][4]
+  float d[4][NT][4];
+#pragma unroll
+  for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) d[mt][nt][i] = 0.f;
+
+  fetch_a(0);
+  load_x(0, 0);
+  stash_a(0);
+  int buf = 0;
+  for (int k0 = 0; k0 < K; k0 += MT_BK, buf ^= 1) {
+    cp_async_wait<0>();
+    __syncthreads();                               // stage buf is complete; everyone is done with stage buf^1
+    const bool more = k0 + MT_BK < K;
+    if (more) { fetch_a(k0 + MT_BK); load_x(k0 + MT_BK, buf ^ 1); }
+#pragma unroll
+    for (int ks = 0; ks < MT_BK / 4; ++ks) {
+      const int kc = ks * 4 + t;
+      float xh[NT][2], xl[NT][2];
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const cf x = Xs[buf][kc][warp * 8 * NT + nt * 8 + gq];
+        mt_split(x.x, xh[nt][0], xl[nt][0]); mt_split(x.y, xh[nt][1], xl[nt][1]);
+      }
+#pragma unroll
+      for (int mt = 0; mt < 4; ++mt) {
+        const float4 a = As[buf][mt * 8 + gq][kc];
+        // rows (m, re): (Ar | -Ai); rows (m, im): (Ai | Ar)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          mma_tf32(d[mt][nt], a.x, a.y, -a.y, a.x, xh[nt][0], xh[nt][1]);
+          mma_tf32(d[mt][nt], a.z, a.w, -a.w, a.z, xh[nt][0], xh[nt][1]);
+          mma_tf32(d[mt][nt], a.x, a.y, -a.y, a.x, xl[nt][0], xl[nt][1]);
+        }
+      }
+    }
+    if (more) stash_a(buf ^ 1);
+  }
+  // d0 = re(m, c = 2t), d1 = re(m, 2t+1), d2 = im(m, 2t), d3 = im(m, 2t+1)
+  cf* outb = out + o * (size_t)M * C;
+#pragma unroll
+  for (int mt = 0; mt < 4; ++mt) {
+    const int m = m0 + mt * 8 + gq;
+    if (m >= M) continue;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const int c = c0 + warp * 8 * NT + nt * 8 + 2 * t;
+      if (c < C) outb[(size_t)m * C + c] = make_float2(d[mt][nt][0], d[mt][nt][2]);
+      if (c + 1 < C) outb[(size_t)m * C + c + 1] = make_float2(d[mt][nt][1], d[mt][nt][3]);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The innermost link of the chain in one launch: last compression product, AdamUpdate of the
+// core, first reconstruction product (all three act on columns c of [.][C] independently):
+//   core[j][c] = sum_i conj(U1[i][j]) X[i][c]        (mode-1 product with U^(1)H, I_1 -> r_1)
+//   N = AdamUpdate(core)                             (moments in place; core and N_L are kept)
+//   out[i][c] = sum_j U1[i][j] N[j][c]               (mode-1 product with U^(1), r_1 -> I_1)
+// A block takes 16 columns: X[:, block] is read into shared memory before anything is written, so
+// `out` may alias `X`.  Blocks past the last column block run the AdamUpdate of the sparse values.  The work is small (two skinny products); what this saves is two launches,
+// two round trips of the core through L2 and the idle SMs of three under-filled grids.
+// ---------------------------------------------------------------------------------------------
+constexpr int SW_CB = 16, SW_THREADS = 256, SW_MAX_I = 256, SW_MAX_R = 64;
+__host__ __device__ inline size_t sandwich_smem(int I1, int r1) {
+  return ((size_t)I1 * (SW_CB + 1) + (size_t)r1 * (SW_CB + 1) + (size_t)I1 * r1) * sizeof(cf);
+}
+
+__global__ void __launch_bounds__(SW_THREADS) core_sandwich_kernel(const cf* __restrict__ X, cf* __restrict__ out,
+                                                                   const cf* __restrict__ U1, cf* __restrict__ core,
+                                                                   cf* __restrict__ m_l, float* __restrict__ v_l,
+                                                                   cf* __restrict__ n_l, int I1, int r1, int C,
+                                                                   const cf* __restrict__ g_s, cf* __restrict__ m_s,
+                                                                   float* __restrict__ v_s, cf* __restrict__ n_s, uint32_t ks,
+                                                                   uint32_t nblk_core, AdamScalars a) {
+  extern __shared__ __align__(16) unsigned char swm[];
+  if (blockIdx.x >= nblk_core) {
+    // trailing blocks: AdamUpdate of the ks gathered sparse values (independent of the core)
+    const uint32_t i = (blockIdx.x - nblk_core) * SW_THREADS + threadIdx.x;
+    if (i < ks) {
+      cf m = m_s[i]; float v = v_s[i];
+      cf r = adam_apply(g_s[i], m, v, a);
+      m_s[i] = m; v_s[i] = v; n_s[i] = r;
+    }
+    return;
+  }
+  constexpr int LD = SW_CB + 1, RP = SW_THREADS / SW_CB;                  // padded row, rows per pass
+  cf* Xs = reinterpret_cast<cf*>(swm);                                    // [I1][LD]
+  cf* Ns = Xs + (size_t)I1 * LD;                                          // [r1][LD]
+  cf* Us = Ns + (size_t)r1 * LD;                                          // [I1][r1]
+  const int tid = threadIdx.x, cc = tid % SW_CB, r0 = tid / SW_CB;
+  const int c = blockIdx.x * SW_CB + cc;
+  const bool cok = c < C;
+  for (int i = r0; i < I1; i += RP) Xs[i * LD + cc] = cok ? X[(size_t)i * C + c] : make_float2(0.f, 0.f);
+  for (int i = tid; i < I1 * r1; i += SW_THREADS) Us[i] = U1[i];
+  __syncthreads();
+  // core rows j and j + RP together: one load of x serves both
+  for (int j = r0; j < r1; j += 2 * RP) {
+    const bool two = j + RP < r1;
+    const int j2 = two ? j + RP : j;
+    cf acc0 = make_float2(0.f, 0.f), acc1 = acc0;
+#pragma unroll 4
+    for (int i = 0; i < I1; ++i) {
+      const cf x = Xs[i * LD + cc];
+      cfma_conj(acc0, x, Us[i * r1 + j]);                                 // x * conj(u)
+      cfma_conj(acc1, x, Us[i * r1 + j2]);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if (h == 1 && !two) break;
+      const int jj = h ? j2 : j;
+      const cf acc = h ? acc1 : acc0;
+      cf n = make_float2(0.f, 0.f);
+      if (cok) {
+        const size_t e = (size_t)jj * C + c;
+        cf m = m_l[e]; float v = v_l[e];
+        n = adam_apply(acc, m, v, a);
+        m_l[e] = m; v_l[e] = v; n_l[e] = n; core[e] = acc;
+      }
+      Ns[jj * LD + cc] = n;
+    }
+  }
+  __syncthreads();
+  // four output rows at a time: one load of N[j][c] serves them
+  for (int i = r0; i < I1; i += 4 * RP) {
+    cf acc[4];
+    int ii[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { acc[q] = make_float2(0.f, 0.f); ii[q] = (i + q * RP < I1) ? i + q * RP : i; }
+#pragma unroll 4
+    for (int j = 0; j < r1; ++j) {
+      const cf nv = Ns[j * LD + cc];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) cfma(acc[q], Us[ii[q] * r1 + j], nv);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (cok && i + q * RP < I1) out[(size_t)(i + q * RP) * C + c] = acc[q];
   }
 }
 

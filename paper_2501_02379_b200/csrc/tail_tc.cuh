@@ -104,14 +104,15 @@ __device__ __forceinline__ void tc_issue_load(const unsigned char* gbase, unsign
 // shared memory, in warp order, one iteration later (so that one block-wide barrier per iteration suffices).
 // RAT = ceil(ra/8); KS = k-steps of stage 1 (>= tc_ksteps(B)).
 // ---------------------------------------------------------------------------------------------
-constexpr int PJ_WARPS = 4;
-constexpr int PJ_THREADS = 32 * PJ_WARPS;
 
-__host__ inline bool proj_tc_geom(int A, int B, int rat, uint32_t nslab, int ntw, uint32_t smem_per_block, TcGeom& g) {
+__host__ inline bool proj_tc_geom(int A, int B, int rat, uint32_t nslab, int ntw, int PJ_WARPS, uint32_t smem_per_block, TcGeom& g) {
   if (A % 8) return false;
   const int tiles = A / 8;
-  if (tiles >= PJ_WARPS) { if (tiles != ntw * PJ_WARPS) return false; g.tps = PJ_WARPS; g.spi = 1; }
-  else { if (ntw != 1 || PJ_WARPS % tiles) return false; g.tps = tiles; g.spi = PJ_WARPS / tiles; }
+  // tps = warps per slab, each with ntw row tiles; spi = slabs per group
+  if (tiles % ntw) return false;
+  g.tps = tiles / ntw;
+  if (g.tps > PJ_WARPS || PJ_WARPS % g.tps) return false;
+  g.spi = PJ_WARPS / g.tps;
   g.nbt = tc_ksteps(B);
   g.slab_bytes = (uint32_t)A * B * 8;
   g.grp_stride = ((uint32_t)g.spi * g.slab_bytes + 127) & ~127u;
@@ -128,9 +129,10 @@ __host__ inline bool proj_tc_geom(int A, int B, int rat, uint32_t nslab, int ntw
   return true;
 }
 
-template <int RAT, int KS, int NTW>
-__global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_kernel(const void* __restrict__ g, TailTcParams P) {
+template <int RAT, int KS, int NTW, int PJ_WARPS>
+__global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW == 1 ? 4 : 3)) proj_tail_tc_kernel(const void* __restrict__ g, TailTcParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
+  constexpr int PJ_THREADS = 32 * PJ_WARPS;
   const TailParams& p = P.p;
   const TcGeom& G = P.g;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t = lane & 3;
@@ -192,16 +194,23 @@ __global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_ker
     uint32_t u = blockIdx.x;
     for (int i = 0; i < nbuf && u < ngroups; ++i, u += gstride) tc_issue_load(gb, smem, G, bars, u, i, nslab);
   }
-  // ---- sparse side, software-pipelined: the next group's entry bounds and first entries are fetched one group ahead ----
+  // ---- sparse side, software-pipelined: a group's entry bounds are fetched three groups ahead, its first
+  //      entries (one per thread) two groups ahead, so that neither load is waited for ----
   const bool sparse = p.k > 0;
-  int b0 = 0, b1 = 0;
-  uint32_t pom = 0;
+  auto bounds = [&](uint32_t ug, int& x0, int& x1) {
+    x0 = 0; x1 = 0;
+    if (ug < ngroups) {
+      uint32_t e = (ug + 1) * spi; if (e > nslab) e = nslab;
+      x0 = (int)p.slab_ptr[ug * spi]; x1 = (int)p.slab_ptr[e];
+    }
+  };
+  int b0 = 0, b1 = 0, c0 = 0, c1 = 0;
+  uint32_t pom = 0, pomc = 0;
   if (sparse) {
-    const uint32_t u = blockIdx.x;
-    uint32_t e = (u + 1) * spi; if (e > nslab) e = nslab;
-    b0 = (int)p.slab_ptr[u * spi]; b1 = (int)p.slab_ptr[e];
-    const int j = b0 + tid;
-    if (j < b1) pom = p.omega[j];
+    bounds(blockIdx.x, b0, b1);
+    bounds(blockIdx.x + gstride, c0, c1);
+    if (b0 + tid < b1) pom = p.omega[b0 + tid];
+    if (c0 + tid < c1) pomc = p.omega[c0 + tid];
   }
 
   // sums the partials of iteration `itp` (group up) in warp order and writes T
@@ -231,13 +240,9 @@ __global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_ker
   uint32_t it = 0, phase = 0;
   int buf = 0, pbuf = 0;      // ring slot of this iteration and of the previous one
   for (uint32_t u = blockIdx.x; u < ngroups; u += gstride, ++it) {
-    // bounds of the next group's entries: issued now, used at the end of this iteration
+    // entry bounds of the group after next: issued now, used at the end of this iteration
     int n0 = 0, n1 = 0;
-    if (sparse && u + gstride < ngroups) {
-      const uint32_t un = u + gstride;
-      uint32_t e = (un + 1) * spi; if (e > nslab) e = nslab;
-      n0 = (int)p.slab_ptr[un * spi]; n1 = (int)p.slab_ptr[e];
-    }
+    if (sparse) bounds(u + 2 * gstride, n0, n1);
     const bool ok = mbar_wait_bounded(&bars[buf], phase);
     float* xg = reinterpret_cast<float*>(smem + (size_t)buf * G.grp_stride);
     // ---- sparse part, before the barrier: gather and zero (the residual); one entry of the group per thread ----
@@ -337,9 +342,9 @@ __global__ void __launch_bounds__(PJ_THREADS, NTW == 1 ? 4 : 3) proj_tail_tc_ker
     // ---- off the critical path: the previous group's T, the next group's entries ----
     if (it > 0) reduce_out(u - gstride, it - 1);
     if (sparse) {
-      b0 = n0; b1 = n1;
-      const int j = b0 + tid;
-      if (j < b1) pom = p.omega[j];
+      b0 = c0; b1 = c1; pom = pomc;
+      c0 = n0; c1 = n1;
+      if (c0 + tid < c1) pomc = p.omega[c0 + tid];
     }
     pbuf = buf;
     if (++buf == nbuf) { buf = 0; phase ^= 1; }

@@ -47,7 +47,7 @@ struct TailPlan {
   size_t smem_proj, smem_back;
   // tensor-core fast path (complex64 storage, 16/32/64 slab rows, small trailing ranks)
   bool tc;
-  int rat, ks, ntw;
+  int rat, ks, ntw, pjw;
   TcGeom gproj, gback;
   int grid_proj, grid_back;
 };
@@ -205,19 +205,20 @@ tgrad_status tail_any(const tgrad_state* s, int op, void* ptr, const TailParams&
                                       : tail_dispatch<StoreC32H>(op, s->tail, ptr, p, st);
 }
 
-template <int RAT, int KS, int NTW>
+template <int RAT, int KS, int NTW, int W>
 tgrad_status tc_proj_op2(int op, const TailPlan& tp, const void* g, const TailTcParams& P, cudaStream_t st) {
   if (op == 0) {
-    return cudaFuncSetAttribute(proj_tail_tc_kernel<RAT, KS, NTW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(proj_tail_tc_kernel<RAT, KS, NTW, W>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)tp.gproj.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
   }
-  proj_tail_tc_kernel<RAT, KS, NTW><<<tp.grid_proj, PJ_THREADS, tp.gproj.total, st>>>(g, P);
+  proj_tail_tc_kernel<RAT, KS, NTW, W><<<tp.grid_proj, 32 * W, tp.gproj.total, st>>>(g, P);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
 template <int RAT, int KS>
 tgrad_status tc_proj_op(int op, const TailPlan& tp, const void* g, const TailTcParams& P, cudaStream_t st) {
-  return tp.ntw == 2 ? tc_proj_op2<RAT, KS, 2>(op, tp, g, P, st) : tc_proj_op2<RAT, KS, 1>(op, tp, g, P, st);
+  if (tp.pjw == 8) return tc_proj_op2<RAT, KS, 1, 8>(op, tp, g, P, st);
+  return tp.ntw == 2 ? tc_proj_op2<RAT, KS, 2, 4>(op, tp, g, P, st) : tc_proj_op2<RAT, KS, 1, 4>(op, tp, g, P, st);
 }
 template <int RAT>
 tgrad_status tc_back_op(int op, const TailPlan& tp, void* w, const TailTcParams& P, cudaStream_t st) {
@@ -289,10 +290,13 @@ tgrad_status plan_tail(tgrad_state* s) {
   const int ks = ksn <= 4 ? 4 : ksn == 5 ? 5 : ksn <= 8 ? 8 : ksn == 9 ? 9 : 0;
   const double dec = 1.0 - (double)c.lr * (double)c.weight_decay;
   if (c.wg_dtype == TGRAD_C64 && (A == 16 || A == 32 || A == 64) && rat <= 2 && rb <= 8 && ks && dec > 0.0) {
-    tp.rat = rat; tp.ks = ks; tp.ntw = (A == 64) ? 2 : 1;
-    const int pj_blocks = tp.ntw == 2 ? 3 : 4;                       // resident blocks per SM of the compression kernel
+    tp.rat = rat; tp.ks = ks;
+    // compression kernel: blocks of 4 warps; two row tiles per warp for 64-row slabs (measured faster than
+    // 8 warps with one tile each: 101 against 122 us on 128x128x64x33)
+    tp.pjw = 4; tp.ntw = (A == 64) ? 2 : 1;
+    const int pj_blocks = tp.pjw == 8 ? 2 : (tp.ntw == 2 ? 3 : 4);     // resident blocks per SM
     const uint32_t pj_smem = (227u * 1024u) / pj_blocks - 1024u;
-    if (proj_tc_geom(A, B, rat, (uint32_t)S, tp.ntw, pj_smem, tp.gproj) && tail_tc_geom(true, A, B, rat, (uint32_t)S, tp.gback)) {
+    if (proj_tc_geom(A, B, rat, (uint32_t)S, tp.ntw, tp.pjw, pj_smem, tp.gproj) && tail_tc_geom(true, A, B, rat, (uint32_t)S, tp.gback)) {
       const uint32_t cap = 2u * (uint32_t)s->sm_count, pcap = (uint32_t)pj_blocks * (uint32_t)s->sm_count;
       tp.grid_proj = (int)(tp.gproj.ngroups < pcap ? tp.gproj.ngroups : pcap);
       tp.grid_back = (int)(tp.gback.ngroups < cap ? tp.gback.ngroups : cap);
@@ -422,10 +426,18 @@ tgrad_status do_refresh(tgrad_state* s, void* d_grad, cudaStream_t st) {
 }
 
 tgrad_status mode_product(bool conj_t, const cf* in, cf* out, const cf* U, uint64_t O, int M, int K, uint64_t C,
-                          int r_n, cudaStream_t st) {
-  dim3 grid((unsigned)((C + MP_BC - 1) / MP_BC), (unsigned)((M + MP_BM - 1) / MP_BM), (unsigned)O);
-  if (conj_t) mode_product_kernel<true><<<grid, MP_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
-  else mode_product_kernel<false><<<grid, MP_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
+                          int r_n, int sm_count, cudaStream_t st) {
+  // narrow column tiles when the wide ones would leave SMs without a block or two
+  const uint64_t wide = ((C + 63) / 64) * ((M + MT_BM - 1) / MT_BM) * O;
+  const int bc = (wide < (uint64_t)4 * sm_count) ? 32 : 64;
+  dim3 grid((unsigned)((C + bc - 1) / bc), (unsigned)((M + MT_BM - 1) / MT_BM), (unsigned)O);
+  if (bc == 64) {
+    if (conj_t) mode_product_tc_kernel<true, 2><<<grid, MT_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
+    else mode_product_tc_kernel<false, 2><<<grid, MT_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
+  } else {
+    if (conj_t) mode_product_tc_kernel<true, 1><<<grid, MT_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
+    else mode_product_tc_kernel<false, 1><<<grid, MT_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
+  }
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
@@ -476,45 +488,57 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
     TG_TRY(tail_any(s, 1, d_grad, p, st));
   }
   TG_MARK(1);
+  // the chain on the small tensor: compression of modes N-2 .. 2, then mode 1 + Adam + mode 1 in one
+  // launch (or three when the first mode is too large for it), then reconstruction of modes 2 .. N-2
+  const bool fused = c.dims[0] <= SW_MAX_I && c.ranks[0] <= SW_MAX_R;
+  const cf* tprime;
   {
     cf* cur = bufa; cf* nxt = bufb;
     uint64_t C = (uint64_t)ra * rb;
-    for (int m = N - 3; m >= 0; --m) {
+    for (int m = N - 3; m >= (fused ? 1 : 0); --m) {
       uint64_t O = 1;
       for (int q = 0; q < m; ++q) O *= c.dims[q];
       cf* dst = (m == 0) ? core : nxt;
       TG_TRY(mode_product(true, cur, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[m]), O, c.ranks[m],
-                          (int)c.dims[m], C, c.ranks[m], st));
+                          (int)c.dims[m], C, c.ranks[m], s->sm_count, st));
       C *= c.ranks[m];
       cf* tmp = cur; cur = nxt; nxt = tmp;
     }
-  }
-  TG_MARK(2);
-  {
-    const uint32_t ks = s->tail.tc ? (uint32_t)c.k : 0u;      // the general streaming kernel updates the sparse moments itself
-    adam_kernel<<<(unsigned)((L.P + ks + 255) / 256), 256, 0, st>>>(
-        core, reinterpret_cast<cf*>(s->dp + L.p_ml), reinterpret_cast<float*>(s->dp + L.p_vl), n_l, (uint32_t)L.P,
-        p.g_s, p.m_s, p.v_s, p.n_s, ks, p.adam);
-    TG_LAUNCH_CHECK();
-  }
-  TG_MARK(3);
-  // reconstruction: modes 1 .. N-2 on the small tensor, trailing two while streaming W
-  const cf* tprime;
-  {
-    const cf* cur = n_l;
+    TG_MARK(2);
     cf* bufs[2] = {bufa, bufb};
     int which = ((N - 2) & 1) ? 0 : 1;          // make the last product land in bufa
-    uint64_t O = 1;
-    for (int m = 0; m <= N - 3; ++m) {
-      uint64_t C = (uint64_t)ra * rb;
-      for (int q = m + 1; q <= N - 3; ++q) C *= c.ranks[q];
+    const uint32_t ks = s->tail.tc ? (uint32_t)c.k : 0u;      // the general streaming kernel updates the sparse moments itself
+    const cf* src;
+    int mfirst;
+    if (fused) {
+      // here cur holds [I_1][C] with C = r_2 .. r_N
       cf* dst = bufs[which];
-      TG_TRY(mode_product(false, cur, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[m]), O, (int)c.dims[m],
-                          c.ranks[m], C, c.ranks[m], st));
-      O *= c.dims[m];
-      cur = dst; which ^= 1;
+      const uint32_t nblk_core = (uint32_t)((C + SW_CB - 1) / SW_CB), nblk_sparse = (ks + SW_THREADS - 1) / SW_THREADS;
+      core_sandwich_kernel<<<nblk_core + nblk_sparse, SW_THREADS, sandwich_smem((int)c.dims[0], c.ranks[0]), st>>>(
+          cur, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[0]), core, reinterpret_cast<cf*>(s->dp + L.p_ml),
+          reinterpret_cast<float*>(s->dp + L.p_vl), n_l, (int)c.dims[0], c.ranks[0], (int)C, p.g_s, p.m_s, p.v_s, p.n_s, ks,
+          nblk_core, p.adam);
+      TG_LAUNCH_CHECK();
+      src = dst; which ^= 1; mfirst = 1;
+    } else {
+      adam_kernel<<<(unsigned)((L.P + ks + 255) / 256), 256, 0, st>>>(
+          core, reinterpret_cast<cf*>(s->dp + L.p_ml), reinterpret_cast<float*>(s->dp + L.p_vl), n_l, (uint32_t)L.P,
+          p.g_s, p.m_s, p.v_s, p.n_s, ks, p.adam);
+      TG_LAUNCH_CHECK();
+      src = n_l; mfirst = 0;
     }
-    tprime = cur;
+    TG_MARK(3);
+    uint64_t O = fused ? (uint64_t)c.dims[0] : 1;
+    for (int m = mfirst; m <= N - 3; ++m) {
+      uint64_t Cm = (uint64_t)ra * rb;
+      for (int q = m + 1; q <= N - 3; ++q) Cm *= c.ranks[q];
+      cf* dst = bufs[which];
+      TG_TRY(mode_product(false, src, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[m]), O, (int)c.dims[m],
+                          c.ranks[m], Cm, c.ranks[m], s->sm_count, st));
+      O *= c.dims[m];
+      src = dst; which ^= 1;
+    }
+    tprime = src;
   }
   TG_MARK(4);
   p.t = const_cast<cf*>(tprime);
@@ -576,6 +600,9 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
     cudaError_t e4 = cudaFuncSetAttribute(gram_partial_kernel<StoreC32H, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GR_SMEM);
     if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
   }
+  if (cfg->dims[0] <= SW_MAX_I && cfg->ranks[0] <= SW_MAX_R &&
+      cudaFuncSetAttribute(core_sandwich_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)sandwich_smem(SW_MAX_I, SW_MAX_R)) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
   if (cudaFuncSetAttribute(jacobi_sweeps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)jac_sweeps_smem(JAC_SMEM_MAX_N)) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
