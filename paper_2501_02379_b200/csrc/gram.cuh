@@ -31,7 +31,7 @@ __device__ __forceinline__ float gr_tf32(float x) { return __uint_as_float((__fl
 constexpr size_t GR_SMEM = 2 * 2 * GR_T * GR_LD * sizeof(cf);      // two stages of (Xa, Xb)
 
 template <class S, bool SPLIT>
-__global__ void __launch_bounds__(GR_THREADS) gram_partial_kernel(const void* __restrict__ g, int In, uint32_t O, uint32_t C,
+__global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void* __restrict__ g, int In, uint32_t O, uint32_t C,
                                                                   uint32_t chunks_total, uint32_t chunks_per_split,
                                                                   cf* __restrict__ partial) {
   const int T = (In + GR_T - 1) / GR_T;
@@ -61,6 +61,16 @@ __global__ void __launch_bounds__(GR_THREADS) gram_partial_kernel(const void* __
     for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
       for (int i = 0; i < 4; ++i) { are[mt][nt][i] = 0.f; aim[mt][nt][i] = 0.f; }
+  // The tensor core adds into its fp32 accumulator with truncation, which biases a long chain of
+  // accumulations; so the MMA accumulators are emptied every other chunk (16 MMAs deep) into
+  // running sums kept with ordinary round-to-nearest adds.
+  float tre[2][4][4], tim[2][4][4];
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { tre[mt][nt][i] = 0.f; tim[mt][nt][i] = 0.f; }
   // loader mapping (fixed per thread): lanes along k when rows are runs of k -- a thread keeps one k of
   // the chunk and walks 16 rows; along the rows when C == 1 -- it keeps one row and walks 16 k
   const bool along_k = C > 1;
@@ -148,6 +158,17 @@ __global__ void __launch_bounds__(GR_THREADS) gram_partial_kernel(const void* __
         }
       }
     }
+    if (((ch - ch0) & 1) || ch + 1 == ch1) {
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            tre[mt][nt][i] += are[mt][nt][i]; are[mt][nt][i] = 0.f;
+            tim[mt][nt][i] += aim[mt][nt][i]; aim[mt][nt][i] = 0.f;
+          }
+    }
   }
   // accumulator (row g | g+8, col 2t | 2t+1) -> partial[split][a][b]
   cf* out = partial + (size_t)blockIdx.y * In * In;
@@ -158,7 +179,7 @@ __global__ void __launch_bounds__(GR_THREADS) gram_partial_kernel(const void* __
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int a = a0 + wm * 32 + mt * 16 + gq + (i >> 1) * 8, b = b0 + wn * 32 + nt * 8 + 2 * t + (i & 1);
-        if (a < In && b < In) out[(size_t)a * In + b] = make_float2(are[mt][nt][i], aim[mt][nt][i]);
+        if (a < In && b < In) out[(size_t)a * In + b] = make_float2(tre[mt][nt][i], tim[mt][nt][i]);
       }
 }
 
