@@ -212,6 +212,15 @@ __global__ void __launch_bounds__(MT_THREADS) mode_product_tc_kernel(const cf* _
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
       for (int i = 0; i < 4; ++i) d[mt][nt][i] = 0.f;
+  // running sums with round-to-nearest adds; the MMA accumulators (whose adds truncate) are emptied into
+  // them after every k-slice of 16, i.e. after at most 12 accumulations
+  float tot[4][NT][4];
+#pragma unroll
+  for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) tot[mt][nt][i] = 0.f;
 
   fetch_a(0);
   load_x(0, 0);
@@ -244,6 +253,12 @@ __global__ void __launch_bounds__(MT_THREADS) mode_product_tc_kernel(const cf* _
       }
     }
     if (more) stash_a(buf ^ 1);
+#pragma unroll
+    for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { tot[mt][nt][i] += d[mt][nt][i]; d[mt][nt][i] = 0.f; }
   }
   // d0 = re(m, c = 2t), d1 = re(m, 2t+1), d2 = im(m, 2t), d3 = im(m, 2t+1)
   cf* outb = out + o * (size_t)M * C;
@@ -254,8 +269,8 @@ __global__ void __launch_bounds__(MT_THREADS) mode_product_tc_kernel(const cf* _
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       const int c = c0 + warp * 8 * NT + nt * 8 + 2 * t;
-      if (c < C) outb[(size_t)m * C + c] = make_float2(d[mt][nt][0], d[mt][nt][2]);
-      if (c + 1 < C) outb[(size_t)m * C + c + 1] = make_float2(d[mt][nt][1], d[mt][nt][3]);
+      if (c < C) outb[(size_t)m * C + c] = make_float2(tot[mt][nt][0], tot[mt][nt][2]);
+      if (c + 1 < C) outb[(size_t)m * C + c + 1] = make_float2(tot[mt][nt][1], tot[mt][nt][3]);
     }
   }
 }
