@@ -86,6 +86,15 @@ WORKLOADS: Dict[str, Workload] = {
                  outlier_frac=(1, 100), outlier_scale=20.0, noise="laplace", noise_scale=0.1),
         Workload("ragged4", 93, (20, 12, 24, 13), (5, 4, 6, 4), (1, 40), 4, 9,
                  outlier_frac=(1, 200), outlier_scale=30.0, noise_scale=0.03),
+        # shapes that reach the tensor-core streaming kernels in their corner cases: a 3-way tensor (no
+        # mode product outside the fused first-mode launch) and a slab count that leaves the last group of
+        # slabs partly empty
+        Workload("small3", 94, (12, 16, 9), (4, 4, 3), (1, 40), 3, 7,
+                 outlier_frac=(1, 200), outlier_scale=25.0, noise_scale=0.02),
+        Workload("odd4", 95, (7, 9, 16, 9), (3, 4, 4, 3), (1, 50), 3, 7,
+                 outlier_frac=(1, 100), outlier_scale=20.0, noise="laplace", noise_scale=0.05),
+        Workload("odd32", 96, (5, 7, 32, 17), (3, 3, 8, 5), (1, 25), 3, 5,
+                 outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.05),
         # the five benchmark configurations
         Workload("cfg1", 1, (32, 32, 16, 9), (8, 8, 4, 3), (1, 100), 5, 20,
                  outliers_equal_k=True, outlier_scale=20.0, noise_scale=0.01, lr=1e-3),
