@@ -208,10 +208,12 @@ int64_t tgrad_launch_count(void);
 
 /* Optional per-stage device timing of tgrad_step (CUDA events recorded on the
  * caller's stream between the stages of a non-refresh step).  Stages, in
- * order: 0 trailing-mode compression fused with the sparse gather/Adam
- * (streams grad), 1 remaining mode products of the compression, 2 Adam on the
- * core, 3 leading mode products of the reconstruction, 4 trailing-mode
- * reconstruction fused with the weight update and sparse add (streams W).
+ * order: 0 trailing-mode compression fused with the sparse gather (streams
+ * grad), 1 mode products of the compression except the first mode, 2 first-mode
+ * compression + Adam on the core and on the sparse values + first-mode
+ * reconstruction, 3 remaining mode products of the reconstruction, 4
+ * trailing-mode reconstruction fused with the weight update and sparse add
+ * (streams W).
  * tgrad_get_stage_times synchronises the stream and returns, for the steps
  * since the last call (at most the 64 most recent), the summed milliseconds
  * per stage in ms_sum[5] and the number of steps in *n_steps. */
