@@ -52,12 +52,12 @@ __host__ __device__ inline int tc_ksteps(int B) {
   return 4 * KB + (rem >= 8 ? 4 : rem / 2);
 }
 
-__host__ inline bool tail_tc_geom(bool back, int A, int B, int rat, uint32_t nslab, TcGeom& g) {
+__host__ inline bool tail_tc_geom(bool back, int A, int B, int rat, uint32_t nslab, int ns, TcGeom& g) {
   const int rows = back ? 16 : 8;
   if (A % rows) return false;
   g.tps = A / rows;
   if (g.tps < 1 || g.tps > TC_WARPS || TC_WARPS % g.tps) return false;
-  g.spi = TC_WARPS / g.tps;
+  g.spi = (TC_WARPS / g.tps) * ns;     // ns slabs per warp and iteration (small slabs)
   g.nbt = tc_ksteps(B);
   g.slab_bytes = (uint32_t)A * B * 8;
   g.grp_stride = ((uint32_t)g.spi * g.slab_bytes + 127) & ~127u;
@@ -368,7 +368,7 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW == 1 ?
 // decayed dense update that follows leaves exactly eta*lambda*N_S), then each warp updates its
 // rows in place and stores them with one bulk copy.
 // ---------------------------------------------------------------------------------------------
-template <int RAT>
+template <int RAT, int NS>
 __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __restrict__ w, TailTcParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
   const TailParams& p = P.p;
@@ -442,18 +442,19 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
   const uint32_t row_bytes = 16u * (uint32_t)B * 8u;            // the 16 rows a warp owns
   uint32_t it = 0, phase = 0;
   int buf = 0, lbuf = la % nbuf;      // ring slot of this iteration and of the group loaded `la` ahead
+  const int qstep = TC_WARPS / tps;      // this warp's NS slabs of a group are q, q + qstep, ...
   for (uint32_t u = blockIdx.x; u < ngroups; u += gstride, ++it) {
-    const uint32_t s = u * spi + q;
-    const bool active = s < nslab;
-    if (lane == 0) bulk_wait_read<1>();     // this warp's store of two iterations ago has read its rows
-    // T' fragments for stage 1 (in flight while the slab arrives): T'[ja = 4 ks + t][jb = gq]
-    cf tv[KS2];
-    {
+    if (lane == 0) bulk_wait_read<1>();     // this warp's stores of two iterations ago have read their rows
+    // T' fragments for stage 1 (in flight while the slabs arrive): T'[ja = 4 ks + t][jb = gq]
+    cf tv[NS][KS2];
+#pragma unroll
+    for (int i = 0; i < NS; ++i) {
+      const uint32_t s = u * spi + q + i * qstep;
       const cf* tin = p.t + (size_t)s * ra * rb;
 #pragma unroll
       for (int ks = 0; ks < KS2; ++ks) {
         const int ja = 4 * ks + t;
-        tv[ks] = (active && ja < ra && gq < rb) ? __ldg(tin + (size_t)ja * rb + gq) : make_float2(0.f, 0.f);
+        tv[i][ks] = (s < nslab && ja < ra && gq < rb) ? __ldg(tin + (size_t)ja * rb + gq) : make_float2(0.f, 0.f);
       }
     }
     const bool ok = mbar_wait_bounded(&bars[buf], phase);
@@ -503,8 +504,13 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
       const uint32_t un = u + (uint32_t)la * gstride;
       if (un < ngroups) tc_issue_load(wb, smem, G, bars, un, lbuf, nslab);
     }
+#pragma unroll
+    for (int i = 0; i < NS; ++i) {
+    const int qi = q + i * qstep;
+    const uint32_t s = u * spi + qi;
+    const bool active = s < nslab;
     if (active) {
-      float* ws = wg + (size_t)q * (2 * E);
+      float* ws = wg + (size_t)qi * (2 * E);
       // ---- stage 1: Y'[a][(c, jb)] for rows r0 and r1; hi*hi, lo*hi and hi*lo accumulate separately ----
       float d1[2][3][4];
 #pragma unroll
@@ -516,7 +522,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
 #pragma unroll
       for (int ks = 0; ks < KS2; ++ks) {
         float trh, trl, tih, til;
-        split_tf32(tv[ks].x, trh, trl); split_tf32(tv[ks].y, tih, til);
+        split_tf32(tv[i][ks].x, trh, trl); split_tf32(tv[i][ks].y, tih, til);
         const float* a = ua[ks];
         // A = (Ua[r0].re, Ua[r1].re, Ua[r0].im, Ua[r1].im);  re tile: B = (Tr, -Ti);  im tile: B = (Ti, Tr)
         mma_tf32(d1[0][0], a[0], a[1], a[2], a[3], trh, -tih);
@@ -560,12 +566,11 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
     }
     fence_async_smem();     // order this lane's shared-memory writes before the bulk store reads them
     __syncwarp();
-    if (lane == 0) {
-      if (active)
-        bulk_s2g(wb + ((size_t)s * E + (size_t)am * B) * 8, smem + (size_t)buf * G.grp_stride + (size_t)q * G.slab_bytes +
-                                                                (size_t)am * B * 8, row_bytes);
-      bulk_commit();
+    if (lane == 0 && active)
+      bulk_s2g(wb + ((size_t)s * E + (size_t)am * B) * 8, smem + (size_t)buf * G.grp_stride + (size_t)qi * G.slab_bytes +
+                                                              (size_t)am * B * 8, row_bytes);
     }
+    if (lane == 0) bulk_commit();      // one group per iteration, whatever it holds
     if (++buf == nbuf) { buf = 0; phase ^= 1; }
     if (++lbuf == nbuf) lbuf = 0;
   }

@@ -47,7 +47,7 @@ struct TailPlan {
   size_t smem_proj, smem_back;
   // tensor-core fast path (complex64 storage, 16/32/64 slab rows, small trailing ranks)
   bool tc;
-  int rat, ks, ntw, pjw;
+  int rat, ks, ntw, pjw, back_ns;
   TcGeom gproj, gback;
   int grid_proj, grid_back;
 };
@@ -218,17 +218,22 @@ tgrad_status tc_proj_op2(int op, const TailPlan& tp, const void* g, const TailTc
 template <int RAT, int KS>
 tgrad_status tc_proj_op(int op, const TailPlan& tp, const void* g, const TailTcParams& P, cudaStream_t st) {
   if (tp.pjw == 8) return tc_proj_op2<RAT, KS, 1, 8>(op, tp, g, P, st);
+  if (tp.ntw == 4) return tc_proj_op2<RAT, KS, 4, 4>(op, tp, g, P, st);
   return tp.ntw == 2 ? tc_proj_op2<RAT, KS, 2, 4>(op, tp, g, P, st) : tc_proj_op2<RAT, KS, 1, 4>(op, tp, g, P, st);
+}
+template <int RAT, int NS>
+tgrad_status tc_back_op2(int op, const TailPlan& tp, void* w, const TailTcParams& P, cudaStream_t st) {
+  if (op == 0) {
+    return cudaFuncSetAttribute(back_tail_tc_kernel<RAT, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)tp.gback.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
+  }
+  back_tail_tc_kernel<RAT, NS><<<tp.grid_back, TC_THREADS, tp.gback.total, st>>>(w, P);
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
 }
 template <int RAT>
 tgrad_status tc_back_op(int op, const TailPlan& tp, void* w, const TailTcParams& P, cudaStream_t st) {
-  if (op == 0) {
-    return cudaFuncSetAttribute(back_tail_tc_kernel<RAT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)tp.gback.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
-  }
-  back_tail_tc_kernel<RAT><<<tp.grid_back, TC_THREADS, tp.gback.total, st>>>(w, P);
-  TG_LAUNCH_CHECK();
-  return TGRAD_OK;
+  return tp.back_ns == 2 ? tc_back_op2<RAT, 2>(op, tp, w, P, st) : tc_back_op2<RAT, 1>(op, tp, w, P, st);
 }
 // op: 0 = set attributes (both kernels), 1 = proj, 2 = back
 tgrad_status tc_dispatch(int op, const TailPlan& tp, void* ptr, const TailTcParams& P, cudaStream_t st) {
@@ -293,10 +298,11 @@ tgrad_status plan_tail(tgrad_state* s) {
     tp.rat = rat; tp.ks = ks;
     // compression kernel: blocks of 4 warps; two row tiles per warp for 64-row slabs (measured faster than
     // 8 warps with one tile each: 101 against 122 us on 128x128x64x33)
-    tp.pjw = 4; tp.ntw = (A == 64) ? 2 : 1;
-    const int pj_blocks = tp.pjw == 8 ? 2 : (tp.ntw == 2 ? 3 : 4);     // resident blocks per SM
+    tp.pjw = 4; tp.ntw = (A == 64) ? 2 : (A == 32 ? 4 : 2);
+    tp.back_ns = ((uint64_t)A * B * 8 <= 8192) ? 2 : 1;      // small slabs: two per warp and iteration
+    const int pj_blocks = tp.pjw == 8 ? 2 : (tp.ntw == 1 ? 4 : 3);     // resident blocks per SM
     const uint32_t pj_smem = (227u * 1024u) / pj_blocks - 1024u;
-    if (proj_tc_geom(A, B, rat, (uint32_t)S, tp.ntw, tp.pjw, pj_smem, tp.gproj) && tail_tc_geom(true, A, B, rat, (uint32_t)S, tp.gback)) {
+    if (proj_tc_geom(A, B, rat, (uint32_t)S, tp.ntw, tp.pjw, pj_smem, tp.gproj) && tail_tc_geom(true, A, B, rat, (uint32_t)S, tp.back_ns, tp.gback)) {
       const uint32_t cap = 2u * (uint32_t)s->sm_count, pcap = (uint32_t)pj_blocks * (uint32_t)s->sm_count;
       tp.grid_proj = (int)(tp.gproj.ngroups < pcap ? tp.gproj.ngroups : pcap);
       tp.grid_back = (int)(tp.gback.ngroups < cap ? tp.gback.ngroups : cap);
