@@ -66,231 +66,204 @@ __device__ __forceinline__ void load_row_bcast(const cf* __restrict__ row, cf (&
   }
 }
 
-// Shared-memory layout (units of cf = 8 bytes; every region starts on 16 bytes):
-//   [B][rbp] small factor | [A][ras] large factor | per warp: [A][Bs] slab, then the small tile
-__host__ __device__ inline size_t tail_even(size_t x) { return (x + 1) & ~(size_t)1; }
-__host__ __device__ inline size_t tail_warp_elems(int A, int Bs, int ra, int rbp, bool back) {
-  return tail_even((size_t)A * Bs) + (back ? (size_t)ra * rbp : (size_t)A * rbp);
-}
-__host__ __device__ inline size_t tail_smem_bytes(int A, int B, int Bs, int ra, int ras, int rbp, int nwarps, bool back) {
-  return 8 * ((size_t)B * rbp + tail_even((size_t)A * ras) + (size_t)nwarps * tail_warp_elems(A, Bs, ra, rbp, back));
+// ---------------------------------------------------------------------------------------------
+// General streaming kernels (any slab shape that fits in shared memory, both storage types): one
+// thread block per slab at a time, fp32 FMA arithmetic.  Shared memory (units of cf):
+//   X/W slab [A][Bs] | Y [A][rbp] | Ub [B][rbp] | (back) T' [ra][rbp] | (back) Ua [A][ras]
+// Bs, ras odd (conflict-free column walks); rbp = rb rounded up to a multiple of 8.
+// ---------------------------------------------------------------------------------------------
+constexpr int TB_THREADS = 256;
+constexpr int TB_YR = 16;        // Y entries a thread keeps in registers in the last product of the reconstruction
+
+struct TailBlkGeom {
+  int Bs, rbp, ras, js;          // padded strides; js = threads per slab row in the products over b
+  uint32_t off_y, off_ub, off_t, off_ua, total;   // byte offsets
+};
+__host__ inline TailBlkGeom tail_blk_geom(int A, int B, int ra, int rb, bool back) {
+  TailBlkGeom g;
+  g.Bs = B | 1; g.rbp = (rb + 7) & ~7; g.ras = ra | 1; g.js = g.rbp / 8;
+  size_t o = (size_t)A * g.Bs * 8; o = (o + 15) & ~(size_t)15;
+  g.off_y = (uint32_t)o; o += (size_t)A * g.rbp * 8;
+  g.off_ub = (uint32_t)o; o += (size_t)B * g.rbp * 8;
+  g.off_t = (uint32_t)o; if (back) o += (size_t)ra * g.rbp * 8;
+  g.off_ua = (uint32_t)o; if (back) o += (((size_t)A * g.ras * 8) + 15) & ~(size_t)15;
+  g.total = (uint32_t)o;
+  return g;
 }
 
-template <class S, int RPL, int RBP>
-__global__ void __launch_bounds__(256) proj_tail_kernel(const void* __restrict__ g, TailParams p) {
+// Compression of the two trailing modes of one slab at a time, fused with the sparse gather and the
+// residual:  Y[a][jb] = sum_b R[a][b] conj(Ub[b][jb]),  T[ja][jb] = sum_a conj(Ua[a][ja]) Y[a][jb].
+// The gathered sparse values go to p.g_s (their AdamUpdate runs with the core's).
+template <class S>
+__global__ void __launch_bounds__(TB_THREADS) proj_tail_blk_kernel(const void* __restrict__ g, TailParams p, TailBlkGeom G) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int nw = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int A = p.A, B = p.B, Bs = p.Bs, ra = p.ra, rb = p.rb, ras = p.ras;
-  cf* ub_s = reinterpret_cast<cf*>(smem_raw);              // [B][RBP]   conj(Ub), zero padded
-  cf* ua_s = ub_s + (size_t)B * RBP;                       // [A][ras]   conj(Ua)
-  cf* xs = ua_s + tail_even((size_t)A * ras) + (size_t)warp * tail_warp_elems(A, Bs, ra, RBP, false);   // [A][Bs]
-  cf* ys = xs + tail_even((size_t)A * Bs);                 // [A][RBP]
-
-  for (int i = threadIdx.x; i < B * RBP; i += blockDim.x) {
-    int b = i / RBP, j = i - b * RBP;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int A = p.A, B = p.B, Bs = G.Bs, ra = p.ra, rb = p.rb, rbp = G.rbp, js = G.js;
+  cf* xs = reinterpret_cast<cf*>(smem_raw);
+  cf* ys = reinterpret_cast<cf*>(smem_raw + G.off_y);
+  cf* ubs = reinterpret_cast<cf*>(smem_raw + G.off_ub);      // conj(Ub), zero padded
+  for (int i = tid; i < B * rbp; i += TB_THREADS) {
+    const int b = i / rbp, j = i - b * rbp;
     cf u = (j < rb) ? p.Ub[b * rb + j] : make_float2(0.f, 0.f);
-    ub_s[i] = make_float2(u.x, -u.y);
+    ubs[i] = make_float2(u.x, -u.y);
   }
-  for (int i = threadIdx.x; i < A * ra; i += blockDim.x) {
-    int a = i / ra, j = i - a * ra;
-    cf u = p.Ua[i];
-    ua_s[a * ras + j] = make_float2(u.x, -u.y);
-  }
-  __syncthreads();
-
   const uint32_t E = p.E;
-  for (uint32_t s = blockIdx.x * nw + warp; s < p.nslab; s += gridDim.x * nw) {
+  const int rows_pp = TB_THREADS / js, arow = tid / js, jq = (tid - arow * js) * 8;
+  for (uint32_t s = blockIdx.x; s < p.nslab; s += gridDim.x) {
     const size_t gbase = (size_t)s * E;
-    // ---- slab -> shared (row stride Bs) ----
-    if (Bs == B) {
-      for (uint32_t i = lane; i < E; i += 32) xs[i] = S::load(g, gbase + i);
-    } else {
-      for (uint32_t i = lane; i < E; i += 32) { uint32_t a = i / B; xs[a * Bs + (i - a * B)] = S::load(g, gbase + i); }
-    }
-    __syncwarp();
-    // ---- sparse part: gather, Adam, zero (residual) ----
+    __syncthreads();                                     // the previous slab's products are done with xs / ys
+    for (int a = warp; a < A; a += TB_THREADS / 32)
+      for (int b = lane; b < B; b += 32) xs[a * Bs + b] = S::load(g, gbase + (size_t)a * B + b);
+    __syncthreads();
     if (p.k > 0) {
       const int j0 = (int)p.slab_ptr[s], j1 = (int)p.slab_ptr[s + 1];
-      for (int j = j0 + lane; j < j1; j += 32) {
-        uint32_t loc = p.omega[j] - (uint32_t)gbase;
-        uint32_t a = loc / B;
-        uint32_t si = a * Bs + (loc - a * B);
-        cf x = xs[si];
+      for (int j = j0 + tid; j < j1; j += TB_THREADS) {
+        const uint32_t loc = p.omega[j] - (uint32_t)gbase;
+        const uint32_t a = loc / B;
+        const uint32_t si = a * Bs + (loc - a * B);
+        p.g_s[j] = xs[si];
         xs[si] = make_float2(0.f, 0.f);
-        cf m = p.m_s[j]; float v = p.v_s[j];
-        cf n = adam_apply(x, m, v, p.adam);
-        p.m_s[j] = m; p.v_s[j] = v; p.n_s[j] = n;
       }
-      __syncwarp();
+      __syncthreads();
     }
-    // ---- mode N:  Y[a][jb] = sum_b R[a][b] conj(Ub[b][jb]) ----
-    for (int a0 = 0; a0 < A; a0 += 32 * RPL) {
-      cf acc[RPL][RBP];
+    // ---- mode N: a thread owns 8 consecutive jb of one row ----
+    for (int a = arow; a < A; a += rows_pp) {
+      cf acc[8];
 #pragma unroll
-      for (int r = 0; r < RPL; ++r)
-#pragma unroll
-        for (int j = 0; j < RBP; ++j) acc[r][j] = make_float2(0.f, 0.f);
-      int arow[RPL];
-#pragma unroll
-      for (int r = 0; r < RPL; ++r) { int a = a0 + lane + 32 * r; arow[r] = (a < A ? a : A - 1) * Bs; }
+      for (int j = 0; j < 8; ++j) acc[j] = make_float2(0.f, 0.f);
+      const cf* xr = xs + a * Bs;
       for (int b = 0; b < B; ++b) {
-        cf u[RBP];
-        load_row_bcast<RBP>(ub_s + b * RBP, u);
+        const cf x = xr[b];
+        cf u[8];
+        load_row_bcast<8>(ubs + b * rbp + jq, u);
 #pragma unroll
-        for (int r = 0; r < RPL; ++r) {
-          cf x = xs[arow[r] + b];
-#pragma unroll
-          for (int j = 0; j < RBP; ++j) cfma(acc[r][j], x, u[j]);
-        }
+        for (int j = 0; j < 8; ++j) cfma(acc[j], x, u[j]);
       }
 #pragma unroll
-      for (int r = 0; r < RPL; ++r) {
-        int a = a0 + lane + 32 * r;
-        if (a < A) {
-#pragma unroll
-          for (int j = 0; j < RBP; ++j) ys[a * RBP + j] = acc[r][j];
-        }
-      }
+      for (int j = 0; j < 8; ++j) ys[a * rbp + jq + j] = acc[j];
     }
-    __syncwarp();
-    // ---- mode N-1:  T[ja][jb] = sum_a conj(Ua[a][ja]) Y[a][jb];  4 consecutive jb per lane ----
-    {
-      constexpr int QJ = RBP / 4;
-      const int ntask = ra * QJ;
-      cf* tout = p.t + (size_t)s * ra * rb;
-      for (int task = lane; task < ntask; task += 32) {
-        int ja = task / QJ, jq = task - ja * QJ;
-        cf acc[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[j] = make_float2(0.f, 0.f);
-        const cf* yp = ys + jq * 4;
-        const cf* up = ua_s + ja;
-        for (int a = 0; a < A; ++a) {
-          cf u = up[a * ras];
-          cf y[4];
-          load_row_bcast<4>(yp + a * RBP, y);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) cfma(acc[j], u, y[j]);
-        }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          int jb = jq * 4 + j;
-          if (jb < rb) tout[ja * rb + jb] = acc[j];
-        }
-      }
+    __syncthreads();
+    // ---- mode N-1: one output T[ja][jb] per thread and pass ----
+    cf* tout = p.t + (size_t)s * ra * rb;
+    for (int o = tid; o < ra * rb; o += TB_THREADS) {
+      const int ja = o / rb, jb = o - ja * rb;
+      cf acc = make_float2(0.f, 0.f);
+#pragma unroll 4
+      for (int a = 0; a < A; ++a) cfma_conj(acc, ys[a * rbp + jb], __ldg(&p.Ua[a * ra + ja]));   // y * conj(u)
+      tout[o] = acc;
     }
-    __syncwarp();
   }
 }
 
-template <class S, int RPL, int RBP>
-__global__ void __launch_bounds__(256) back_tail_kernel(void* __restrict__ w, TailParams p) {
+// Reconstruction of the two trailing modes of one slab at a time, fused with the weight update and the
+// sparse add:  Y'[a][jb] = sum_ja Ua[a][ja] T'[ja][jb],  D[a][b] = sum_jb Y'[a][jb] Ub[b][jb],
+// W <- (1 - eta wd) W - eta alpha D, then W[Omega] -= eta lambda N_S (half storage: the dense result is
+// rounded to fp16 before the sparse term is added, and once more when stored).
+template <class S>
+__global__ void __launch_bounds__(TB_THREADS) back_tail_blk_kernel(void* __restrict__ w, TailParams p, TailBlkGeom G) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int nw = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int A = p.A, B = p.B, Bs = p.Bs, ra = p.ra, rb = p.rb, ras = p.ras;
-  cf* ub_s = reinterpret_cast<cf*>(smem_raw);              // [B][RBP]  Ub, zero padded
-  cf* ua_s = ub_s + (size_t)B * RBP;                       // [A][ras]  Ua
-  cf* ws = ua_s + tail_even((size_t)A * ras) + (size_t)warp * tail_warp_elems(A, Bs, ra, RBP, true);    // [A][Bs]
-  cf* ts = ws + tail_even((size_t)A * Bs);                 // [ra][RBP]
-
-  for (int i = threadIdx.x; i < B * RBP; i += blockDim.x) {
-    int b = i / RBP, j = i - b * RBP;
-    ub_s[i] = (j < rb) ? p.Ub[b * rb + j] : make_float2(0.f, 0.f);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int A = p.A, B = p.B, Bs = G.Bs, ra = p.ra, rb = p.rb, rbp = G.rbp, ras = G.ras, js = G.js;
+  cf* ws = reinterpret_cast<cf*>(smem_raw);
+  cf* ys = reinterpret_cast<cf*>(smem_raw + G.off_y);
+  cf* ubs = reinterpret_cast<cf*>(smem_raw + G.off_ub);      // Ub, zero padded
+  cf* ts = reinterpret_cast<cf*>(smem_raw + G.off_t);
+  cf* uas = reinterpret_cast<cf*>(smem_raw + G.off_ua);
+  for (int i = tid; i < B * rbp; i += TB_THREADS) {
+    const int b = i / rbp, j = i - b * rbp;
+    ubs[i] = (j < rb) ? p.Ub[b * rb + j] : make_float2(0.f, 0.f);
   }
-  for (int i = threadIdx.x; i < A * ra; i += blockDim.x) {
-    int a = i / ra, j = i - a * ra;
-    ua_s[a * ras + j] = p.Ua[i];
+  for (int i = tid; i < A * ra; i += TB_THREADS) {
+    const int a = i / ra, j = i - a * ra;
+    uas[a * ras + j] = p.Ua[i];
   }
-  __syncthreads();
-
   const uint32_t E = p.E;
   const bool decay = p.decay != 1.0f;
-  for (uint32_t s = blockIdx.x * nw + warp; s < p.nslab; s += gridDim.x * nw) {
+  const int rows_pp = TB_THREADS / js, arow = tid / js, jq = (tid - arow * js) * 8;
+  // last product: tpr threads share a row, each walks every tpr-th column
+  const int tpr = (A >= TB_THREADS) ? 1 : TB_THREADS / A, rows_pp2 = TB_THREADS / tpr;
+  const int arow2 = tid / tpr, bq = tid - arow2 * tpr;
+  for (uint32_t s = blockIdx.x; s < p.nslab; s += gridDim.x) {
     const size_t gbase = (size_t)s * E;
-    // ---- W slab and T' tile -> shared ----
-    if (Bs == B) {
-      for (uint32_t i = lane; i < E; i += 32) ws[i] = S::load(w, gbase + i);
-    } else {
-      for (uint32_t i = lane; i < E; i += 32) { uint32_t a = i / B; ws[a * Bs + (i - a * B)] = S::load(w, gbase + i); }
-    }
+    __syncthreads();                                     // the previous slab has been stored
+    for (int a = warp; a < A; a += TB_THREADS / 32)
+      for (int b = lane; b < B; b += 32) {
+        cf v = S::load(w, gbase + (size_t)a * B + b);
+        if (decay) { v.x *= p.decay; v.y *= p.decay; }
+        ws[a * Bs + b] = v;
+      }
     {
       const cf* tin = p.t + (size_t)s * ra * rb;
-      for (int i = lane; i < ra * RBP; i += 32) {
-        int ja = i / RBP, j = i - ja * RBP;
+      for (int i = tid; i < ra * rbp; i += TB_THREADS) {
+        const int ja = i / rbp, j = i - ja * rbp;
         ts[i] = (j < rb) ? tin[ja * rb + j] : make_float2(0.f, 0.f);
       }
     }
-    __syncwarp();
-    for (int a0 = 0; a0 < A; a0 += 32 * RPL) {
-      // ---- mode N-1:  Y'[a][jb] = sum_ja Ua[a][ja] T'[ja][jb] ----
-      cf y[RPL][RBP];
+    __syncthreads();
+    // ---- mode N-1: a thread owns 8 consecutive jb of one row ----
+    for (int a = arow; a < A; a += rows_pp) {
+      cf acc[8];
 #pragma unroll
-      for (int r = 0; r < RPL; ++r)
-#pragma unroll
-        for (int j = 0; j < RBP; ++j) y[r][j] = make_float2(0.f, 0.f);
-      int urow[RPL], wrow[RPL];
-      bool ok[RPL];
-#pragma unroll
-      for (int r = 0; r < RPL; ++r) {
-        int a = a0 + lane + 32 * r;
-        ok[r] = a < A;
-        int ac = ok[r] ? a : A - 1;
-        urow[r] = ac * ras; wrow[r] = ac * Bs;
-      }
+      for (int j = 0; j < 8; ++j) acc[j] = make_float2(0.f, 0.f);
+      const cf* ur = uas + a * ras;
       for (int ja = 0; ja < ra; ++ja) {
-        cf tv[RBP];
-        load_row_bcast<RBP>(ts + ja * RBP, tv);
+        const cf u = ur[ja];
+        cf tv[8];
+        load_row_bcast<8>(ts + ja * rbp + jq, tv);
 #pragma unroll
-        for (int r = 0; r < RPL; ++r) {
-          cf u = ua_s[urow[r] + ja];
-#pragma unroll
-          for (int j = 0; j < RBP; ++j) cfma(y[r][j], u, tv[j]);
-        }
+        for (int j = 0; j < 8; ++j) cfma(acc[j], u, tv[j]);
       }
-      // ---- mode N:  D[a][b] = sum_jb Y'[a][jb] Ub[b][jb];  W <- decay*W - eta*alpha*D ----
-      for (int b = 0; b < B; ++b) {
-        cf u[RBP];
-        load_row_bcast<RBP>(ub_s + b * RBP, u);
 #pragma unroll
-        for (int r = 0; r < RPL; ++r) {
+      for (int j = 0; j < 8; ++j) ys[a * rbp + jq + j] = acc[j];
+    }
+    __syncthreads();
+    // ---- mode N: Y'[a][.] in registers (TB_YR at a time), applied to the row column by column ----
+    for (int a = arow2; a < A; a += rows_pp2) {
+      for (int jc = 0; jc < rbp; jc += TB_YR) {
+        cf y[TB_YR];
+#pragma unroll
+        for (int j = 0; j < TB_YR; j += 8) {
+          if (jc + j < rbp) load_row_bcast<8>(ys + a * rbp + jc + j, *reinterpret_cast<cf(*)[8]>(&y[j]));
+          else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) y[j + q] = make_float2(0.f, 0.f);
+          }
+        }
+        for (int b = bq; b < B; b += tpr) {
           cf d = make_float2(0.f, 0.f);
 #pragma unroll
-          for (int j = 0; j < RBP; ++j) cfma(d, y[r][j], u[j]);
-          if (ok[r]) {
-            cf wv = ws[wrow[r] + b];
-            if (decay) { wv.x *= p.decay; wv.y *= p.decay; }
-            wv.x = fmaf(-p.s_low, d.x, wv.x);
-            wv.y = fmaf(-p.s_low, d.y, wv.y);
-            ws[wrow[r] + b] = wv;
+          for (int j = 0; j < TB_YR; j += 8) {
+            if (jc + j < rbp) {
+              cf u[8];
+              load_row_bcast<8>(ubs + b * rbp + jc + j, u);
+#pragma unroll
+              for (int q = 0; q < 8; ++q) cfma(d, y[j + q], u[q]);
+            }
           }
+          cf wv = ws[a * Bs + b];
+          wv.x = fmaf(-p.s_low, d.x, wv.x); wv.y = fmaf(-p.s_low, d.y, wv.y);
+          ws[a * Bs + b] = wv;
         }
       }
     }
-    __syncwarp();
+    __syncthreads();
     // ---- scaled sparse add at Omega (on top of the dense update) ----
     if (p.k > 0) {
       const int j0 = (int)p.slab_ptr[s], j1 = (int)p.slab_ptr[s + 1];
-      for (int j = j0 + lane; j < j1; j += 32) {
-        uint32_t loc = p.omega[j] - (uint32_t)gbase;
-        uint32_t a = loc / B;
-        uint32_t si = a * Bs + (loc - a * B);
+      for (int j = j0 + tid; j < j1; j += TB_THREADS) {
+        const uint32_t loc = p.omega[j] - (uint32_t)gbase;
+        const uint32_t a = loc / B;
+        const uint32_t si = a * Bs + (loc - a * B);
         cf wv = ws[si];
-        if (S::kBytes == 4) {   // half storage: the dense update is rounded to fp16 before the sparse add
-          wv = __half22float2(__floats2half2_rn(wv.x, wv.y));
-        }
-        cf n = p.n_s[j];
-        wv.x = fmaf(-p.s_sparse, n.x, wv.x);
-        wv.y = fmaf(-p.s_sparse, n.y, wv.y);
+        if (S::kBytes == 4) wv = __half22float2(__floats2half2_rn(wv.x, wv.y));
+        const cf n = p.n_s[j];
+        wv.x = fmaf(-p.s_sparse, n.x, wv.x); wv.y = fmaf(-p.s_sparse, n.y, wv.y);
         ws[si] = wv;
       }
-      __syncwarp();
+      __syncthreads();
     }
-    if (Bs == B) {
-      for (uint32_t i = lane; i < E; i += 32) S::store(w, gbase + i, ws[i]);
-    } else {
-      for (uint32_t i = lane; i < E; i += 32) { uint32_t a = i / B; S::store(w, gbase + i, ws[a * Bs + (i - a * B)]); }
-    }
-    __syncwarp();
+    for (int a = warp; a < A; a += TB_THREADS / 32)
+      for (int b = lane; b < B; b += 32) S::store(w, gbase + (size_t)a * B + b, ws[a * Bs + b]);
   }
 }
 

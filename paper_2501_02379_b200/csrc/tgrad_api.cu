@@ -43,8 +43,9 @@ struct Layout {
 };
 
 struct TailPlan {
-  int rpl, rbp, nwarps, grid;
-  size_t smem_proj, smem_back;
+  // general path: one block per slab
+  TailBlkGeom bproj, bback;
+  int grid_bproj, grid_bback;
   // tensor-core fast path (complex64 storage, 16/32/64 slab rows, small trailing ranks)
   bool tc;
   int rat, ks, ntw, pjw, back_ns;
@@ -76,7 +77,6 @@ tgrad_status validate(const tgrad_config* c) {
   return TGRAD_OK;
 }
 
-int pick_rbp(int rb) { return rb <= 4 ? 4 : rb <= 8 ? 8 : rb <= 16 ? 16 : 32; }
 
 void plan_gram(const tgrad_config* c, int n, int sm, uint32_t& chunks, uint32_t& cps, int& splits) {
   uint64_t O = 1, C = 1;
@@ -170,34 +170,20 @@ namespace {
     if (cudaPeekAtLastError() != cudaSuccess) return TGRAD_ERR_CUDA; \
   } while (0)
 
-template <class S, int RPL, int RBP>
-tgrad_status tail_attr(const TailPlan& tp) {
-  if (cudaFuncSetAttribute(proj_tail_kernel<S, RPL, RBP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)tp.smem_proj) != cudaSuccess) return TGRAD_ERR_CUDA;
-  if (cudaFuncSetAttribute(back_tail_kernel<S, RPL, RBP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)tp.smem_back) != cudaSuccess) return TGRAD_ERR_CUDA;
-  return TGRAD_OK;
-}
-
-template <class S, int RPL, int RBP>
-tgrad_status tail_launch(bool back, const TailPlan& tp, void* ptr, const TailParams& p, cudaStream_t st) {
-  if (back) back_tail_kernel<S, RPL, RBP><<<tp.grid, tp.nwarps * 32, tp.smem_back, st>>>(ptr, p);
-  else proj_tail_kernel<S, RPL, RBP><<<tp.grid, tp.nwarps * 32, tp.smem_proj, st>>>(ptr, p);
-  TG_LAUNCH_CHECK();
-  return TGRAD_OK;
-}
-
 // op: 0 = set attributes, 1 = proj, 2 = back
 template <class S>
 tgrad_status tail_dispatch(int op, const TailPlan& tp, void* ptr, const TailParams& p, cudaStream_t st) {
-#define TG_CASE(RPL_, RBP_)                                                     \
-  if (tp.rpl == RPL_ && tp.rbp == RBP_) {                                       \
-    if (op == 0) return tail_attr<S, RPL_, RBP_>(tp);                           \
-    return tail_launch<S, RPL_, RBP_>(op == 2, tp, ptr, p, st);                 \
+  if (op == 0) {
+    if (cudaFuncSetAttribute(proj_tail_blk_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tp.bproj.total) != cudaSuccess) return TGRAD_ERR_CUDA;
+    if (cudaFuncSetAttribute(back_tail_blk_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tp.bback.total) != cudaSuccess) return TGRAD_ERR_CUDA;
+    return TGRAD_OK;
   }
-  TG_CASE(1, 4) TG_CASE(2, 4) TG_CASE(4, 4) TG_CASE(1, 8) TG_CASE(2, 8) TG_CASE(1, 16) TG_CASE(1, 32)
-#undef TG_CASE
-  return TGRAD_ERR_UNSUPPORTED;
+  if (op == 2) back_tail_blk_kernel<S><<<tp.grid_bback, TB_THREADS, tp.bback.total, st>>>(ptr, p, tp.bback);
+  else proj_tail_blk_kernel<S><<<tp.grid_bproj, TB_THREADS, tp.bproj.total, st>>>(ptr, p, tp.bproj);
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
 }
 
 tgrad_status tail_any(const tgrad_state* s, int op, void* ptr, const TailParams& p, cudaStream_t st) {
@@ -259,33 +245,18 @@ tgrad_status plan_tail(tgrad_state* s) {
   const int N = c.ndim;
   const int A = (int)c.dims[N - 2], B = (int)c.dims[N - 1], ra = c.ranks[N - 2], rb = c.ranks[N - 1];
   TailPlan& tp = s->tail;
-  tp.rbp = pick_rbp(rb);
-  int rows = (A + 31) / 32, cap = 16 / tp.rbp; if (cap < 1) cap = 1;
-  int rpl = rows < cap ? rows : cap;
-  tp.rpl = rpl >= 4 ? 4 : rpl >= 2 ? 2 : 1;
-  const int Bs = B | 1, ras = ra | 1;
   const size_t kMax = 227 * 1024;
-  int nw = 0;
-  const int cand[4] = {8, 4, 2, 1};
-  const size_t lim[3] = {56 * 1024, 113 * 1024, kMax};
-  for (int li = 0; li < 3 && !nw; ++li)
-    for (int ci = (li == 0 ? 0 : 1); ci < 4; ++ci) {
-      size_t a = tail_smem_bytes(A, B, Bs, ra, ras, tp.rbp, cand[ci], false);
-      size_t b = tail_smem_bytes(A, B, Bs, ra, ras, tp.rbp, cand[ci], true);
-      if ((a > b ? a : b) <= lim[li]) { nw = cand[ci]; break; }
-    }
-  if (!nw) return TGRAD_ERR_UNSUPPORTED;   // a trailing A x B slab does not fit in shared memory
-  tp.nwarps = nw;
-  tp.smem_proj = tail_smem_bytes(A, B, Bs, ra, ras, tp.rbp, nw, false);
-  tp.smem_back = tail_smem_bytes(A, B, Bs, ra, ras, tp.rbp, nw, true);
-  size_t sm = tp.smem_proj > tp.smem_back ? tp.smem_proj : tp.smem_back;
-  int per_sm = (int)(kMax / (sm + 1024)); if (per_sm < 1) per_sm = 1;
-  int by_threads = 2048 / (nw * 32); if (per_sm > by_threads) per_sm = by_threads;
-  if (per_sm > 16) per_sm = 16;
+  tp.bproj = tail_blk_geom(A, B, ra, rb, false);
+  tp.bback = tail_blk_geom(A, B, ra, rb, true);
+  if (tp.bproj.total > kMax || tp.bback.total > kMax) return TGRAD_ERR_UNSUPPORTED;   // a trailing A x B slab does not fit in shared memory
   uint64_t S = s->L.numel / ((uint64_t)A * B);
-  uint64_t need = (S + nw - 1) / nw;
-  uint64_t g = (uint64_t)s->sm_count * per_sm;
-  tp.grid = (int)(need < g ? need : g);
+  {
+    const int pp = (int)(kMax / (tp.bproj.total + 1024)), pb = (int)(kMax / (tp.bback.total + 1024));
+    const uint64_t gp = (uint64_t)s->sm_count * (pp < 1 ? 1 : (pp > 8 ? 8 : pp));
+    const uint64_t gb = (uint64_t)s->sm_count * (pb < 1 ? 1 : (pb > 8 ? 8 : pb));
+    tp.grid_bproj = (int)(S < gp ? S : gp);
+    tp.grid_bback = (int)(S < gb ? S : gb);
+  }
   TailParams dummy; memset(&dummy, 0, sizeof(dummy));
   tgrad_status r = tail_any(s, 0, nullptr, dummy, 0);
   if (r != TGRAD_OK) return r;
@@ -513,7 +484,7 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
     TG_MARK(2);
     cf* bufs[2] = {bufa, bufb};
     int which = ((N - 2) & 1) ? 0 : 1;          // make the last product land in bufa
-    const uint32_t ks = s->tail.tc ? (uint32_t)c.k : 0u;      // the general streaming kernel updates the sparse moments itself
+    const uint32_t ks = (uint32_t)c.k;
     const cf* src;
     int mfirst;
     if (fused) {
