@@ -260,7 +260,6 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW == 1 ?
         p.g_s[j] = *xp;
         *xp = make_float2(0.f, 0.f);
       }
-      fence_async_smem();      // the zeroed entries were written through the generic proxy; a later bulk copy overwrites them
     }
     if (__syncthreads_or(!ok)) {
       // a copy did not arrive: record it, let the copies still in flight land (bounded), leave
@@ -342,6 +341,9 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW == 1 ?
     // ---- off the critical path: the previous group's T, the next group's entries ----
     if (it > 0) reduce_out(u - gstride, it - 1);
     if (sparse) {
+      // the zeroed entries were written through the generic proxy and a later bulk copy overwrites them: the
+      // proxy fence of the writing threads can wait until here (the refill is issued after the next barrier)
+      if (jcur < b1) fence_async_smem();
       b0 = c0; b1 = c1; pom = pomc;
       c0 = n0; c1 = n1;
       if (c0 + tid < c1) pomc = p.omega[c0 + tid];
