@@ -91,6 +91,15 @@ __device__ __forceinline__ void mma_tf32(float (&d)[4], float a0, float a1, floa
         "r"(__float_as_uint(b0)), "r"(__float_as_uint(b1)));
 }
 
+// D(16x8) += A(16x16, row) * B(16x8, col), fp16 inputs (two per register), fp32 accumulate.
+// lane = 4 g + t:  a0 (g, 2t..2t+1)  a1 (g+8, 2t..)  a2 (g, 2t+8..)  a3 (g+8, 2t+8..);
+// b0 (k = 2t..2t+1, n = g)  b1 (k = 2t+8..2t+9, n = g);  d as for the TF32 shape.
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
 // The same MMA with operand a1 (resp. a1 and a3) negated inside the instruction sequence, so that the
 // negated copies of loop-invariant fragments do not occupy registers across the loop.
 __device__ __forceinline__ void mma_tf32_n1(float (&d)[4], float a0, float a1, float a2, float a3, float b0, float b1) {

@@ -1,0 +1,283 @@
+// Streaming kernels for half-precision storage (W and G as interleaved fp16 pairs; the mixed-precision
+// recipe of Section 2.3) and slabs of up to 128 rows.
+//
+// A slab arrives by one bulk asynchronous copy as it is stored (fp16), and stays fp16 in shared memory.
+// fp16 values are exact fp16 MMA operands, so the first trailing-mode product needs no splitting of the
+// streamed operand at all: Y = X conj(Ub) is two m16n8k16 MMAs per step (Ub = hi + lo in fp16, X exact),
+// at twice the K per instruction of the TF32 shape.  The second product (over the slab rows) and the
+// reconstruction run as split-precision TF32 like the fp32-storage kernels.
+//
+// A block has one warp per tile of 8 slab rows (A/8 warps, at most 16) and works on one slab at a time
+// from a ring of bulk copies; one block per SM.
+#pragma once
+#include "common.cuh"
+#include "ptx.cuh"
+#include "tail.cuh"
+#include "tail_tc.cuh"
+
+namespace tg {
+
+struct TailHGeom {
+  int nwarps, nbuf, ks16;      // warps (= row tiles of 8), ring depth, k16-steps of the first product (8 columns b each)
+  int ldy, ldu;                // row lengths (complex) of the Y and Ua copies in shared memory
+  int ntile2, ksplit;          // second product: (m, n) output tiles, and how many warps share one tile's K range
+  uint32_t slab_bytes, buf_stride;
+  uint32_t off_u1, off_ua, off_y, off_part, off_bar, total;
+};
+
+__host__ inline bool tail_h_geom(int A, int B, int ra, int rb, TailHGeom& g) {
+  if (A % 8 || A < 8 || A > 128) return false;
+  const int rat = (ra + 7) / 8, rbt = (rb + 7) / 8;
+  if (rat > 4 || rbt > 2) return false;
+  g.nwarps = A / 8;
+  g.ks16 = 4 * (B / 32) + ((B % 32) < 4 ? (B % 32) : 4);     // see the column mapping of the first product
+  g.ldy = 8 * rbt + 4; g.ldu = 8 * rat + 4;
+  g.ntile2 = rat * rbt;
+  g.ksplit = g.nwarps >= g.ntile2 ? g.nwarps / g.ntile2 : 1;
+  if ((A / 4) % g.ksplit) return false;
+  g.slab_bytes = (uint32_t)A * B * 4;
+  if (g.slab_bytes % 16) return false;
+  g.buf_stride = (g.slab_bytes + 127) & ~127u;
+  const uint32_t u1 = (uint32_t)g.ks16 * rbt * 2 * 32 * 16;              // (hi, lo) x 4 registers per lane
+  const uint32_t ua = (uint32_t)A * g.ldu * 8;
+  const uint32_t y = 2u * A * g.ldy * 8;                                  // two stages
+  const uint32_t units = (uint32_t)g.ntile2 * g.ksplit;
+  const uint32_t part = 2u * units * 128 * 4;                             // two stages of partial tiles
+  const uint32_t fixed = u1 + ua + y + part + 256;
+  if (fixed + 2 * g.buf_stride > 227u * 1024u) return false;
+  int nbuf = (int)((227u * 1024u - fixed) / g.buf_stride);
+  if (nbuf > 4) nbuf = 4;
+  g.nbuf = nbuf;
+  g.off_u1 = (uint32_t)nbuf * g.buf_stride;
+  g.off_ua = g.off_u1 + u1;
+  g.off_y = g.off_ua + ua;
+  g.off_part = g.off_y + y;
+  g.off_bar = g.off_part + part;
+  g.total = g.off_bar + 256;
+  return true;
+}
+
+struct TailHParams {
+  TailParams p;
+  TailHGeom g;
+  int* flags;
+};
+
+__device__ __forceinline__ uint32_t h2_bits(__half2 v) { return *reinterpret_cast<uint32_t*>(&v); }
+
+// x = hi + lo in fp16 (|x| <= 1: the factor matrices have orthonormal columns)
+__device__ __forceinline__ void split_f16(float x, __half& hi, __half& lo) {
+  hi = __float2half_rn(x);
+  lo = __float2half_rn(x - __half2float(hi));
+}
+
+// ---------------------------------------------------------------------------------------------
+// Compression of the two trailing modes (half storage), fused with the sparse gather and the residual.
+//   stage 1 (fp16 m16n8k16), warp = tile of 8 rows a:
+//     D1[(c,jb)][a] = sum_{(b,c')} W1[(c,jb)][(b,c')] X[a][(b,c')],  W1 rows (re,jb): (ur, ui), rows (im,jb): (-ui, ur)
+//     step ks = (kb, jj): k = 2t, 2t+1 <-> (b1, re|im), k = 2t+8, 2t+9 <-> (b2, re|im), b1 = 32 kb + 8 t + jj, b2 = b1 + 4
+//     (lanes of a quad read columns 8 apart: with rows of 65 words, all 32 loads of a step hit distinct banks)
+//   stage 2 (split TF32 m16n8k8), block-wide: T'[(c,ja)][jb] = sum_{(a,c')} W2[(c,ja)][(a,c')] Y[(a,c')][jb];
+//     a warp owns output tile (mt, nt) over one share of the rows a; step: k = t <-> (a, re), k = t+4 <-> (a, im), a = 4 q + t
+// Software pipeline over the slabs of a block: iteration `it` runs stage 1 of slab it, stage 2 of slab it-1
+// and the final sum of slab it-2, with one block-wide barrier.
+// ---------------------------------------------------------------------------------------------
+template <int RAT, int RBT>
+__global__ void __launch_bounds__(512, 1) proj_tail_h_kernel(const void* __restrict__ g, TailHParams P) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const TailParams& p = P.p;
+  const TailHGeom& G = P.g;
+  const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t = lane & 3;
+  const int A = p.A, B = p.B, ra = p.ra, rb = p.rb, nbuf = G.nbuf, ldy = G.ldy, ldu = G.ldu, nwarps = G.nwarps;
+  const int ks16 = G.ks16, ksplit = G.ksplit, units = G.ntile2 * G.ksplit;
+  const uint32_t E = p.E, nslab = p.nslab, gstride = gridDim.x;
+  uint4* u1tab = reinterpret_cast<uint4*>(smem + G.off_u1);       // [ks16][RBT][hi|lo][32]
+  cf* uas = reinterpret_cast<cf*>(smem + G.off_ua);               // [A][ldu]
+  cf* ysb = reinterpret_cast<cf*>(smem + G.off_y);                // [2][A][ldy]
+  float* part = reinterpret_cast<float*>(smem + G.off_part);      // [2][units][128]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + G.off_bar);
+  const unsigned char* gb = static_cast<const unsigned char*>(g);
+
+  // ---- Ub as stage-1 A fragments ----
+  for (int idx = tid; idx < ks16 * RBT * 32; idx += nthr) {
+    const int ks = idx / (RBT * 32), rem = idx - ks * (RBT * 32), jt = rem >> 5, ln = rem & 31;
+    const int jb = 8 * jt + (ln >> 2), b1 = 32 * (ks >> 2) + 8 * (ln & 3) + (ks & 3), b2 = b1 + 4;
+    cf v1 = (b1 < B && jb < rb) ? p.Ub[b1 * rb + jb] : make_float2(0.f, 0.f);
+    cf v2 = (b2 < B && jb < rb) ? p.Ub[b2 * rb + jb] : make_float2(0.f, 0.f);
+    __half r1h, r1l, i1h, i1l, r2h, r2l, i2h, i2l;
+    split_f16(v1.x, r1h, r1l); split_f16(v1.y, i1h, i1l);
+    split_f16(v2.x, r2h, r2l); split_f16(v2.y, i2h, i2l);
+    uint4 hi, lo;
+    hi.x = h2_bits(__halves2half2(r1h, i1h)); hi.y = h2_bits(__halves2half2(__hneg(i1h), r1h));
+    hi.z = h2_bits(__halves2half2(r2h, i2h)); hi.w = h2_bits(__halves2half2(__hneg(i2h), r2h));
+    lo.x = h2_bits(__halves2half2(r1l, i1l)); lo.y = h2_bits(__halves2half2(__hneg(i1l), r1l));
+    lo.z = h2_bits(__halves2half2(r2l, i2l)); lo.w = h2_bits(__halves2half2(__hneg(i2l), r2l));
+    u1tab[((ks * RBT + jt) * 2 + 0) * 32 + ln] = hi;
+    u1tab[((ks * RBT + jt) * 2 + 1) * 32 + ln] = lo;
+  }
+  for (int idx = tid; idx < A * ldu; idx += nthr) {
+    const int a = idx / ldu, j = idx - a * ldu;
+    uas[idx] = (j < ra) ? p.Ua[a * ra + j] : make_float2(0.f, 0.f);
+  }
+  // ---- this thread's first two outputs of a slab: where their partial sums sit ----
+  const int n_out = ra * rb;
+  int o_src[2];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int o = tid + i * nthr;
+    o_src[i] = -1;
+    if (o < n_out) {
+      const int ja = o / rb, jb = o - ja * rb;
+      o_src[i] = (((ja >> 3) * RBT + (jb >> 3)) * ksplit) * 128 + (4 * (ja & 7) + ((jb & 7) >> 1)) * 4 + (jb & 1);
+    }
+  }
+  if (tid == 0) {
+    for (int i = 0; i < nbuf; ++i) mbar_init(&bars[i], 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  const uint32_t nmine = (nslab > blockIdx.x) ? (nslab - blockIdx.x + gstride - 1) / gstride : 0;   // slabs of this block
+  if (tid == 0) {
+    for (uint32_t i = 0; i < (uint32_t)nbuf && i < nmine; ++i) {
+      mbar_expect_tx(&bars[i], G.slab_bytes);
+      bulk_g2s(smem + (size_t)i * G.buf_stride, gb + (size_t)(blockIdx.x + i * gstride) * G.slab_bytes, G.slab_bytes, &bars[i]);
+    }
+  }
+  // ---- sparse side: entry bounds three slabs ahead, first entries two slabs ahead ----
+  const bool sparse = p.k > 0;
+  auto bounds = [&](uint32_t s, int& x0, int& x1) {
+    x0 = 0; x1 = 0;
+    if (s < nslab) { x0 = (int)p.slab_ptr[s]; x1 = (int)p.slab_ptr[s + 1]; }
+  };
+  int b0 = 0, b1 = 0, c0 = 0, c1 = 0;
+  uint32_t pom = 0, pomc = 0;
+  if (sparse) {
+    bounds(blockIdx.x, b0, b1);
+    bounds(blockIdx.x + gstride, c0, c1);
+    if (b0 + tid < b1) pom = p.omega[b0 + tid];
+    if (c0 + tid < c1) pomc = p.omega[c0 + tid];
+  }
+
+  uint32_t phase = 0;
+  int buf = 0, pbuf = 0;
+  for (uint32_t it = 0; it < nmine + 2; ++it) {
+    const uint32_t s = blockIdx.x + it * gstride;          // slab of stage 1 (valid while it < nmine)
+    bool ok = true;
+    if (it < nmine) {
+      int n0 = 0, n1 = 0;
+      if (sparse) bounds(s + 2 * gstride, n0, n1);
+      ok = mbar_wait_bounded(&bars[buf], phase);
+      uint32_t* xs = reinterpret_cast<uint32_t*>(smem + (size_t)buf * G.buf_stride);
+      if (sparse && ok) {
+        const uint32_t base = s * E;
+        for (int j = b0 + tid, first = 1; j < b1; j += nthr, first = 0) {
+          const uint32_t loc = (first ? pom : p.omega[j]) - base;
+          const uint32_t xv = xs[loc];
+          p.g_s[j] = __half22float2(*reinterpret_cast<const __half2*>(&xv));
+          xs[loc] = 0u;
+        }
+        if (b0 + tid < b1) fence_async_smem();   // the zeroed words were written through the generic proxy; a bulk copy overwrites them later
+        b0 = c0; b1 = c1; pom = pomc;
+        c0 = n0; c1 = n1;
+        if (c0 + tid < c1) pomc = p.omega[c0 + tid];
+      }
+    }
+    if (__syncthreads_or(!ok)) {
+      if (tid == 0) {
+        atomicOr(P.flags, 4);
+        uint32_t ph = phase; int bx = buf;
+        for (int i = 1; i + 1 < nbuf && it + i < nmine; ++i) {
+          if (++bx == nbuf) { bx = 0; ph ^= 1; }
+          mbar_wait_bounded(&bars[bx], ph, 1u << 16);
+        }
+      }
+      return;
+    }
+    // every warp is past its reads of the previous slab: its ring buffer takes the slab nbuf ahead of it
+    if (tid == 0 && it >= 1 && it - 1 + nbuf < nmine) {
+      mbar_expect_tx(&bars[pbuf], G.slab_bytes);
+      bulk_g2s(smem + (size_t)pbuf * G.buf_stride, gb + (size_t)(blockIdx.x + (it - 1 + nbuf) * gstride) * G.slab_bytes,
+               G.slab_bytes, &bars[pbuf]);
+    }
+    // ---- final sum of slab it-2 (its partial tiles were written during iteration it-1) ----
+    if (it >= 2) {
+      const float* pp = part + (size_t)((it - 1) & 1) * units * 128;
+      float* tg_ = reinterpret_cast<float*>(p.t + (size_t)(blockIdx.x + (it - 2) * gstride) * n_out);
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        if (o_src[i] < 0) continue;
+        float re = 0.f, im = 0.f;
+        for (int kh = 0; kh < ksplit; ++kh) { re += pp[o_src[i] + kh * 128]; im += pp[o_src[i] + kh * 128 + 2]; }
+        reinterpret_cast<float2*>(tg_)[tid + i * nthr] = make_float2(re, im);
+      }
+      for (int o = tid + 2 * nthr; o < n_out; o += nthr) {
+        const int ja = o / rb, jb = o - ja * rb;
+        const int src = (((ja >> 3) * RBT + (jb >> 3)) * ksplit) * 128 + (4 * (ja & 7) + ((jb & 7) >> 1)) * 4 + (jb & 1);
+        float re = 0.f, im = 0.f;
+        for (int kh = 0; kh < ksplit; ++kh) { re += pp[src + kh * 128]; im += pp[src + kh * 128 + 2]; }
+        reinterpret_cast<float2*>(tg_)[o] = make_float2(re, im);
+      }
+    }
+    // ---- stage 1 of slab it ----
+    if (it < nmine) {
+      const uint32_t* xs = reinterpret_cast<const uint32_t*>(smem + (size_t)buf * G.buf_stride);
+      const uint32_t* xrow = xs + (size_t)(8 * warp + gq) * B;
+      float d[RBT][4];
+#pragma unroll
+      for (int jt = 0; jt < RBT; ++jt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) d[jt][i] = 0.f;
+      for (int ks = 0; ks < ks16; ++ks) {
+        const int c1_ = 32 * (ks >> 2) + 8 * t + (ks & 3), c2_ = c1_ + 4;
+        const uint32_t x1 = c1_ < B ? xrow[c1_] : 0u, x2 = c2_ < B ? xrow[c2_] : 0u;
+#pragma unroll
+        for (int jt = 0; jt < RBT; ++jt) {
+          const uint4 h = u1tab[((ks * RBT + jt) * 2 + 0) * 32 + lane], l = u1tab[((ks * RBT + jt) * 2 + 1) * 32 + lane];
+          mma_f16(d[jt], h.x, h.y, h.z, h.w, x1, x2);
+          mma_f16(d[jt], l.x, l.y, l.z, l.w, x1, x2);
+        }
+      }
+      // d0 = Yre[a][jb], d1 = Yre[a+1][jb], d2 = Yim[a][jb], d3 = Yim[a+1][jb], a = 8 warp + 2t, jb = 8 jt + gq
+      cf* ys = ysb + (size_t)(it & 1) * A * ldy;
+#pragma unroll
+      for (int jt = 0; jt < RBT; ++jt) {
+        ys[(8 * warp + 2 * t) * ldy + 8 * jt + gq] = make_float2(d[jt][0], d[jt][2]);
+        ys[(8 * warp + 2 * t + 1) * ldy + 8 * jt + gq] = make_float2(d[jt][1], d[jt][3]);
+      }
+    }
+    // ---- stage 2 of slab it-1 ----
+    if (it >= 1 && it <= nmine) {
+      const cf* ys = ysb + (size_t)((it - 1) & 1) * A * ldy;
+      float* pw = part + (size_t)(it & 1) * units * 128;
+      const int steps = (A / 4) / ksplit;
+      for (int unit = warp; unit < units; unit += nwarps) {
+        const int tile = unit / ksplit, kh = unit - tile * ksplit, mt = tile / RBT, nt = tile - mt * RBT;
+        float tot[4] = {0.f, 0.f, 0.f, 0.f}, acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int q = 0; q < steps; ++q) {
+          const int a = 4 * (kh * steps + q) + t;
+          const cf y = ys[a * ldy + 8 * nt + gq], u = uas[a * ldu + 8 * mt + gq];
+          float yh0, yl0, yh1, yl1, urh, url, uih, uil;
+          split_tf32(y.x, yh0, yl0); split_tf32(y.y, yh1, yl1);
+          split_tf32(u.x, urh, url); split_tf32(u.y, uih, uil);
+          // rows (re, ja): (ur | ui); rows (im, ja): (-ui | ur)
+          mma_tf32(acc, urh, -uih, uih, urh, yh0, yh1);
+          mma_tf32(acc, url, -uil, uil, url, yh0, yh1);
+          mma_tf32(acc, urh, -uih, uih, urh, yl0, yl1);
+          if ((q & 7) == 7) {      // the tensor core's accumulator adds truncate: keep its chains short
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { tot[i] += acc[i]; acc[i] = 0.f; }
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) tot[i] += acc[i];
+        *reinterpret_cast<float4*>(pw + (size_t)unit * 128 + lane * 4) = make_float4(tot[0], tot[1], tot[2], tot[3]);
+      }
+    }
+    if (it < nmine) {
+      pbuf = buf;
+      if (++buf == nbuf) { buf = 0; phase ^= 1; }
+    }
+  }
+}
+
+}  // namespace tg

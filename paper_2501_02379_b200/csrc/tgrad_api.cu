@@ -16,6 +16,7 @@
 #include "select.cuh"
 #include "tail.cuh"
 #include "tail_tc.cuh"
+#include "tail_h.cuh"
 
 using namespace tg;
 
@@ -51,6 +52,10 @@ struct TailPlan {
   int rat, ks, ntw, pjw, back_ns;
   TcGeom gproj, gback;
   int grid_proj, grid_back;
+  // half-storage compression kernel (fp16 MMA)
+  bool th;
+  int h_rat, h_rbt, grid_h;
+  TailHGeom gh;
 };
 
 tgrad_status validate(const tgrad_config* c) {
@@ -221,6 +226,23 @@ template <int RAT>
 tgrad_status tc_back_op(int op, const TailPlan& tp, void* w, const TailTcParams& P, cudaStream_t st) {
   return tp.back_ns == 2 ? tc_back_op2<RAT, 2>(op, tp, w, P, st) : tc_back_op2<RAT, 1>(op, tp, w, P, st);
 }
+template <int RAT, int RBT>
+tgrad_status th_proj_op(int op, const TailPlan& tp, const void* g, const TailHParams& P, cudaStream_t st) {
+  if (op == 0) {
+    return cudaFuncSetAttribute(proj_tail_h_kernel<RAT, RBT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)tp.gh.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
+  }
+  proj_tail_h_kernel<RAT, RBT><<<tp.grid_h, 32 * tp.gh.nwarps, tp.gh.total, st>>>(g, P);
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
+}
+tgrad_status th_dispatch(int op, const TailPlan& tp, const void* g, const TailHParams& P, cudaStream_t st) {
+#define TG_HCASE(RAT_, RBT_) if (tp.h_rat == RAT_ && tp.h_rbt == RBT_) return th_proj_op<RAT_, RBT_>(op, tp, g, P, st);
+  TG_HCASE(1, 1) TG_HCASE(2, 1) TG_HCASE(3, 1) TG_HCASE(4, 1) TG_HCASE(1, 2) TG_HCASE(2, 2) TG_HCASE(3, 2) TG_HCASE(4, 2)
+#undef TG_HCASE
+  return TGRAD_ERR_UNSUPPORTED;
+}
+
 // op: 0 = set attributes (both kernels), 1 = proj, 2 = back
 tgrad_status tc_dispatch(int op, const TailPlan& tp, void* ptr, const TailTcParams& P, cudaStream_t st) {
 #define TG_TCASE(RAT_)                                                                           \
@@ -280,6 +302,14 @@ tgrad_status plan_tail(tgrad_state* s) {
       TailTcParams dm; memset(&dm, 0, sizeof(dm));
       if (tc_dispatch(0, tp, nullptr, dm, 0) == TGRAD_OK) tp.tc = true;
     }
+  }
+  // half storage: compression with fp16 MMAs on the stored values
+  tp.th = false;
+  if (c.wg_dtype == TGRAD_C32H && tail_h_geom(A, B, ra, rb, tp.gh)) {
+    tp.h_rat = (ra + 7) / 8; tp.h_rbt = (rb + 7) / 8;
+    tp.grid_h = (int)(S < (uint64_t)s->sm_count ? S : (uint64_t)s->sm_count);
+    TailHParams dm; memset(&dm, 0, sizeof(dm));
+    if (th_dispatch(0, tp, nullptr, dm, 0) == TGRAD_OK) tp.th = true;
   }
   return TGRAD_OK;
 }
@@ -461,6 +491,9 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   if (s->tail.tc) {
     mp.p = p; mp.g = s->tail.gproj;
     TG_TRY(tc_dispatch(1, s->tail, d_grad, mp, st));
+  } else if (s->tail.th) {
+    TailHParams hp; hp.p = p; hp.g = s->tail.gh; hp.flags = mp.flags;
+    TG_TRY(th_dispatch(1, s->tail, d_grad, hp, st));
   } else {
     TG_TRY(tail_any(s, 1, d_grad, p, st));
   }
