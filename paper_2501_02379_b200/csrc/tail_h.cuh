@@ -280,4 +280,221 @@ __global__ void __launch_bounds__(512, 1) proj_tail_h_kernel(const void* __restr
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Reconstruction of the two trailing modes (half storage), fused with the weight update and the sparse add.
+// Two warps share a tile of 16 rows of the slab (each takes half of the column tiles); the products are the
+// split-TF32 ones of back_tail_tc_kernel, with the Ua and Ub fragments in shared-memory tables.  The slab
+// stays fp16 in shared memory: the dense update is rounded to fp16 when it is written back there, the
+// sparse term is then added by one thread per entry and rounded again (the two roundings the oracle makes),
+// and one bulk copy stores the slab.
+// ---------------------------------------------------------------------------------------------
+struct TailHBGeom {
+  int nwarps, nbuf, nbt, ks2;
+  uint32_t slab_bytes, buf_stride;
+  uint32_t off_ub, off_ua, off_bar, total;
+};
+__host__ inline bool tail_hb_geom(int A, int B, int ra, int rb, TailHBGeom& g) {
+  if (A % 16 || A < 16 || A > 128) return false;
+  const int rat = (ra + 7) / 8, rbt = (rb + 7) / 8;
+  if (rat > 4 || rbt > 2) return false;
+  g.nwarps = 2 * (A / 16);
+  g.nbt = tc_ksteps(B);
+  g.ks2 = 2 * rat;
+  g.slab_bytes = (uint32_t)A * B * 4;
+  if (g.slab_bytes % 16) return false;
+  g.buf_stride = (g.slab_bytes + 127) & ~127u;
+  const uint32_t ub = (uint32_t)g.nbt * rbt * 2 * 32 * 16, ua = (uint32_t)(A / 16) * g.ks2 * 2 * 32 * 16;
+  g.nbuf = 3;
+  g.off_ub = 3 * g.buf_stride;
+  g.off_ua = g.off_ub + ub;
+  g.off_bar = g.off_ua + ua;
+  g.total = g.off_bar + 256;
+  return g.total <= 227u * 1024u;
+}
+struct TailHBParams {
+  TailParams p;
+  TailHBGeom g;
+  int* flags;
+};
+
+template <int RAT, int RBT>
+__global__ void __launch_bounds__(512, 1) back_tail_h_kernel(void* __restrict__ w, TailHBParams P) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const TailParams& p = P.p;
+  const TailHBGeom& G = P.g;
+  const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t = lane & 3;
+  const int A = p.A, B = p.B, ra = p.ra, rb = p.rb, nbuf = G.nbuf, nbt = G.nbt;
+  constexpr int KS2 = 2 * RAT;
+  const uint32_t E = p.E, nslab = p.nslab, gstride = gridDim.x;
+  const int mtile = warp >> 1, am = 16 * mtile, r0 = am + gq, r1 = r0 + 8;
+  const int nbh = (nbt + 1) / 2, nb0 = (warp & 1) ? nbh : 0, nb1 = (warp & 1) ? nbt : nbh;   // this warp's column tiles
+  float4* ubf = reinterpret_cast<float4*>(smem + G.off_ub);     // [nbt][RBT][2][32]
+  float4* uaf = reinterpret_cast<float4*>(smem + G.off_ua);     // [A/16][KS2][hi|lo][32]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + G.off_bar);
+  unsigned char* wb = static_cast<unsigned char*>(w);
+
+  // Ub as stage-2 operand fragments (see back_tail_tc_kernel): per column tile, jb tile and lane
+  for (int idx = tid; idx < nbt * RBT * 32; idx += nthr) {
+    const int nb = idx / (RBT * 32), rem = idx - nb * (RBT * 32), jt = rem >> 5, ln = rem & 31, g_ = ln >> 2, t_ = ln & 3;
+    const int bq = 16 * (nb >> 2) + (nb & 3) + 4 * (g_ >> 1), jb = 8 * jt + 2 * t_;
+    const bool odd = g_ & 1;
+    cf va = (bq < B && jb < rb) ? p.Ub[bq * rb + jb] : make_float2(0.f, 0.f);
+    cf vb = (bq < B && jb + 1 < rb) ? p.Ub[bq * rb + jb + 1] : make_float2(0.f, 0.f);
+    cf ah, al, bh, bl;
+    split_tf32(va.x, ah.x, al.x); split_tf32(va.y, ah.y, al.y);
+    split_tf32(vb.x, bh.x, bl.x); split_tf32(vb.y, bh.y, bl.y);
+    ubf[((nb * RBT + jt) * 2 + 0) * 32 + ln] = odd ? make_float4(ah.y, bh.y, al.y, bl.y) : make_float4(ah.x, bh.x, al.x, bl.x);
+    ubf[((nb * RBT + jt) * 2 + 1) * 32 + ln] = odd ? make_float4(ah.x, bh.x, al.x, bl.x) : make_float4(-ah.y, -bh.y, -al.y, -bl.y);
+  }
+  // Ua as stage-1 operand fragments: rows am + g and am + g + 8, ja = 4 ks + t: (u0.x, u1.x, u0.y, u1.y) hi, then lo
+  for (int idx = tid; idx < (A / 16) * KS2 * 32; idx += nthr) {
+    const int mt = idx / (KS2 * 32), rem = idx - mt * (KS2 * 32), ks = rem >> 5, ln = rem & 31;
+    const int ja = 4 * ks + (ln & 3), q0 = 16 * mt + (ln >> 2), q1 = q0 + 8;
+    cf v0 = (ja < ra) ? p.Ua[q0 * ra + ja] : make_float2(0.f, 0.f);
+    cf v1 = (ja < ra) ? p.Ua[q1 * ra + ja] : make_float2(0.f, 0.f);
+    cf h0, l0, h1, l1;
+    split_tf32(v0.x, h0.x, l0.x); split_tf32(v0.y, h0.y, l0.y);
+    split_tf32(v1.x, h1.x, l1.x); split_tf32(v1.y, h1.y, l1.y);
+    uaf[((mt * KS2 + ks) * 2 + 0) * 32 + ln] = make_float4(h0.x, h1.x, h0.y, h1.y);
+    uaf[((mt * KS2 + ks) * 2 + 1) * 32 + ln] = make_float4(l0.x, l1.x, l0.y, l1.y);
+  }
+  if (tid == 0) {
+    for (int i = 0; i < nbuf; ++i) mbar_init(&bars[i], 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  const uint32_t nmine = (nslab > blockIdx.x) ? (nslab - blockIdx.x + gstride - 1) / gstride : 0;
+  if (tid == 0 && nmine > 0) {
+    mbar_expect_tx(&bars[0], G.slab_bytes);
+    bulk_g2s(smem, wb + (size_t)blockIdx.x * G.slab_bytes, G.slab_bytes, &bars[0]);
+  }
+  const bool sparse = p.k > 0;
+  auto bounds = [&](uint32_t s, int& x0, int& x1) {
+    x0 = 0; x1 = 0;
+    if (s < nslab) { x0 = (int)p.slab_ptr[s]; x1 = (int)p.slab_ptr[s + 1]; }
+  };
+  int b0 = 0, b1 = 0, n0 = 0, n1 = 0;
+  uint32_t pom = 0; cf pn = make_float2(0.f, 0.f);
+  if (sparse) {
+    bounds(blockIdx.x, b0, b1);
+    bounds(blockIdx.x + gstride, n0, n1);
+    if (b0 + tid < b1) { pom = p.omega[b0 + tid]; pn = p.n_s[b0 + tid]; }
+  }
+  const bool decay = p.decay != 1.0f;
+  uint32_t phase = 0;
+  int buf = 0, lbuf = 1;            // ring slot of this iteration and of the slab loaded one ahead
+  for (uint32_t it = 0; it < nmine; ++it) {
+    const uint32_t s = blockIdx.x + it * gstride;
+    if (tid == 0) bulk_wait_read<1>();          // the store of two iterations ago has read its buffer
+    // T' fragments for stage 1 (in flight while the slab arrives): T'[ja = 4 ks + t][jb = 8 jt + gq]
+    cf tv[KS2][RBT];
+    {
+      const cf* tin = p.t + (size_t)s * ra * rb;
+#pragma unroll
+      for (int ks = 0; ks < KS2; ++ks)
+#pragma unroll
+        for (int jt = 0; jt < RBT; ++jt) {
+          const int ja = 4 * ks + t, jb = 8 * jt + gq;
+          tv[ks][jt] = (ja < ra && jb < rb) ? __ldg(tin + (size_t)ja * rb + jb) : make_float2(0.f, 0.f);
+        }
+    }
+    const bool ok = mbar_wait_bounded(&bars[buf], phase);
+    if (__syncthreads_or(!ok)) {
+      if (tid == 0) { atomicOr(P.flags, 4); bulk_wait_all<0>(); }
+      return;
+    }
+    if (tid == 0 && it + 1 < nmine) {             // buffer lbuf was stored two iterations ago (read checked above)
+      mbar_expect_tx(&bars[lbuf], G.slab_bytes);
+      bulk_g2s(smem + (size_t)lbuf * G.buf_stride, wb + (size_t)(s + gstride) * G.slab_bytes, G.slab_bytes, &bars[lbuf]);
+    }
+    uint32_t* ws = reinterpret_cast<uint32_t*>(smem + (size_t)buf * G.buf_stride);     // half2 words [A][B]
+    {
+      // ---- stage 1: Y'[a][(c, jb)] for rows r0 and r1 ----
+      float d1[2][RBT][4];
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
+#pragma unroll
+        for (int jt = 0; jt < RBT; ++jt)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) d1[c][jt][i] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < KS2; ++ks) {
+        const float4 uh = uaf[((mtile * KS2 + ks) * 2 + 0) * 32 + lane], ul = uaf[((mtile * KS2 + ks) * 2 + 1) * 32 + lane];
+#pragma unroll
+        for (int jt = 0; jt < RBT; ++jt) {
+          float trh, trl, tih, til;
+          split_tf32(tv[ks][jt].x, trh, trl); split_tf32(tv[ks][jt].y, tih, til);
+          // A = (Ua[r0].re, Ua[r1].re, Ua[r0].im, Ua[r1].im);  re tile: B = (Tr, -Ti);  im tile: B = (Ti, Tr)
+          mma_tf32(d1[0][jt], uh.x, uh.y, uh.z, uh.w, trh, -tih);
+          mma_tf32(d1[0][jt], ul.x, ul.y, ul.z, ul.w, trh, -tih);
+          mma_tf32(d1[0][jt], uh.x, uh.y, uh.z, uh.w, trl, -til);
+          mma_tf32(d1[1][jt], uh.x, uh.y, uh.z, uh.w, tih, trh);
+          mma_tf32(d1[1][jt], ul.x, ul.y, ul.z, ul.w, tih, trh);
+          mma_tf32(d1[1][jt], uh.x, uh.y, uh.z, uh.w, til, trl);
+        }
+      }
+      float yh[2][RBT][4], yl[2][RBT][4];
+#pragma unroll
+      for (int c = 0; c < 2; ++c)
+#pragma unroll
+        for (int jt = 0; jt < RBT; ++jt)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) split_tf32(d1[c][jt][i], yh[c][jt][i], yl[c][jt][i]);
+      // ---- stage 2, one column tile at a time, applied to the slab right away ----
+      for (int nb = nb0; nb < nb1; ++nb) {
+        float dh[4] = {0.f, 0.f, 0.f, 0.f}, dl[4] = {0.f, 0.f, 0.f, 0.f}, dx[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int jt = 0; jt < RBT; ++jt) {
+          const float4 fr = ubf[((nb * RBT + jt) * 2 + 0) * 32 + lane], fi = ubf[((nb * RBT + jt) * 2 + 1) * 32 + lane];
+          mma_tf32(dh, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.x, fr.y);
+          mma_tf32(dl, yl[0][jt][0], yl[0][jt][2], yl[0][jt][1], yl[0][jt][3], fr.x, fr.y);
+          mma_tf32(dx, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.z, fr.w);
+          mma_tf32(dh, yh[1][jt][0], yh[1][jt][2], yh[1][jt][1], yh[1][jt][3], fi.x, fi.y);
+          mma_tf32(dl, yl[1][jt][0], yl[1][jt][2], yl[1][jt][1], yl[1][jt][3], fi.x, fi.y);
+          mma_tf32(dx, yh[1][jt][0], yh[1][jt][2], yh[1][jt][1], yh[1][jt][3], fi.z, fi.w);
+        }
+        // d0 + i d1 = D[r0][b], d2 + i d3 = D[r1][b] with b = 16 (nb>>2) + (nb&3) + 4 t
+        const int bo = 16 * (nb >> 2) + (nb & 3) + 4 * t;
+        if (bo < B) {
+          uint32_t* p0 = ws + (size_t)r0 * B + bo;
+          uint32_t* p1 = ws + (size_t)r1 * B + bo;
+          const uint32_t w0 = *p0, w1 = *p1;
+          float2 v0 = __half22float2(*reinterpret_cast<const __half2*>(&w0));
+          float2 v1 = __half22float2(*reinterpret_cast<const __half2*>(&w1));
+          if (decay) { v0.x *= p.decay; v0.y *= p.decay; v1.x *= p.decay; v1.y *= p.decay; }
+          v0.x = fmaf(-p.s_low, dh[0] + (dl[0] + dx[0]), v0.x); v0.y = fmaf(-p.s_low, dh[1] + (dl[1] + dx[1]), v0.y);
+          v1.x = fmaf(-p.s_low, dh[2] + (dl[2] + dx[2]), v1.x); v1.y = fmaf(-p.s_low, dh[3] + (dl[3] + dx[3]), v1.y);
+          *p0 = h2_bits(__floats2half2_rn(v0.x, v0.y));
+          *p1 = h2_bits(__floats2half2_rn(v1.x, v1.y));
+        }
+      }
+    }
+    __syncthreads();                                   // the dense update of the slab is complete (rounded to fp16)
+    // ---- scaled sparse add at Omega, one entry per thread, rounded again ----
+    if (sparse) {
+      const uint32_t base = s * E;
+      for (int j = b0 + tid, first = 1; j < b1; j += nthr, first = 0) {
+        const uint32_t loc = (first ? pom : p.omega[j]) - base;
+        const cf n = first ? pn : p.n_s[j];
+        const uint32_t wv = ws[loc];
+        float2 v = __half22float2(*reinterpret_cast<const __half2*>(&wv));
+        v.x = fmaf(-p.s_sparse, n.x, v.x); v.y = fmaf(-p.s_sparse, n.y, v.y);
+        ws[loc] = h2_bits(__floats2half2_rn(v.x, v.y));
+      }
+      b0 = n0; b1 = n1;
+      if (b0 + tid < b1) { pom = p.omega[b0 + tid]; pn = p.n_s[b0 + tid]; }
+      bounds(s + 2 * gstride, n0, n1);
+    }
+    fence_async_smem();                                // order the shared-memory writes before the bulk store reads them
+    __syncthreads();
+    if (tid == 0) {
+      bulk_s2g(wb + (size_t)s * G.slab_bytes, smem + (size_t)buf * G.buf_stride, G.slab_bytes);
+      bulk_commit();
+    }
+    if (++buf == nbuf) { buf = 0; phase ^= 1; }
+    if (++lbuf == nbuf) lbuf = 0;
+  }
+  if (tid == 0) bulk_wait_all<0>();   // stores complete before the block's shared memory goes away
+}
+
 }  // namespace tg

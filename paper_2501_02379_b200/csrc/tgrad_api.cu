@@ -53,9 +53,10 @@ struct TailPlan {
   TcGeom gproj, gback;
   int grid_proj, grid_back;
   // half-storage compression kernel (fp16 MMA)
-  bool th;
-  int h_rat, h_rbt, grid_h;
+  bool th, thb;
+  int h_rat, h_rbt, grid_h, grid_hb;
   TailHGeom gh;
+  TailHBGeom ghb;
 };
 
 tgrad_status validate(const tgrad_config* c) {
@@ -243,6 +244,23 @@ tgrad_status th_dispatch(int op, const TailPlan& tp, const void* g, const TailHP
   return TGRAD_ERR_UNSUPPORTED;
 }
 
+template <int RAT, int RBT>
+tgrad_status th_back_op(int op, const TailPlan& tp, void* w, const TailHBParams& P, cudaStream_t st) {
+  if (op == 0) {
+    return cudaFuncSetAttribute(back_tail_h_kernel<RAT, RBT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)tp.ghb.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
+  }
+  back_tail_h_kernel<RAT, RBT><<<tp.grid_hb, 32 * tp.ghb.nwarps, tp.ghb.total, st>>>(w, P);
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
+}
+tgrad_status thb_dispatch(int op, const TailPlan& tp, void* w, const TailHBParams& P, cudaStream_t st) {
+#define TG_HCASE(RAT_, RBT_) if (tp.h_rat == RAT_ && tp.h_rbt == RBT_) return th_back_op<RAT_, RBT_>(op, tp, w, P, st);
+  TG_HCASE(1, 1) TG_HCASE(2, 1) TG_HCASE(3, 1) TG_HCASE(4, 1) TG_HCASE(1, 2) TG_HCASE(2, 2) TG_HCASE(3, 2) TG_HCASE(4, 2)
+#undef TG_HCASE
+  return TGRAD_ERR_UNSUPPORTED;
+}
+
 // op: 0 = set attributes (both kernels), 1 = proj, 2 = back
 tgrad_status tc_dispatch(int op, const TailPlan& tp, void* ptr, const TailTcParams& P, cudaStream_t st) {
 #define TG_TCASE(RAT_)                                                                           \
@@ -310,6 +328,13 @@ tgrad_status plan_tail(tgrad_state* s) {
     tp.grid_h = (int)(S < (uint64_t)s->sm_count ? S : (uint64_t)s->sm_count);
     TailHParams dm; memset(&dm, 0, sizeof(dm));
     if (th_dispatch(0, tp, nullptr, dm, 0) == TGRAD_OK) tp.th = true;
+  }
+  tp.thb = false;
+  if (c.wg_dtype == TGRAD_C32H && tail_hb_geom(A, B, ra, rb, tp.ghb)) {
+    tp.h_rat = (ra + 7) / 8; tp.h_rbt = (rb + 7) / 8;
+    tp.grid_hb = (int)(S < (uint64_t)s->sm_count ? S : (uint64_t)s->sm_count);
+    TailHBParams dm; memset(&dm, 0, sizeof(dm));
+    if (thb_dispatch(0, tp, nullptr, dm, 0) == TGRAD_OK) tp.thb = true;
   }
   return TGRAD_OK;
 }
@@ -555,6 +580,9 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   if (s->tail.tc) {
     mp.p = p; mp.g = s->tail.gback;
     TG_TRY(tc_dispatch(2, s->tail, d_weight, mp, st));
+  } else if (s->tail.thb) {
+    TailHBParams hp; hp.p = p; hp.g = s->tail.ghb; hp.flags = mp.flags;
+    TG_TRY(thb_dispatch(2, s->tail, d_weight, hp, st));
   } else {
     TG_TRY(tail_any(s, 2, d_weight, p, st));
   }

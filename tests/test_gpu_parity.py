@@ -74,13 +74,15 @@ def test_topk_multi_block_ragged():
         assert np.array_equal(st.export(B.WHAT_OMEGA), orc.sparse_indices_topk(g, k)), k
 
 
-def test_half_storage_small():
+@pytest.mark.parametrize("name", ["ragged4", "odd32", "odd4", "small3"])
+def test_half_storage_small(name):
+    # fp16-stored W and G: the general kernels (24-row slabs) and the fp16-MMA kernels (8k / 16k-row slabs)
     import dataclasses
-    wl = dataclasses.replace(synth.WORKLOADS["ragged4"], half_storage=True)
+    wl = dataclasses.replace(synth.WORKLOADS[name], half_storage=True)
     p = Pair(wl)
     for t in range(wl.T + 2):
         p.step(t)
-    print("half", p.report)
+    print("half", name, p.report)
 
 
 def test_auto_refresh_matches_explicit():
