@@ -83,6 +83,13 @@ __device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
   lo = x - hi;
 }
 
+// The same with hi truncated instead of rounded (one integer op less).  lo = x - hi is still exact; it is
+// at most 2^-10 |x| instead of 2^-11 |x|, so what the tensor core drops of it is at most 2^-20 |x|.
+__device__ __forceinline__ void split_tf32_trunc(float x, float& hi, float& lo) {
+  hi = __uint_as_float(__float_as_uint(x) & 0xffffe000u);
+  lo = x - hi;
+}
+
 // one group of slabs -> ring buffer `buf`
 __device__ __forceinline__ void tc_issue_load(const unsigned char* gbase, unsigned char* smem, const TcGeom& G,
                                               uint64_t* bars, uint32_t u, int buf, uint32_t nslab) {
@@ -304,7 +311,7 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW == 1 ?
         for (int nt = 0; nt < NTW; ++nt) {
           float2 x = (f < twoB) ? *reinterpret_cast<const float2*>(xrow + (size_t)(8 * nt * tw) * twoB + f) : make_float2(0.f, 0.f);
           float xh0, xl0, xh1, xl1;
-          split_tf32(x.x, xh0, xl0); split_tf32(x.y, xh1, xl1);
+          split_tf32_trunc(x.x, xh0, xl0); split_tf32_trunc(x.y, xh1, xl1);      // the streamed operand: cheapest split
           // A = (ur, -ui, ui, ur): rows (re, jb) and (im, jb) of W1
           mma_tf32(dh[nt], uf.x, nhy, uf.y, uf.x, xh0, xh1);
           mma_tf32(dl[nt], uf.z, nly, uf.w, uf.z, xh0, xh1);
