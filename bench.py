@@ -28,9 +28,11 @@ from paper_2501_02379_b200 import replicas, synth  # noqa: E402
 METRIC = "tgrad_step effective HBM GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# captures summarised under profiles/ (bytes); None where no capture exists for the workload.
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the two streaming kernels, from the ncu
+# capture summarised in profiles/cfg3_step_and_refresh_block_cooperative.md (bytes); None where no
+# capture exists for the workload.  (back_tail: 304.1 MB read + 218.0 MB written -- the rest of the
+# 277 MB it writes is still in L2 when the kernel ends.)
+NCU_TRAFFIC_BYTES = {("cfg3", "proj_tail"): 280.4e6 + 19.6e6, ("cfg3", "back_tail"): 304.1e6 + 218.0e6}
 
 
 def step_bytes(wl: synth.Workload) -> int:
@@ -256,22 +258,25 @@ def run_ours(args, wl):
     ms = replicas.max_over_ranks(ms, dist, "cuda")
     flags = [s.query_status()[0] for s in states]
 
-    # ---- per-stage device times of non-refresh steps (events on the launching stream) ----
+    # ---- non-refresh steps alone, then their per-stage device times (events on the launching stream) ----
     st0 = states[0]
-    st0.set_stage_timing(True)
     while t % wl.T == 0:
         one_step(t); t += 1
-    n_stage_steps = min(60, max(1, wl.T - (t % wl.T) - 1))
+    n_stage_steps = min(30, max(1, (wl.T - (t % wl.T) - 1) // 2))
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2.record(stream)
     for _ in range(n_stage_steps):
-        states[0].step(weights[0], grads[0][t % ring], stream)
+        states[0].step(weights[0], grads[0][t % ring], stream); t += 1
     e3.record(stream)
+    torch.cuda.synchronize()
+    nonrefresh_ms = e2.elapsed_time(e3) / n_stage_steps
+    st0.set_stage_timing(True)                       # the events between the stages add a few microseconds per stage
+    for _ in range(n_stage_steps):
+        states[0].step(weights[0], grads[0][t % ring], stream); t += 1
     torch.cuda.synchronize()
     stage_ms, n_rec = st0.stage_times(stream)
     st0.set_stage_timing(False)
     # the counter of tensor 0 ran ahead of the others; irrelevant from here on
-    nonrefresh_ms = e2.elapsed_time(e3) / n_stage_steps
     stage_us = {name: 1e3 * v / max(1, n_rec) for name, v in zip(B.STAGE_NAMES, stage_ms)}
 
     # ---- one refresh step timed alone ----

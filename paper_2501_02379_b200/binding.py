@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libtgrad.so")
 MAX_NDIM = 8
 NUM_STAGES = 5
-STAGE_NAMES = ["proj_tail", "proj_chain", "adam_core", "back_chain", "back_tail"]
+STAGE_NAMES = ["proj_tail", "proj_chain", "mode1_adam", "back_chain", "back_tail"]
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BUFFER_TOO_SMALL, ERR_CUDA, ERR_NO_CONVERGE, ERR_NONFINITE, ERR_BAD_STATE = range(8)
 ERR_TOO_LARGE = 8
