@@ -181,9 +181,11 @@ __global__ void __launch_bounds__(JAC_THREADS) jacobi_kernel(JacobiParams P) {
 // (3) jacobi_factors_kernel, one block per mode: eigenvalue ranks, canonical phase, U.
 // ---------------------------------------------------------------------------------------------
 constexpr int JAC_SMEM_MAX_N = 160;      // 160^2 complex64 = 200 KB of shared memory
+constexpr int JAC_FAST_MAX_N = 256;      // up to here the same kernel runs with the matrix in global memory (L2)
 
 struct JacobiFastMode {
   const cf* A;       // n x n input (left untouched)
+  cf* work;          // n x (n | 1) working copy in global memory, used when n > JAC_SMEM_MAX_N
   float4* log;       // [sweeps][m-1][m/2] rotations
   float* lam;        // out: n eigenvalues (unsorted)
   cf* V;             // out: n x n eigenvectors in columns (row-major)
@@ -195,6 +197,7 @@ struct JacobiFastMode {
 struct JacobiFastParams {
   JacobiFastMode mode[8];
   int nmodes, total_rows;
+  int row_stride;    // jacobi_vectors_kernel: complex entries per warp row buffer (>= largest n)
   int max_sweeps;
   float tol;
   int* flags;        // flags[0] sticky bits, flags[1 + mode] sweeps used
@@ -206,9 +209,9 @@ __host__ __device__ inline size_t jac_log_entries(int n, int max_sweeps) {
   return (size_t)max_sweeps * (m - 1) * (m / 2);
 }
 __host__ __device__ inline size_t jac_a_bytes(int n) { return ((size_t)n * (n | 1) * sizeof(cf) + 15) & ~(size_t)15; }
-__host__ __device__ inline size_t jac_sweeps_smem(int n) {
+__host__ __device__ inline size_t jac_sweeps_smem(int n, bool insmem = true) {
   const size_t m = (size_t)((n + 1) & ~1);
-  return jac_a_bytes(n) + (m / 2) * (sizeof(float4) + sizeof(float2) + sizeof(int2));
+  return (insmem ? jac_a_bytes(n) : 0) + (m / 2) * (sizeof(float4) + sizeof(float2) + sizeof(int2));
 }
 
 __device__ __forceinline__ void jac_pair(int m, int stage, int tb, int& p, int& q) {
@@ -259,13 +262,16 @@ __device__ __forceinline__ void jac_put(cf* A, int ld, int i, int j, cf v) {
   else A[(size_t)j * ld + i] = make_float2(v.x, -v.y);
 }
 
+// INSMEM: the matrix is in shared memory (n <= JAC_SMEM_MAX_N); otherwise in the mode's global work buffer, where
+// a block's own writes are visible to it after a barrier.
+template <bool INSMEM>
 __global__ void __launch_bounds__(JAC_THREADS) jacobi_sweeps_kernel(JacobiFastParams P) {
   extern __shared__ __align__(16) unsigned char jsm[];
   const JacobiFastMode md = P.mode[blockIdx.x];
   const int n = md.n;
   const int m = (n + 1) & ~1, half = m >> 1;
-  cf* A = reinterpret_cast<cf*>(jsm);                                  // [n][n | 1], upper triangle live
-  float4* rotc = reinterpret_cast<float4*>(jsm + jac_a_bytes(n));      // [half] (c, s, g.x, g.y); 16-byte aligned
+  cf* A = INSMEM ? reinterpret_cast<cf*>(jsm) : md.work;               // [n][n | 1], upper triangle live
+  float4* rotc = reinterpret_cast<float4*>(jsm + (INSMEM ? jac_a_bytes(n) : 0));      // [half] (c, s, g.x, g.y); 16-byte aligned
   float2* rotd = reinterpret_cast<float2*>(rotc + half);               // [half] new diagonal entries of the pair
   int2* rotp = reinterpret_cast<int2*>(rotd + half);                   // [half] (p, q); p < 0: no rotation, p = -1 - p
   __shared__ float red[32];
@@ -389,8 +395,11 @@ __global__ void __launch_bounds__(JAC_THREADS) jacobi_sweeps_kernel(JacobiFastPa
   for (int i = tid; i < n; i += nt) md.lam[i] = A[(size_t)i * ld + i].x;
 }
 
+// NP = pairs per lane (>= n/64), D = stages of the log kept in flight
+template <int NP, int D>
 __global__ void __launch_bounds__(256) jacobi_vectors_kernel(JacobiFastParams P) {
-  __shared__ cf rows[8][JAC_SMEM_MAX_N];
+  extern __shared__ __align__(16) unsigned char jvs[];
+  cf* rows = reinterpret_cast<cf*>(jvs);                    // [8][row_stride]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int gw = blockIdx.x * 8 + warp;
   if (gw >= P.total_rows) return;
@@ -400,18 +409,17 @@ __global__ void __launch_bounds__(256) jacobi_vectors_kernel(JacobiFastParams P)
   const int n = md.n, i_row = gw - md.row0;
   const int m = (n + 1) & ~1, half = m >> 1;
   const int sweeps = P.flags[1 + md.index];
-  cf* row = rows[warp];
+  cf* row = rows + (size_t)warp * P.row_stride;
   for (int j = lane; j < n; j += 32) row[j] = make_float2(j == i_row ? 1.f : 0.f, 0.f);
   __syncwarp();
-  // the log is replayed four stages at a time, the next four already in flight
-  constexpr int NP = (JAC_SMEM_MAX_N / 2 + 31) / 32;      // pairs per lane
+  // the log is replayed D stages at a time, the next D already in flight
   const float4* lg = md.log;
   const int nst = sweeps * (m - 1);
   const float4 ident = make_float4(1.f, 0.f, 1.f, 0.f);
-  float4 cur[4][NP], nxt[4][NP];
-  auto fetch = [&](float4 (&buf)[4][NP], int s0) {
+  float4 cur[D][NP], nxt[D][NP];
+  auto fetch = [&](float4 (&buf)[D][NP], int s0) {
 #pragma unroll
-    for (int d = 0; d < 4; ++d)
+    for (int d = 0; d < D; ++d)
 #pragma unroll
       for (int e = 0; e < NP; ++e) {
         const int tb = lane + 32 * e;
@@ -420,10 +428,10 @@ __global__ void __launch_bounds__(256) jacobi_vectors_kernel(JacobiFastParams P)
   };
   fetch(cur, 0);
   int stage = 0;
-  for (int s0 = 0; s0 < nst; s0 += 4) {
-    fetch(nxt, s0 + 4);
+  for (int s0 = 0; s0 < nst; s0 += D) {
+    fetch(nxt, s0 + D);
 #pragma unroll
-    for (int d = 0; d < 4; ++d) {
+    for (int d = 0; d < D; ++d) {
       if (s0 + d < nst) {
 #pragma unroll
         for (int e = 0; e < NP; ++e) {
@@ -442,7 +450,7 @@ __global__ void __launch_bounds__(256) jacobi_vectors_kernel(JacobiFastParams P)
       }
     }
 #pragma unroll
-    for (int d = 0; d < 4; ++d)
+    for (int d = 0; d < D; ++d)
 #pragma unroll
       for (int e = 0; e < NP; ++e) cur[d][e] = nxt[d][e];
   }
@@ -453,8 +461,8 @@ __global__ void __launch_bounds__(JAC_THREADS) jacobi_factors_kernel(JacobiFastP
   const JacobiFastMode md = P.mode[blockIdx.x];
   const int n = md.n, r = md.r;
   const cf* __restrict__ V = md.V;
-  __shared__ float lam[JAC_SMEM_MAX_N];
-  __shared__ int rank_of[JAC_SMEM_MAX_N];
+  __shared__ float lam[JAC_FAST_MAX_N];
+  __shared__ int rank_of[JAC_FAST_MAX_N];
   const int tid = threadIdx.x, nt = blockDim.x;
   for (int i = tid; i < n; i += nt) lam[i] = md.lam[i];
   __syncthreads();

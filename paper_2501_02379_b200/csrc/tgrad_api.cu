@@ -135,11 +135,11 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
   for (int n = 0; n < N; ++n) {
     size_t sq = (size_t)c->dims[n] * c->dims[n] * 8;
     L.w_gram[n] = o; o = align_up(o + sq);   // A_n, kept for inspection
-    L.w_jac[n] = o; o = align_up(o + sq);    // working copy the solver diagonalises
+    L.w_jac[n] = o; o = align_up(o + (size_t)c->dims[n] * (c->dims[n] | 1) * 8);    // working copy the solver diagonalises
     L.w_v[n] = o; o = align_up(o + sq);      // accumulated rotations
     const int sweeps = c->jacobi_max_sweeps > 0 ? c->jacobi_max_sweeps : 30;
     const size_t logb = jac_log_entries((int)c->dims[n], sweeps) * sizeof(float4);
-    L.jac_fast[n] = c->dims[n] <= JAC_SMEM_MAX_N && logb <= ((size_t)64 << 20);
+    L.jac_fast[n] = c->dims[n] <= JAC_FAST_MAX_N && logb <= ((size_t)64 << 20);
     L.w_log[n] = o; if (L.jac_fast[n]) o = align_up(o + logb);
     L.w_lam[n] = o; o = align_up(o + (size_t)c->dims[n] * 4);
     plan_gram(c, n, sm, L.gram_chunks[n], L.gram_cps[n], L.gram_splits[n]);
@@ -396,7 +396,6 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   JacobiParams jp; memset(&jp, 0, sizeof(jp));
   JacobiFastParams fp; memset(&fp, 0, sizeof(fp));
   int nslow = 0;
-  size_t fast_smem = 0;
   for (int m = 0; m < N; ++m) {
     uint64_t O = 1, C = 1;
     for (int q = 0; q < m; ++q) O *= c.dims[q];
@@ -417,14 +416,14 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
     if (L.jac_fast[m]) {
       JacobiFastMode& fm = fp.mode[fp.nmodes++];
       fm.A = A;
+      fm.work = reinterpret_cast<cf*>(s->dw + L.w_jac[m]);
       fm.log = reinterpret_cast<float4*>(s->dw + L.w_log[m]);
       fm.lam = reinterpret_cast<float*>(s->dw + L.w_lam[m]);
       fm.V = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
       fm.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
       fm.n = In; fm.r = c.ranks[m]; fm.index = m; fm.row0 = fp.total_rows;
       fp.total_rows += In;
-      const size_t sm = jac_sweeps_smem(In);
-      if (sm > fast_smem) fast_smem = sm;
+      if (In > fp.row_stride) fp.row_stride = In;
     } else {
       JacobiMode& jm = jp.mode[nslow];
       jp.index[nslow++] = m;
@@ -445,8 +444,22 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   }
   if (fp.nmodes) {
     fp.max_sweeps = max_sweeps; fp.tol = tol; fp.flags = flags;
-    jacobi_sweeps_kernel<<<fp.nmodes, JAC_THREADS, fast_smem, st>>>(fp); TG_LAUNCH_CHECK();
-    jacobi_vectors_kernel<<<(fp.total_rows + 7) / 8, 256, 0, st>>>(fp); TG_LAUNCH_CHECK();
+    // the sweeps: modes whose matrix fits in shared memory in one launch, the larger ones (matrix in L2) in another
+    JacobiFastParams fs = fp, fg = fp;
+    fs.nmodes = fg.nmodes = 0;
+    size_t smem_s = 0, smem_g = 0;
+    for (int i = 0; i < fp.nmodes; ++i) {
+      const int n = fp.mode[i].n;
+      if (n <= JAC_SMEM_MAX_N) { fs.mode[fs.nmodes++] = fp.mode[i]; const size_t b = jac_sweeps_smem(n, true); if (b > smem_s) smem_s = b; }
+      else { fg.mode[fg.nmodes++] = fp.mode[i]; const size_t b = jac_sweeps_smem(n, false); if (b > smem_g) smem_g = b; }
+    }
+    if (fg.nmodes) { jacobi_sweeps_kernel<false><<<fg.nmodes, JAC_THREADS, smem_g, st>>>(fg); TG_LAUNCH_CHECK(); }
+    if (fs.nmodes) { jacobi_sweeps_kernel<true><<<fs.nmodes, JAC_THREADS, smem_s, st>>>(fs); TG_LAUNCH_CHECK(); }
+    fp.row_stride = (fp.row_stride + 1) & ~1;
+    const size_t vsm = (size_t)8 * fp.row_stride * sizeof(cf);
+    if (fp.row_stride <= 192) jacobi_vectors_kernel<3, 4><<<(fp.total_rows + 7) / 8, 256, vsm, st>>>(fp);
+    else jacobi_vectors_kernel<4, 2><<<(fp.total_rows + 7) / 8, 256, vsm, st>>>(fp);
+    TG_LAUNCH_CHECK();
     jacobi_factors_kernel<<<fp.nmodes, JAC_THREADS, 0, st>>>(fp); TG_LAUNCH_CHECK();
   }
   s->have_subspace = true;
@@ -641,7 +654,7 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
   if (cfg->dims[0] <= SW_MAX_I && cfg->ranks[0] <= SW_MAX_R &&
       cudaFuncSetAttribute(core_sandwich_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)sandwich_smem(SW_MAX_I, SW_MAX_R)) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
-  if (cudaFuncSetAttribute(jacobi_sweeps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (cudaFuncSetAttribute(jacobi_sweeps_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)jac_sweeps_smem(JAC_SMEM_MAX_N)) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   // Algorithm 1 initialisation: zero moments (and flags, Omega, factors for determinism)
