@@ -38,9 +38,14 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
   const int ta = blockIdx.x / T, tb = blockIdx.x % T;
   if (ta > tb) return;
   extern __shared__ __align__(16) unsigned char gsm[];
-  typedef cf Tile[GR_T][GR_LD];
+  // tiles hold the entries as they are stored (fp32 pairs, or fp16 pairs in one word): fp16 values are exact
+  // TF32 operands, so half storage needs neither rounding nor the split products
+  typedef typename S::elem Elem;
+  typedef Elem Tile[GR_T][GR_LD];
   Tile* XA = reinterpret_cast<Tile*>(gsm);            // [2]
   Tile* XBs = XA + 2;                                 // [2]
+  constexpr bool HALF = S::kBytes == 4;
+  constexpr bool DOSPLIT = SPLIT && !HALF;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t = lane & 3;
   const int wm = warp >> 1, wn = warp & 1;           // 2 x 2 warps of 32 x 32
   const int a0 = ta * GR_T, b0 = tb * GR_T;
@@ -82,8 +87,8 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
   // loads through registers with widening for fp16 storage
   auto load_chunk = [&](uint32_t ch, int st) {
     const uint32_t kk0 = ch * GR_KT;
-    cf (*xa)[GR_LD] = XA[st];
-    cf (*xb)[GR_LD] = XBs[st];
+    Elem (*xa)[GR_LD] = XA[st];
+    Elem (*xb)[GR_LD] = XBs[st];
     if (along_k) {
       const uint32_t kk = kk0 + ld_kc;
       const bool kok = kk < K32;
@@ -93,12 +98,12 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
       for (int i = 0; i < GR_T / (GR_THREADS / GR_KT); ++i) {
         const int row = ld_row + i * (GR_THREADS / GR_KT);
         const bool va = kok && a0 + row < In, vb = kok && b0 + row < In;
-        if (S::kBytes == 8) {
+        if (!HALF) {
           cp_async8(&xa[row][ld_kc], va ? gb + (base + (size_t)(a0 + row) * C) * 8 : gb, va ? 8u : 0u);
           if (!diag) cp_async8(&xb[row][ld_kc], vb ? gb + (base + (size_t)(b0 + row) * C) * 8 : gb, vb ? 8u : 0u);
         } else {
-          xa[row][ld_kc] = va ? S::load(g, base + (size_t)(a0 + row) * C) : make_float2(0.f, 0.f);
-          if (!diag) xb[row][ld_kc] = vb ? S::load(g, base + (size_t)(b0 + row) * C) : make_float2(0.f, 0.f);
+          cp_async4(&xa[row][ld_kc], va ? gb + (base + (size_t)(a0 + row) * C) * 4 : gb, va ? 4u : 0u);
+          if (!diag) cp_async4(&xb[row][ld_kc], vb ? gb + (base + (size_t)(b0 + row) * C) * 4 : gb, vb ? 4u : 0u);
         }
       }
     } else {
@@ -107,12 +112,12 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
         const int kc = ld_k2 + i * (GR_THREADS / GR_T);
         const uint32_t kk = kk0 + kc;
         const bool va = kk < K32 && a0 + ld_row < In, vb = kk < K32 && b0 + ld_row < In;
-        if (S::kBytes == 8) {
+        if (!HALF) {
           cp_async8(&xa[ld_row][kc], va ? gb + ((size_t)kk * In + a0 + ld_row) * 8 : gb, va ? 8u : 0u);
           if (!diag) cp_async8(&xb[ld_row][kc], vb ? gb + ((size_t)kk * In + b0 + ld_row) * 8 : gb, vb ? 8u : 0u);
         } else {
-          xa[ld_row][kc] = va ? S::load(g, (size_t)kk * In + a0 + ld_row) : make_float2(0.f, 0.f);
-          if (!diag) xb[ld_row][kc] = vb ? S::load(g, (size_t)kk * In + b0 + ld_row) : make_float2(0.f, 0.f);
+          cp_async4(&xa[ld_row][kc], va ? gb + ((size_t)kk * In + a0 + ld_row) * 4 : gb, va ? 4u : 0u);
+          if (!diag) cp_async4(&xb[ld_row][kc], vb ? gb + ((size_t)kk * In + b0 + ld_row) * 4 : gb, vb ? 4u : 0u);
         }
       }
     }
@@ -125,8 +130,11 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
     cp_async_wait<0>();
     __syncthreads();                                   // chunk ch has landed; everyone is done with stage st^1
     if (ch + 1 < ch1) load_chunk(ch + 1, st ^ 1);
-    const cf (*Xa)[GR_LD] = XA[st];
-    const cf (*XB)[GR_LD] = diag ? XA[st] : XBs[st];
+    const Elem (*Xa)[GR_LD] = XA[st];
+    const Elem (*XB)[GR_LD] = diag ? XA[st] : XBs[st];
+    auto widen = [](const Elem& e) -> cf {
+      if constexpr (HALF) return __half22float2(e); else return e;
+    };
 #pragma unroll
     for (int ks = 0; ks < GR_KT / 4; ++ks) {
       const int kc = ks * 4 + t;
@@ -134,22 +142,23 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
       float ah[2][4], al[2][4];
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt) {
-        const cf x0 = Xa[wm * 32 + mt * 16 + gq][kc], x1 = Xa[wm * 32 + mt * 16 + gq + 8][kc];
-        ah[mt][0] = gr_tf32(x0.x); ah[mt][1] = gr_tf32(x1.x); ah[mt][2] = gr_tf32(x0.y); ah[mt][3] = gr_tf32(x1.y);
-        if (SPLIT) { al[mt][0] = x0.x - ah[mt][0]; al[mt][1] = x1.x - ah[mt][1]; al[mt][2] = x0.y - ah[mt][2]; al[mt][3] = x1.y - ah[mt][3]; }
+        const cf x0 = widen(Xa[wm * 32 + mt * 16 + gq][kc]), x1 = widen(Xa[wm * 32 + mt * 16 + gq + 8][kc]);
+        if (HALF) { ah[mt][0] = x0.x; ah[mt][1] = x1.x; ah[mt][2] = x0.y; ah[mt][3] = x1.y; }
+        else { ah[mt][0] = gr_tf32(x0.x); ah[mt][1] = gr_tf32(x1.x); ah[mt][2] = gr_tf32(x0.y); ah[mt][3] = gr_tf32(x1.y); }
+        if (DOSPLIT) { al[mt][0] = x0.x - ah[mt][0]; al[mt][1] = x1.x - ah[mt][1]; al[mt][2] = x0.y - ah[mt][2]; al[mt][3] = x1.y - ah[mt][3]; }
       }
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt) {
         if (!nok[nt]) continue;
-        const cf y = XB[wn * 32 + nt * 8 + gq][kc];
-        const float yh0 = gr_tf32(y.x), yh1 = gr_tf32(y.y);
+        const cf y = widen(XB[wn * 32 + nt * 8 + gq][kc]);
+        const float yh0 = HALF ? y.x : gr_tf32(y.x), yh1 = HALF ? y.y : gr_tf32(y.y);
         const float yl0 = y.x - yh0, yl1 = y.y - yh1;
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
           if (!mok[mt]) continue;
           mma_tf32(are[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], yh0, yh1);
           mma_tf32(aim[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], -yh1, yh0);
-          if (SPLIT) {
+          if (DOSPLIT) {
             mma_tf32(are[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], yl0, yl1);
             mma_tf32(aim[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], -yl1, yl0);
             mma_tf32(are[mt][nt], al[mt][0], al[mt][1], al[mt][2], al[mt][3], yh0, yh1);
