@@ -538,7 +538,12 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   TG_MARK(1);
   // the chain on the small tensor: compression of modes N-2 .. 2, then mode 1 + Adam + mode 1 in one
   // launch (or three when the first mode is too large for it), then reconstruction of modes 2 .. N-2
-  const bool fused = c.dims[0] <= SW_MAX_I && c.ranks[0] <= SW_MAX_R;
+  // (the fused launch does its two products with fp32 FMAs: beyond 64 M complex multiply-adds per product the
+  //  tensor-core GEMM launches win even with the extra round trips)
+  uint64_t c_first = (uint64_t)ra * rb;
+  for (int q = 1; q <= N - 3; ++q) c_first *= c.ranks[q];
+  const bool fused = c.dims[0] <= SW_MAX_I && c.ranks[0] <= SW_MAX_R &&
+                     c_first * (uint64_t)c.dims[0] * (uint64_t)c.ranks[0] <= ((uint64_t)64 << 20);
   const cf* tprime;
   {
     cf* cur = bufa; cf* nxt = bufb;
