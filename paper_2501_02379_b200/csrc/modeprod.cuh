@@ -282,24 +282,29 @@ __global__ void __launch_bounds__(MT_THREADS) mode_product_tc_kernel(const cf* _
 //   N = AdamUpdate(core)                             (moments in place; core and N_L are kept)
 //   out[i][c] = sum_j U1[i][j] N[j][c]               (mode-1 product with U^(1), r_1 -> I_1)
 // A block takes 16 columns: X[:, block] is read into shared memory before anything is written, so
-// `out` may alias `X`.  Blocks past the last column block run the AdamUpdate of the sparse values.  The work is small (two skinny products); what this saves is two launches,
-// two round trips of the core through L2 and the idle SMs of three under-filled grids.
+// `out` may alias `X`.  Blocks past the last column block run the AdamUpdate of the sparse values.
 // ---------------------------------------------------------------------------------------------
 constexpr int SW_CB = 16, SW_THREADS = 256, SW_MAX_I = 256, SW_MAX_R = 64;
-__host__ __device__ inline size_t sandwich_smem(int I1, int r1) {
-  return ((size_t)I1 * (SW_CB + 1) + (size_t)r1 * (SW_CB + 1) + (size_t)I1 * r1) * sizeof(cf);
+// ---------------------------------------------------------------------------------------------
+// Both products run on the tensor cores (split TF32, fragment conventions of mode_product_tc_kernel): the
+// whole X[:, 16 columns] block and U1 sit in shared memory, so each product runs without intermediate barriers.
+// ---------------------------------------------------------------------------------------------
+constexpr int SWT_LDX = SW_CB + 4;      // row length of the X / core tiles: fragment loads hit distinct banks
+__host__ __device__ inline int swt_ldu(int r1) { return ((r1 + 7) & ~7) + 4; }
+__host__ __device__ inline size_t sandwich_tc_smem(int I1, int r1) {
+  const size_t I1p = (size_t)((I1 + 7) & ~7), r1p = (size_t)((r1 + 7) & ~7);
+  return (I1p * SWT_LDX + I1p * swt_ldu(r1) + r1p * SWT_LDX) * sizeof(cf);
 }
 
-__global__ void __launch_bounds__(SW_THREADS) core_sandwich_kernel(const cf* __restrict__ X, cf* __restrict__ out,
-                                                                   const cf* __restrict__ U1, cf* __restrict__ core,
-                                                                   cf* __restrict__ m_l, float* __restrict__ v_l,
-                                                                   cf* __restrict__ n_l, int I1, int r1, int C,
-                                                                   const cf* __restrict__ g_s, cf* __restrict__ m_s,
-                                                                   float* __restrict__ v_s, cf* __restrict__ n_s, uint32_t ks,
-                                                                   uint32_t nblk_core, AdamScalars a) {
+__global__ void __launch_bounds__(SW_THREADS) core_sandwich_tc_kernel(const cf* __restrict__ X, cf* __restrict__ out,
+                                                                      const cf* __restrict__ U1, cf* __restrict__ core,
+                                                                      cf* __restrict__ m_l, float* __restrict__ v_l,
+                                                                      cf* __restrict__ n_l, int I1, int r1, int C,
+                                                                      const cf* __restrict__ g_s, cf* __restrict__ m_s,
+                                                                      float* __restrict__ v_s, cf* __restrict__ n_s, uint32_t ks,
+                                                                      uint32_t nblk_core, AdamScalars a) {
   extern __shared__ __align__(16) unsigned char swm[];
   if (blockIdx.x >= nblk_core) {
-    // trailing blocks: AdamUpdate of the ks gathered sparse values (independent of the core)
     const uint32_t i = (blockIdx.x - nblk_core) * SW_THREADS + threadIdx.x;
     if (i < ks) {
       cf m = m_s[i]; float v = v_s[i];
@@ -308,58 +313,83 @@ __global__ void __launch_bounds__(SW_THREADS) core_sandwich_kernel(const cf* __r
     }
     return;
   }
-  constexpr int LD = SW_CB + 1, RP = SW_THREADS / SW_CB;                  // padded row, rows per pass
-  cf* Xs = reinterpret_cast<cf*>(swm);                                    // [I1][LD]
-  cf* Ns = Xs + (size_t)I1 * LD;                                          // [r1][LD]
-  cf* Us = Ns + (size_t)r1 * LD;                                          // [I1][r1]
-  const int tid = threadIdx.x, cc = tid % SW_CB, r0 = tid / SW_CB;
-  const int c = blockIdx.x * SW_CB + cc;
-  const bool cok = c < C;
-  for (int i = r0; i < I1; i += RP) Xs[i * LD + cc] = cok ? X[(size_t)i * C + c] : make_float2(0.f, 0.f);
-  for (int i = tid; i < I1 * r1; i += SW_THREADS) Us[i] = U1[i];
-  __syncthreads();
-  // core rows j and j + RP together: one load of x serves both
-  for (int j = r0; j < r1; j += 2 * RP) {
-    const bool two = j + RP < r1;
-    const int j2 = two ? j + RP : j;
-    cf acc0 = make_float2(0.f, 0.f), acc1 = acc0;
-#pragma unroll 4
-    for (int i = 0; i < I1; ++i) {
-      const cf x = Xs[i * LD + cc];
-      cfma_conj(acc0, x, Us[i * r1 + j]);                                 // x * conj(u)
-      cfma_conj(acc1, x, Us[i * r1 + j2]);
-    }
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      if (h == 1 && !two) break;
-      const int jj = h ? j2 : j;
-      const cf acc = h ? acc1 : acc0;
-      cf n = make_float2(0.f, 0.f);
-      if (cok) {
-        const size_t e = (size_t)jj * C + c;
-        cf m = m_l[e]; float v = v_l[e];
-        n = adam_apply(acc, m, v, a);
-        m_l[e] = m; v_l[e] = v; n_l[e] = n; core[e] = acc;
-      }
-      Ns[jj * LD + cc] = n;
-    }
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t = lane & 3;
+  const int I1p = (I1 + 7) & ~7, r1p = (r1 + 7) & ~7, ldu = swt_ldu(r1);
+  cf* Xs = reinterpret_cast<cf*>(swm);                 // [I1p][SWT_LDX]
+  cf* Us = Xs + (size_t)I1p * SWT_LDX;                 // [I1p][ldu], zero padded
+  cf* Cs = Us + (size_t)I1p * ldu;                     // [r1p][SWT_LDX]: the core block, then N
+  const int c0 = blockIdx.x * SW_CB;
+  for (int idx = tid; idx < I1p * SW_CB; idx += SW_THREADS) {
+    const int i = idx / SW_CB, cc = idx - i * SW_CB;
+    Xs[i * SWT_LDX + cc] = (i < I1 && c0 + cc < C) ? X[(size_t)i * C + c0 + cc] : make_float2(0.f, 0.f);
+  }
+  for (int idx = tid; idx < I1p * (ldu - 4); idx += SW_THREADS) {
+    const int i = idx / (ldu - 4), j = idx - i * (ldu - 4);
+    Us[i * ldu + j] = (i < I1 && j < r1) ? U1[(size_t)i * r1 + j] : make_float2(0.f, 0.f);
   }
   __syncthreads();
-  // four output rows at a time: one load of N[j][c] serves them
-  for (int i = r0; i < I1; i += 4 * RP) {
-    cf acc[4];
-    int ii[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) { acc[q] = make_float2(0.f, 0.f); ii[q] = (i + q * RP < I1) ? i + q * RP : i; }
+  // ---- core[j][c] = sum_i conj(U1[i][j]) X[i][c]: rows (j, re|im), k = (i, re|im) ----
+  for (int tile = warp; tile < (r1p / 8) * 2; tile += SW_THREADS / 32) {
+    const int mt = tile >> 1, nt = tile & 1;
+    float tot[4] = {0.f, 0.f, 0.f, 0.f}, acc[4] = {0.f, 0.f, 0.f, 0.f}, acl[4] = {0.f, 0.f, 0.f, 0.f}, acx[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 4
-    for (int j = 0; j < r1; ++j) {
-      const cf nv = Ns[j * LD + cc];
+    for (int q = 0; q < I1p / 4; ++q) {
+      const int i = 4 * q + t;
+      const cf u = Us[i * ldu + 8 * mt + gq], x = Xs[i * SWT_LDX + 8 * nt + gq];
+      float urh, url, uih, uil, xh0, xl0, xh1, xl1;
+      mt_split(u.x, urh, url); mt_split(u.y, uih, uil);
+      mt_split(x.x, xh0, xl0); mt_split(x.y, xh1, xl1);
+      // Aop = conj(u): (Ar, Ai) = (ur, -ui); fragment (Ar, Ai, -Ai, Ar); the three products keep their own chains
+      mma_tf32(acc, urh, -uih, uih, urh, xh0, xh1);
+      mma_tf32(acl, url, -uil, uil, url, xh0, xh1);
+      mma_tf32(acx, urh, -uih, uih, urh, xl0, xl1);
+      if ((q & 15) == 15) {
 #pragma unroll
-      for (int q = 0; q < 4; ++q) cfma(acc[q], Us[ii[q] * r1 + j], nv);
+        for (int e = 0; e < 4; ++e) { tot[e] += acc[e] + (acl[e] + acx[e]); acc[e] = 0.f; acl[e] = 0.f; acx[e] = 0.f; }
+      }
     }
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
-      if (cok && i + q * RP < I1) out[(size_t)(i + q * RP) * C + c] = acc[q];
+    for (int e = 0; e < 4; ++e) tot[e] += acc[e] + (acl[e] + acx[e]);
+    Cs[(8 * mt + gq) * SWT_LDX + 8 * nt + 2 * t] = make_float2(tot[0], tot[2]);
+    Cs[(8 * mt + gq) * SWT_LDX + 8 * nt + 2 * t + 1] = make_float2(tot[1], tot[3]);
+  }
+  __syncthreads();
+  // ---- AdamUpdate of the block (rows past r1 are zero and stay zero) ----
+  for (int e = tid; e < r1 * SW_CB; e += SW_THREADS) {
+    const int j = e / SW_CB, cc = e - j * SW_CB;
+    cf n = make_float2(0.f, 0.f);
+    if (c0 + cc < C) {
+      const size_t idx = (size_t)j * C + c0 + cc;
+      const cf x = Cs[j * SWT_LDX + cc];
+      cf m = m_l[idx]; float v = v_l[idx];
+      n = adam_apply(x, m, v, a);
+      m_l[idx] = m; v_l[idx] = v; n_l[idx] = n; core[idx] = x;
+    }
+    Cs[j * SWT_LDX + cc] = n;
+  }
+  __syncthreads();
+  // ---- out[i][c] = sum_j U1[i][j] N[j][c] ----
+  for (int tile = warp; tile < (I1p / 8) * 2; tile += SW_THREADS / 32) {
+    const int mt = tile >> 1, nt = tile & 1;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f}, acl[4] = {0.f, 0.f, 0.f, 0.f}, acx[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+    for (int q = 0; q < r1p / 4; ++q) {
+      const int j = 4 * q + t;
+      const cf u = Us[(8 * mt + gq) * ldu + j], x = Cs[j * SWT_LDX + 8 * nt + gq];
+      float urh, url, uih, uil, xh0, xl0, xh1, xl1;
+      mt_split(u.x, urh, url); mt_split(u.y, uih, uil);
+      mt_split(x.x, xh0, xl0); mt_split(x.y, xh1, xl1);
+      mma_tf32(acc, urh, uih, -uih, urh, xh0, xh1);
+      mma_tf32(acl, url, uil, -uil, url, xh0, xh1);
+      mma_tf32(acx, urh, uih, -uih, urh, xl0, xl1);
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) acc[e] += acl[e] + acx[e];
+    const int i = 8 * mt + gq, c = c0 + 8 * nt + 2 * t;
+    if (i < I1) {
+      if (c < C) out[(size_t)i * C + c] = make_float2(acc[0], acc[2]);
+      if (c + 1 < C) out[(size_t)i * C + c + 1] = make_float2(acc[1], acc[3]);
+    }
   }
 }
 

@@ -567,7 +567,7 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
       // here cur holds [I_1][C] with C = r_2 .. r_N
       cf* dst = bufs[which];
       const uint32_t nblk_core = (uint32_t)((C + SW_CB - 1) / SW_CB), nblk_sparse = (ks + SW_THREADS - 1) / SW_THREADS;
-      core_sandwich_kernel<<<nblk_core + nblk_sparse, SW_THREADS, sandwich_smem((int)c.dims[0], c.ranks[0]), st>>>(
+      core_sandwich_tc_kernel<<<nblk_core + nblk_sparse, SW_THREADS, sandwich_tc_smem((int)c.dims[0], c.ranks[0]), st>>>(
           cur, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[0]), core, reinterpret_cast<cf*>(s->dp + L.p_ml),
           reinterpret_cast<float*>(s->dp + L.p_vl), n_l, (int)c.dims[0], c.ranks[0], (int)C, p.g_s, p.m_s, p.v_s, p.n_s, ks,
           nblk_core, p.adam);
@@ -657,8 +657,8 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
     if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
   }
   if (cfg->dims[0] <= SW_MAX_I && cfg->ranks[0] <= SW_MAX_R &&
-      cudaFuncSetAttribute(core_sandwich_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)sandwich_smem(SW_MAX_I, SW_MAX_R)) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
+      cudaFuncSetAttribute(core_sandwich_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)sandwich_tc_smem(SW_MAX_I, SW_MAX_R)) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
   if (cudaFuncSetAttribute(jacobi_sweeps_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)jac_sweeps_smem(JAC_SMEM_MAX_N)) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
