@@ -103,26 +103,20 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1,
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// The same MMA with operand a1 (resp. a1 and a3) negated inside the instruction sequence, so that the
-// negated copies of loop-invariant fragments do not occupy registers across the loop.
-__device__ __forceinline__ void mma_tf32_n1(float (&d)[4], float a0, float a1, float a2, float a3, float b0, float b1) {
-  asm(
-      "{\n\t.reg .b32 na1;\n\t"
-      "xor.b32 na1, %5, 0x80000000;\n\t"
-      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,na1,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n\t}"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(__float_as_uint(a0)), "r"(__float_as_uint(a1)), "r"(__float_as_uint(a2)), "r"(__float_as_uint(a3)),
-        "r"(__float_as_uint(b0)), "r"(__float_as_uint(b1)));
+// 16-byte read-only load that the compiler neither hoists out of a loop nor merges with its repeats.
+__device__ __forceinline__ float4 ld_nc_f4_volatile(const float4* p) {
+  float4 v;
+  asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
 }
-__device__ __forceinline__ void mma_tf32_n13(float (&d)[4], float a0, float a1, float a2, float a3, float b0, float b1) {
+
+// D = A * B: the first MMA of a chain, with the zero register as accumulator input (no clearing moves).
+__device__ __forceinline__ void mma_tf32_z(float (&d)[4], float a0, float a1, float a2, float a3, float b0, float b1) {
   asm(
-      "{\n\t.reg .b32 na1, na3;\n\t"
-      "xor.b32 na1, %5, 0x80000000;\n\t"
-      "xor.b32 na3, %7, 0x80000000;\n\t"
-      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,na1,%6,na3}, {%8,%9}, {%0,%1,%2,%3};\n\t}"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
       : "r"(__float_as_uint(a0)), "r"(__float_as_uint(a1)), "r"(__float_as_uint(a2)), "r"(__float_as_uint(a3)),
-        "r"(__float_as_uint(b0)), "r"(__float_as_uint(b1)));
+        "r"(__float_as_uint(b0)), "r"(__float_as_uint(b1)), "f"(0.f));
 }
 
 }  // namespace tg

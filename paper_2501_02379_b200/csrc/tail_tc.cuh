@@ -44,6 +44,7 @@ struct TailTcParams {
   TcGeom g;
   int* flags;               // sticky status word (bit 4: a bulk copy did not arrive within the wait limit)
   float s_sparse_pre;       // eta*lambda / (1 - eta*wd): the sparse term is applied before the decayed dense update
+  const float4* u2tab;      // compression: stage-2 operand fragments of Ua (proj_u2tab_kernel)
 };
 
 // k-steps of the compression's first product that hold any (b, re|im) of a row of 2B floats
@@ -136,8 +137,25 @@ __host__ inline bool proj_tc_geom(int A, int B, int rat, uint32_t nslab, int ntw
   return true;
 }
 
+// Stage-2 operand fragments of the compression kernel: for row tile `tile`, ja tile `mt` and lane (gq, t), with
+// a = 8 tile + 2 t and ja = 8 mt + gq: (u0.hi.x, u0.hi.y, u1.hi.x, u1.hi.y), (u0.lo.x, u0.lo.y, u1.lo.x, u1.lo.y),
+// u0 = Ua[a][ja], u1 = Ua[a+1][ja] split as TF32 value + remainder.  Rebuilt whenever Ua changes.
+__global__ void proj_u2tab_kernel(const cf* __restrict__ Ua, int A, int ra, int rat, float4* __restrict__ tab) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (A / 8) * rat * 32) return;
+  const int ln = idx & 31, mt = (idx >> 5) % rat, tile = (idx >> 5) / rat, g_ = ln >> 2, t_ = ln & 3;
+  const int a = 8 * tile + 2 * t_, ja = 8 * mt + g_;
+  const cf v0 = (ja < ra) ? Ua[a * ra + ja] : make_float2(0.f, 0.f);
+  const cf v1 = (ja < ra) ? Ua[(a + 1) * ra + ja] : make_float2(0.f, 0.f);
+  cf h0, l0, h1, l1;
+  split_tf32(v0.x, h0.x, l0.x); split_tf32(v0.y, h0.y, l0.y);
+  split_tf32(v1.x, h1.x, l1.x); split_tf32(v1.y, h1.y, l1.y);
+  tab[2 * idx] = make_float4(h0.x, h0.y, h1.x, h1.y);
+  tab[2 * idx + 1] = make_float4(l0.x, l0.y, l1.x, l1.y);
+}
+
 template <int RAT, int KS, int NTW, int PJ_WARPS>
-__global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW == 1 ? 4 : 3)) proj_tail_tc_kernel(const void* __restrict__ g, TailTcParams P) {
+__global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW <= 2 ? 4 : 3)) proj_tail_tc_kernel(const void* __restrict__ g, TailTcParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int PJ_THREADS = 32 * PJ_WARPS;
   const TailParams& p = P.p;
@@ -160,23 +178,11 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW == 1 ?
     cf h, l; split_tf32(u.x, h.x, l.x); split_tf32(u.y, h.y, l.y);
     u1tab[idx] = make_float4(h.x, h.y, l.x, l.y);
   }
-  // ---- operand fragments that stay in registers ----
-  // Ua[a][ja], Ua[a+1][ja] with a = 8 tile + 2t, ja = 8 mt + gq: (x, y, -y) of u0.hi, u1.hi, u0.lo, u1.lo
-  float u2[NTW][RAT][12];
+  // ---- stage-2 operand fragments come from the table in global memory (L1-resident): two float4 per
+  //      (row tile, ja tile, lane), read again for every slab so that they hold no registers across the loop ----
+  const float4* u2p[NTW];
 #pragma unroll
-  for (int nt = 0; nt < NTW; ++nt)
-#pragma unroll
-    for (int mt = 0; mt < RAT; ++mt) {
-      const int a = 8 * (wt + nt * tw) + 2 * t, ja = 8 * mt + gq;
-      cf v0 = (ja < ra) ? p.Ua[a * ra + ja] : make_float2(0.f, 0.f);
-      cf v1 = (ja < ra) ? p.Ua[(a + 1) * ra + ja] : make_float2(0.f, 0.f);
-      cf h0, l0, h1, l1;
-      split_tf32(v0.x, h0.x, l0.x); split_tf32(v0.y, h0.y, l0.y);
-      split_tf32(v1.x, h1.x, l1.x); split_tf32(v1.y, h1.y, l1.y);
-      float* w = u2[nt][mt];
-      w[0] = h0.x; w[1] = h0.y; w[2] = -h0.y; w[3] = h1.x; w[4] = h1.y; w[5] = -h1.y;
-      w[6] = l0.x; w[7] = l0.y; w[8] = -l0.y; w[9] = l1.x; w[10] = l1.y; w[11] = -l1.y;
-    }
+  for (int nt = 0; nt < NTW; ++nt) u2p[nt] = P.u2tab + ((size_t)(wt + nt * tw) * RAT * 32 + lane) * 2;
   // ---- this thread's first two output floats of a group: which partial element each sums, where it goes ----
   const int out_per_slab = 2 * ra * rb, n_out = spi * out_per_slab;
   int o_src[2], o_dst[2], o_q[2];
@@ -288,34 +294,37 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW == 1 ?
     }
     // ---- this group's contraction ----
     float d2[RAT][2][4];
-#pragma unroll
-    for (int mt = 0; mt < RAT; ++mt)
-#pragma unroll
-      for (int c = 0; c < 2; ++c)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) d2[mt][c][i] = 0.f;
     if (u * spi + q < nslab) {
       // stage 1 for the warp's NTW row tiles together: one Ub fragment load serves them all
       const float* xrow = xg + (size_t)q * (2 * E) + (size_t)(8 * wt + gq) * twoB;
       float dh[NTW][4], dl[NTW][4], dx[NTW][4];
 #pragma unroll
-      for (int nt = 0; nt < NTW; ++nt)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { dh[nt][i] = 0.f; dl[nt][i] = 0.f; dx[nt][i] = 0.f; }
-#pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
+        // Where a lane's float offset f lies past the row (the table holds zeros there) it reads the row's last
+        // entry instead: finite data, no predicate.  KS odd means B = 4 (KS - 1) + 1: every step but the last is
+        // whole, the last holds b = B - 1 alone.  KS == 8 means 16 <= B <= 32: the first four steps are whole.
         const int f = 32 * (ks >> 2) + 8 * t + 2 * (ks & 3);
+        int fo;
+        if ((KS & 1) && ks == KS - 1) fo = twoB - 2;
+        else if ((KS & 1) || (KS == 8 && ks < 4)) fo = f;
+        else fo = min(f, twoB - 2);
         const float4 uf = u1tab[ks * 32 + lane];
         const float nhy = -uf.y, nly = -uf.w;
 #pragma unroll
         for (int nt = 0; nt < NTW; ++nt) {
-          float2 x = (f < twoB) ? *reinterpret_cast<const float2*>(xrow + (size_t)(8 * nt * tw) * twoB + f) : make_float2(0.f, 0.f);
+          const float2 x = *reinterpret_cast<const float2*>(xrow + (size_t)(8 * nt * tw) * twoB + fo);
           float xh0, xl0, xh1, xl1;
           split_tf32_trunc(x.x, xh0, xl0); split_tf32_trunc(x.y, xh1, xl1);      // the streamed operand: cheapest split
           // A = (ur, -ui, ui, ur): rows (re, jb) and (im, jb) of W1
-          mma_tf32(dh[nt], uf.x, nhy, uf.y, uf.x, xh0, xh1);
-          mma_tf32(dl[nt], uf.z, nly, uf.w, uf.z, xh0, xh1);
-          mma_tf32(dx[nt], uf.x, nhy, uf.y, uf.x, xl0, xl1);
+          if (ks == 0) {
+            mma_tf32_z(dh[nt], uf.x, nhy, uf.y, uf.x, xh0, xh1);
+            mma_tf32_z(dl[nt], uf.z, nly, uf.w, uf.z, xh0, xh1);
+            mma_tf32_z(dx[nt], uf.x, nhy, uf.y, uf.x, xl0, xl1);
+          } else {
+            mma_tf32(dh[nt], uf.x, nhy, uf.y, uf.x, xh0, xh1);
+            mma_tf32(dl[nt], uf.z, nly, uf.w, uf.z, xh0, xh1);
+            mma_tf32(dx[nt], uf.x, nhy, uf.y, uf.x, xl0, xl1);
+          }
         }
       }
 #pragma unroll
@@ -326,16 +335,30 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW == 1 ?
         for (int i = 0; i < 4; ++i) split_tf32(dh[nt][i] + (dl[nt][i] + dx[nt][i]), yh[i], yl[i]);
 #pragma unroll
         for (int mt = 0; mt < RAT; ++mt) {
-          const float* w = u2[nt][mt];
+          // (x, y, -y) of u0.hi, u1.hi, u0.lo, u1.lo with u0 = Ua[a][ja], u1 = Ua[a+1][ja]
+          const float4 fh = ld_nc_f4_volatile(u2p[nt] + mt * 64), fl = ld_nc_f4_volatile(u2p[nt] + mt * 64 + 1);
+          const float w[12] = {fh.x, fh.y, -fh.y, fh.z, fh.w, -fh.w, fl.x, fl.y, -fl.y, fl.z, fl.w, -fl.w};
           // step c = re: A = (u0.x, -u0.y, u1.x, -u1.y), B = (Yre[a], Yre[a+1]);  step c = im: A = (u0.y, u0.x, u1.y, u1.x)
-          mma_tf32(d2[mt][0], w[0], w[2], w[3], w[5], yh[0], yh[1]);
-          mma_tf32(d2[mt][1], w[6], w[8], w[9], w[11], yh[0], yh[1]);
+          if (nt == 0) {
+            mma_tf32_z(d2[mt][0], w[0], w[2], w[3], w[5], yh[0], yh[1]);
+            mma_tf32_z(d2[mt][1], w[6], w[8], w[9], w[11], yh[0], yh[1]);
+          } else {
+            mma_tf32(d2[mt][0], w[0], w[2], w[3], w[5], yh[0], yh[1]);
+            mma_tf32(d2[mt][1], w[6], w[8], w[9], w[11], yh[0], yh[1]);
+          }
           mma_tf32(d2[mt][1], w[0], w[2], w[3], w[5], yl[0], yl[1]);
           mma_tf32(d2[mt][0], w[1], w[0], w[4], w[3], yh[2], yh[3]);
           mma_tf32(d2[mt][1], w[7], w[6], w[10], w[9], yh[2], yh[3]);
           mma_tf32(d2[mt][1], w[1], w[0], w[4], w[3], yl[2], yl[3]);
         }
       }
+    } else {
+#pragma unroll
+      for (int mt = 0; mt < RAT; ++mt)
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) d2[mt][c][i] = 0.f;
     }
     // partial T of this warp's rows: row-major [8 RAT][8] complex, (d0, d2) = T[ja][2t], (d1, d3) = T[ja][2t+1]
     {

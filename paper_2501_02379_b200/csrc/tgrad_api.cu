@@ -31,7 +31,7 @@ inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
 struct Layout {
   // persistent block
-  size_t p_flags, p_omega, p_slab, p_factor[TGRAD_MAX_NDIM], p_ml, p_vl, p_ms, p_vs, p_total;
+  size_t p_flags, p_omega, p_slab, p_factor[TGRAD_MAX_NDIM], p_ml, p_vl, p_ms, p_vs, p_u2tab, p_total;
   uint32_t nslab, E;          // slabs of the trailing two modes, entries per slab
   // workspace block
   size_t w_ns, w_gs, w_core, w_nl, w_bufa, w_bufb, w_sel, w_hist, w_blk, w_gram[TGRAD_MAX_NDIM], w_jac[TGRAD_MAX_NDIM],
@@ -119,6 +119,8 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
   L.p_vl = o; o = align_up(o + P * 4);
   L.p_ms = o; o = align_up(o + k * 8);
   L.p_vs = o; o = align_up(o + k * 4);
+  // operand-fragment table of the compression kernel: 32 lanes x 32 bytes per (8-row tile, 8-column tile) of U^(N-1)
+  L.p_u2tab = o; o = align_up(o + (size_t)((c->dims[N - 2] + 7) / 8) * ((c->ranks[N - 2] + 7) / 8) * 1024);
   L.p_total = o;
   o = 0;
   L.w_ns = o; o = align_up(o + k * 8);
@@ -160,6 +162,7 @@ struct tgrad_state {
   char* dw;
   int64_t t;
   bool have_subspace;
+  bool tabs_stale;      // U^(N-1) changed since the compression kernel's fragment table was built
   int sm_count;
   TailPlan tail;
   // optional per-stage timing
@@ -311,7 +314,7 @@ tgrad_status plan_tail(tgrad_state* s) {
     // 8 warps with one tile each: 101 against 122 us on 128x128x64x33)
     tp.pjw = 4; tp.ntw = (A == 64) ? 2 : (A == 32 ? 4 : 2);
     tp.back_ns = ((uint64_t)A * B * 8 <= 8192) ? 2 : 1;      // small slabs: two per warp and iteration
-    const int pj_blocks = tp.pjw == 8 ? 2 : (tp.ntw == 1 ? 4 : 3);     // resident blocks per SM
+    const int pj_blocks = tp.pjw == 8 ? 2 : (tp.ntw <= 2 ? 4 : 3);     // resident blocks per SM
     const uint32_t pj_smem = (227u * 1024u) / pj_blocks - 1024u;
     if (proj_tc_geom(A, B, rat, (uint32_t)S, tp.ntw, tp.pjw, pj_smem, tp.gproj) && tail_tc_geom(true, A, B, rat, (uint32_t)S, tp.back_ns, tp.gback)) {
       const uint32_t cap = 2u * (uint32_t)s->sm_count, pcap = (uint32_t)pj_blocks * (uint32_t)s->sm_count;
@@ -463,6 +466,7 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
     jacobi_factors_kernel<<<fp.nmodes, JAC_THREADS, 0, st>>>(fp); TG_LAUNCH_CHECK();
   }
   s->have_subspace = true;
+  s->tabs_stale = true;
   return TGRAD_OK;
 }
 
@@ -528,6 +532,14 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   mp.s_sparse_pre = (float)((double)c.lr * (double)c.lambda / (1.0 - (double)c.lr * (double)c.weight_decay));
   if (s->tail.tc) {
     mp.p = p; mp.g = s->tail.gproj;
+    float4* tab = reinterpret_cast<float4*>(s->dp + L.p_u2tab);
+    if (s->tabs_stale) {
+      const int n_ent = (A / 8) * s->tail.rat * 32;
+      proj_u2tab_kernel<<<(n_ent + 127) / 128, 128, 0, st>>>(p.Ua, A, ra, s->tail.rat, tab);
+      TG_LAUNCH_CHECK();
+      s->tabs_stale = false;
+    }
+    mp.u2tab = tab;
     TG_TRY(tc_dispatch(1, s->tail, d_grad, mp, st));
   } else if (s->tail.th) {
     TailHParams hp; hp.p = p; hp.g = s->tail.gh; hp.flags = mp.flags;
@@ -642,7 +654,7 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
   memset(st, 0, sizeof(*st));
   st->cfg = *cfg; st->L = L;
   st->dp = static_cast<char*>(d_persistent); st->dw = static_cast<char*>(d_workspace);
-  st->t = 0; st->have_subspace = false;
+  st->t = 0; st->have_subspace = false; st->tabs_stale = true;
   int dev = 0, sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
@@ -780,6 +792,7 @@ tgrad_status tgrad_import_state(tgrad_state* st, int32_t what, const void* host_
     if (cudaStreamSynchronize(stream) != cudaSuccess) return TGRAD_ERR_CUDA;
   }
   if (what == TGRAD_WHAT_OMEGA || what >= TGRAD_WHAT_FACTOR_BASE) st->have_subspace = true;
+  if (what >= TGRAD_WHAT_FACTOR_BASE) st->tabs_stale = true;
   return TGRAD_OK;
 }
 
