@@ -21,7 +21,8 @@
  *  - Pointers named d_* are DEVICE pointers, everything else is host memory.
  *  - The library never allocates or frees device memory and never creates
  *    streams.  The caller owns: the weight, the gradient, one persistent
- *    block (Omega, U^(n), moments, status words) and one workspace block
+ *    block (Omega, U^(n), moments, status words, a split copy of U^(N-1)
+ *    laid out for the compression kernel) and one workspace block
  *    (scratch; contents need not survive between calls, but the same
  *    workspace must not be used by two states concurrently).  Sizes come
  *    from tgrad_state_bytes().  Both blocks must be 256-byte aligned.
