@@ -125,7 +125,7 @@ __host__ inline bool proj_tc_geom(int A, int B, int rat, uint32_t nslab, int ntw
   g.slab_bytes = (uint32_t)A * B * 8;
   g.grp_stride = ((uint32_t)g.spi * g.slab_bytes + 127) & ~127u;
   g.ngroups = (nslab + g.spi - 1) / g.spi;
-  const uint32_t aux = 2u * PJ_WARPS * rat * 128 * 4 + (uint32_t)g.nbt * 32 * 16;   // partial sums, then the Ub fragment table
+  const uint32_t aux = 2u * PJ_WARPS * rat * 128 * 4 + (uint32_t)g.nbt * 32 * 32;   // partial sums, then the Ub fragment table
   const uint32_t fixed = ((aux + 127) & ~127u) + 128;
   if (fixed + 2 * g.grp_stride > smem_per_block) return false;
   int nbuf = (int)((smem_per_block - fixed) / g.grp_stride);
@@ -169,14 +169,16 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW <= 2 ?
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + G.off_bar);
   const unsigned char* gb = static_cast<const unsigned char*>(g);
 
-  // ---- Ub as stage-1 operand fragments, per k-step and lane: (hi.x, hi.y, lo.x, lo.y) of Ub[b][jb = gq] ----
-  float4* u1tab = reinterpret_cast<float4*>(red + 2 * PJ_WARPS * REDW);   // [nbt][32]
+  // ---- Ub as stage-1 operand fragments, per k-step and lane, in MMA register order (a0, a1, a2, a3) =
+  //      (ur, -ui, ui, ur) of Ub[b][jb = gq]: [0] of the TF32 part, [1] of the remainder ----
+  float4* u1tab = reinterpret_cast<float4*>(red + 2 * PJ_WARPS * REDW);   // [2][nbt][32]
   for (int idx = tid; idx < G.nbt * 32; idx += PJ_THREADS) {
     const int ks = idx >> 5, ln = idx & 31, g_ = ln >> 2, t_ = ln & 3;
     const int f = 32 * (ks >> 2) + 8 * t_ + 2 * (ks & 3);
     cf u = (f < twoB && g_ < rb) ? p.Ub[(f >> 1) * rb + g_] : make_float2(0.f, 0.f);
     cf h, l; split_tf32(u.x, h.x, l.x); split_tf32(u.y, h.y, l.y);
-    u1tab[idx] = make_float4(h.x, h.y, l.x, l.y);
+    u1tab[idx] = make_float4(h.x, -h.y, h.y, h.x);
+    u1tab[G.nbt * 32 + idx] = make_float4(l.x, -l.y, l.y, l.x);
   }
   // ---- stage-2 operand fragments come from the table in global memory (L1-resident): two float4 per
   //      (row tile, ja tile, lane), read again for every slab so that they hold no registers across the loop ----
@@ -308,8 +310,7 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW <= 2 ?
         if ((KS & 1) && ks == KS - 1) fo = twoB - 2;
         else if ((KS & 1) || (KS == 8 && ks < 4)) fo = f;
         else fo = min(f, twoB - 2);
-        const float4 uf = u1tab[ks * 32 + lane];
-        const float nhy = -uf.y, nly = -uf.w;
+        const float4 uh = u1tab[ks * 32 + lane], ul = u1tab[(G.nbt + ks) * 32 + lane];
 #pragma unroll
         for (int nt = 0; nt < NTW; ++nt) {
           const float2 x = *reinterpret_cast<const float2*>(xrow + (size_t)(8 * nt * tw) * twoB + fo);
@@ -317,13 +318,13 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW <= 2 ?
           split_tf32_trunc(x.x, xh0, xl0); split_tf32_trunc(x.y, xh1, xl1);      // the streamed operand: cheapest split
           // A = (ur, -ui, ui, ur): rows (re, jb) and (im, jb) of W1
           if (ks == 0) {
-            mma_tf32_z(dh[nt], uf.x, nhy, uf.y, uf.x, xh0, xh1);
-            mma_tf32_z(dl[nt], uf.z, nly, uf.w, uf.z, xh0, xh1);
-            mma_tf32_z(dx[nt], uf.x, nhy, uf.y, uf.x, xl0, xl1);
+            mma_tf32_z(dh[nt], uh.x, uh.y, uh.z, uh.w, xh0, xh1);
+            mma_tf32_z(dl[nt], ul.x, ul.y, ul.z, ul.w, xh0, xh1);
+            mma_tf32_z(dx[nt], uh.x, uh.y, uh.z, uh.w, xl0, xl1);
           } else {
-            mma_tf32(dh[nt], uf.x, nhy, uf.y, uf.x, xh0, xh1);
-            mma_tf32(dl[nt], uf.z, nly, uf.w, uf.z, xh0, xh1);
-            mma_tf32(dx[nt], uf.x, nhy, uf.y, uf.x, xl0, xl1);
+            mma_tf32(dh[nt], uh.x, uh.y, uh.z, uh.w, xh0, xh1);
+            mma_tf32(dl[nt], ul.x, ul.y, ul.z, ul.w, xh0, xh1);
+            mma_tf32(dx[nt], uh.x, uh.y, uh.z, uh.w, xl0, xl1);
           }
         }
       }
