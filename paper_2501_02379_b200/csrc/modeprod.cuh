@@ -122,6 +122,7 @@ __global__ void __launch_bounds__(MP_THREADS) mode_product_kernel(const cf* __re
 __global__ void adam_kernel(const cf* __restrict__ core, cf* __restrict__ m_l, float* __restrict__ v_l,
                             cf* __restrict__ n_l, uint32_t n, const cf* __restrict__ g_s, cf* __restrict__ m_s,
                             float* __restrict__ v_s, cf* __restrict__ n_s, uint32_t ks, AdamScalars a) {
+  griddep_chain();
   uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) {
     cf m = m_l[i]; float v = v_l[i];
@@ -156,6 +157,7 @@ __device__ __forceinline__ void mt_split(float x, float& hi, float& lo) {
 template <bool CONJ_T, int NT>
 __global__ void __launch_bounds__(MT_THREADS) mode_product_tc_kernel(const cf* __restrict__ in, cf* __restrict__ out,
                                                                      const cf* __restrict__ U, int M, int K, int C, int r_n) {
+  griddep_chain();
   constexpr int BC = 32 * NT, LDX = BC + 4;      // X tile row length: rows 4 slots apart in the 16 bank pairs
   __shared__ __align__(16) float4 As[2][MT_BM][MT_LDA];   // (re.hi, im.hi, re.lo, im.lo) of Aop[m][k]
   __shared__ __align__(16) cf Xs[2][MT_BK][LDX];
@@ -303,6 +305,7 @@ __global__ void __launch_bounds__(SW_THREADS) core_sandwich_tc_kernel(const cf* 
                                                                       const cf* __restrict__ g_s, cf* __restrict__ m_s,
                                                                       float* __restrict__ v_s, cf* __restrict__ n_s, uint32_t ks,
                                                                       uint32_t nblk_core, AdamScalars a) {
+  griddep_chain();
   extern __shared__ __align__(16) unsigned char swm[];
   if (blockIdx.x >= nblk_core) {
     const uint32_t i = (blockIdx.x - nblk_core) * SW_THREADS + threadIdx.x;

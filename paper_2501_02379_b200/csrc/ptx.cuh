@@ -103,6 +103,16 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1,
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute may be
+// scheduled before its predecessor in the stream has finished; griddep_wait() blocks until that predecessor
+// has completed and its writes are visible, griddep_launch_dependents() lets the successor be scheduled as
+// soon as every block of this grid has got this far.  Both are no-ops in a kernel launched the ordinary way.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// What every kernel of the step starts with: nothing in global memory is touched before the predecessor is done,
+// so only the launch itself and the scheduling of the blocks overlap with the predecessor's tail.
+__device__ __forceinline__ void griddep_chain() { griddep_launch_dependents(); griddep_wait(); }
+
 // 16-byte read-only load that the compiler neither hoists out of a loop nor merges with its repeats.
 __device__ __forceinline__ float4 ld_nc_f4_volatile(const float4* p) {
   float4 v;

@@ -96,6 +96,7 @@ __host__ inline TailBlkGeom tail_blk_geom(int A, int B, int ra, int rb, bool bac
 // The gathered sparse values go to p.g_s (their AdamUpdate runs with the core's).
 template <class S>
 __global__ void __launch_bounds__(TB_THREADS) proj_tail_blk_kernel(const void* __restrict__ g, TailParams p, TailBlkGeom G) {
+  griddep_chain();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int A = p.A, B = p.B, Bs = G.Bs, ra = p.ra, rb = p.rb, rbp = G.rbp, js = G.js;
@@ -161,6 +162,7 @@ __global__ void __launch_bounds__(TB_THREADS) proj_tail_blk_kernel(const void* _
 // rounded to fp16 before the sparse term is added, and once more when stored).
 template <class S>
 __global__ void __launch_bounds__(TB_THREADS) back_tail_blk_kernel(void* __restrict__ w, TailParams p, TailBlkGeom G) {
+  griddep_chain();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int A = p.A, B = p.B, Bs = G.Bs, ra = p.ra, rb = p.rb, rbp = G.rbp, ras = G.ras, js = G.js;

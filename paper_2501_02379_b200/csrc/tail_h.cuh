@@ -84,6 +84,7 @@ __device__ __forceinline__ void split_f16(float x, __half& hi, __half& lo) {
 // ---------------------------------------------------------------------------------------------
 template <int RAT, int RBT>
 __global__ void __launch_bounds__(512, 1) proj_tail_h_kernel(const void* __restrict__ g, TailHParams P) {
+  griddep_chain();
   extern __shared__ __align__(128) unsigned char smem[];
   const TailParams& p = P.p;
   const TailHGeom& G = P.g;
@@ -319,6 +320,7 @@ struct TailHBParams {
 
 template <int RAT, int RBT>
 __global__ void __launch_bounds__(512, 1) back_tail_h_kernel(void* __restrict__ w, TailHBParams P) {
+  griddep_chain();
   extern __shared__ __align__(128) unsigned char smem[];
   const TailParams& p = P.p;
   const TailHBGeom& G = P.g;

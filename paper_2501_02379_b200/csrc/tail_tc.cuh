@@ -156,6 +156,7 @@ __global__ void proj_u2tab_kernel(const cf* __restrict__ Ua, int A, int ra, int 
 
 template <int RAT, int KS, int NTW, int PJ_WARPS>
 __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW <= 2 ? 4 : 3)) proj_tail_tc_kernel(const void* __restrict__ g, TailTcParams P) {
+  griddep_chain();
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int PJ_THREADS = 32 * PJ_WARPS;
   const TailParams& p = P.p;
@@ -403,6 +404,7 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW <= 2 ?
 // ---------------------------------------------------------------------------------------------
 template <int RAT, int NS>
 __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __restrict__ w, TailTcParams P) {
+  griddep_chain();
   extern __shared__ __align__(128) unsigned char smem[];
   const TailParams& p = P.p;
   const TcGeom& G = P.g;

@@ -179,6 +179,18 @@ namespace {
     if (cudaPeekAtLastError() != cudaSuccess) return TGRAD_ERR_CUDA; \
   } while (0)
 
+// Launch of a kernel of the step: programmatic dependent launch, so that its blocks are scheduled while the
+// previous kernel of the stream drains (every such kernel begins with griddep_chain()).
+template <typename... KA, typename... AA>
+inline void launch_chained(void (*kern)(KA...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, AA&&... args) {
+  cudaLaunchConfig_t lc; memset(&lc, 0, sizeof(lc));
+  lc.gridDim = grid; lc.blockDim = block; lc.dynamicSmemBytes = smem; lc.stream = st;
+  cudaLaunchAttribute at; memset(&at, 0, sizeof(at));
+  at.id = cudaLaunchAttributeProgrammaticStreamSerialization; at.val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = &at; lc.numAttrs = 1;
+  (void)cudaLaunchKernelEx(&lc, kern, static_cast<KA>(args)...);     // an error stays pending for TG_LAUNCH_CHECK
+}
+
 // op: 0 = set attributes, 1 = proj, 2 = back
 template <class S>
 tgrad_status tail_dispatch(int op, const TailPlan& tp, void* ptr, const TailParams& p, cudaStream_t st) {
@@ -189,8 +201,8 @@ tgrad_status tail_dispatch(int op, const TailPlan& tp, void* ptr, const TailPara
                              (int)tp.bback.total) != cudaSuccess) return TGRAD_ERR_CUDA;
     return TGRAD_OK;
   }
-  if (op == 2) back_tail_blk_kernel<S><<<tp.grid_bback, TB_THREADS, tp.bback.total, st>>>(ptr, p, tp.bback);
-  else proj_tail_blk_kernel<S><<<tp.grid_bproj, TB_THREADS, tp.bproj.total, st>>>(ptr, p, tp.bproj);
+  if (op == 2) launch_chained(back_tail_blk_kernel<S>, dim3(tp.grid_bback), dim3(TB_THREADS), tp.bback.total, st, ptr, p, tp.bback);
+  else launch_chained(proj_tail_blk_kernel<S>, dim3(tp.grid_bproj), dim3(TB_THREADS), tp.bproj.total, st, ptr, p, tp.bproj);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
@@ -206,7 +218,7 @@ tgrad_status tc_proj_op2(int op, const TailPlan& tp, const void* g, const TailTc
     return cudaFuncSetAttribute(proj_tail_tc_kernel<RAT, KS, NTW, W>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)tp.gproj.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
   }
-  proj_tail_tc_kernel<RAT, KS, NTW, W><<<tp.grid_proj, 32 * W, tp.gproj.total, st>>>(g, P);
+  launch_chained(proj_tail_tc_kernel<RAT, KS, NTW, W>, dim3(tp.grid_proj), dim3(32 * W), tp.gproj.total, st, g, P);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
@@ -222,7 +234,7 @@ tgrad_status tc_back_op2(int op, const TailPlan& tp, void* w, const TailTcParams
     return cudaFuncSetAttribute(back_tail_tc_kernel<RAT, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)tp.gback.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
   }
-  back_tail_tc_kernel<RAT, NS><<<tp.grid_back, TC_THREADS, tp.gback.total, st>>>(w, P);
+  launch_chained(back_tail_tc_kernel<RAT, NS>, dim3(tp.grid_back), dim3(TC_THREADS), tp.gback.total, st, w, P);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
@@ -236,7 +248,7 @@ tgrad_status th_proj_op(int op, const TailPlan& tp, const void* g, const TailHPa
     return cudaFuncSetAttribute(proj_tail_h_kernel<RAT, RBT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)tp.gh.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
   }
-  proj_tail_h_kernel<RAT, RBT><<<tp.grid_h, 32 * tp.gh.nwarps, tp.gh.total, st>>>(g, P);
+  launch_chained(proj_tail_h_kernel<RAT, RBT>, dim3(tp.grid_h), dim3(32 * tp.gh.nwarps), tp.gh.total, st, g, P);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
@@ -253,7 +265,7 @@ tgrad_status th_back_op(int op, const TailPlan& tp, void* w, const TailHBParams&
     return cudaFuncSetAttribute(back_tail_h_kernel<RAT, RBT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)tp.ghb.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
   }
-  back_tail_h_kernel<RAT, RBT><<<tp.grid_hb, 32 * tp.ghb.nwarps, tp.ghb.total, st>>>(w, P);
+  launch_chained(back_tail_h_kernel<RAT, RBT>, dim3(tp.grid_hb), dim3(32 * tp.ghb.nwarps), tp.ghb.total, st, w, P);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
@@ -481,11 +493,11 @@ tgrad_status mode_product(bool conj_t, const cf* in, cf* out, const cf* U, uint6
   const int bc = (wide < (uint64_t)4 * sm_count) ? 32 : 64;
   dim3 grid((unsigned)((C + bc - 1) / bc), (unsigned)((M + MT_BM - 1) / MT_BM), (unsigned)O);
   if (bc == 64) {
-    if (conj_t) mode_product_tc_kernel<true, 2><<<grid, MT_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
-    else mode_product_tc_kernel<false, 2><<<grid, MT_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
+    if (conj_t) launch_chained(mode_product_tc_kernel<true, 2>, dim3(grid), dim3(MT_THREADS), 0, st, in, out, U, M, K, (int)C, r_n);
+    else launch_chained(mode_product_tc_kernel<false, 2>, dim3(grid), dim3(MT_THREADS), 0, st, in, out, U, M, K, (int)C, r_n);
   } else {
-    if (conj_t) mode_product_tc_kernel<true, 1><<<grid, MT_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
-    else mode_product_tc_kernel<false, 1><<<grid, MT_THREADS, 0, st>>>(in, out, U, M, K, (int)C, r_n);
+    if (conj_t) launch_chained(mode_product_tc_kernel<true, 1>, dim3(grid), dim3(MT_THREADS), 0, st, in, out, U, M, K, (int)C, r_n);
+    else launch_chained(mode_product_tc_kernel<false, 1>, dim3(grid), dim3(MT_THREADS), 0, st, in, out, U, M, K, (int)C, r_n);
   }
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
@@ -579,14 +591,14 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
       // here cur holds [I_1][C] with C = r_2 .. r_N
       cf* dst = bufs[which];
       const uint32_t nblk_core = (uint32_t)((C + SW_CB - 1) / SW_CB), nblk_sparse = (ks + SW_THREADS - 1) / SW_THREADS;
-      core_sandwich_tc_kernel<<<nblk_core + nblk_sparse, SW_THREADS, sandwich_tc_smem((int)c.dims[0], c.ranks[0]), st>>>(
+      launch_chained(core_sandwich_tc_kernel, dim3(nblk_core + nblk_sparse), dim3(SW_THREADS), sandwich_tc_smem((int)c.dims[0], c.ranks[0]), st, 
           cur, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[0]), core, reinterpret_cast<cf*>(s->dp + L.p_ml),
           reinterpret_cast<float*>(s->dp + L.p_vl), n_l, (int)c.dims[0], c.ranks[0], (int)C, p.g_s, p.m_s, p.v_s, p.n_s, ks,
           nblk_core, p.adam);
       TG_LAUNCH_CHECK();
       src = dst; which ^= 1; mfirst = 1;
     } else {
-      adam_kernel<<<(unsigned)((L.P + ks + 255) / 256), 256, 0, st>>>(
+      launch_chained(adam_kernel, dim3((unsigned)((L.P + ks + 255) / 256)), dim3(256), 0, st, 
           core, reinterpret_cast<cf*>(s->dp + L.p_ml), reinterpret_cast<float*>(s->dp + L.p_vl), n_l, (uint32_t)L.P,
           p.g_s, p.m_s, p.v_s, p.n_s, ks, p.adam);
       TG_LAUNCH_CHECK();
