@@ -249,6 +249,23 @@ __device__ __forceinline__ void jac_rotation(float a, float d, cf b, float absb,
   R.npp = a - t * absb; R.nqq = d + t * absb;
 }
 
+// The same with the hardware's approximate reciprocal, square root and reciprocal square root (each good to a
+// few ulp, but several times shorter than the IEEE sequences): the angle is then off by a few ulp, which the next
+// sweep sees as a slightly larger remainder, while c^2 + s^2 = 1 and |g| = 1 are restored by jac_unit as above.
+// On the critical path of every stage of the rotation-log kernels, where all other warps wait for these values.
+__device__ __forceinline__ void jac_rotation_fast(float a, float d, cf b, float b2, JacRot& R) {
+  const float inv = rsqrtf(b2), absb = b2 * inv;
+  const float tau = 0.5f * (d - a) * inv, at = fminf(fabsf(tau), 1e18f);     // the cap keeps tau^2 finite
+  const float q = fmaf(at, at, 1.f);
+  const float t = copysignf(__fdividef(1.f, at + q * rsqrtf(q)), tau);
+  float c = rsqrtf(fmaf(t, t, 1.f)), s = t * c;
+  jac_unit(c, s);
+  float gx = b.x * inv, gy = -b.y * inv;
+  jac_unit(gx, gy);
+  R.c = c; R.s = s; R.gx = gx; R.gy = gy;
+  R.npp = a - t * absb; R.nqq = d + t * absb;
+}
+
 // Only the upper triangle of A (i <= j) is kept up to date: A is Hermitian before and after every
 // stage, so block (I, J) with I < J determines block (J, I), and half of the shared-memory traffic
 // -- which is what bounds this kernel -- goes away.
@@ -366,7 +383,7 @@ __global__ void __launch_bounds__(JAC_THREADS) jacobi_sweeps_kernel(JacobiFastPa
           cf b = A[(size_t)p * ld + q];
           float b2 = b.x * b.x + b.y * b.y;
           if (b2 > thr2 && b2 > 0.f) {
-            jac_rotation(a, d, b, sqrtf(b2), R);
+            jac_rotation_fast(a, d, b, b2, R);
             act = true;
           }
         }
