@@ -29,10 +29,10 @@ METRIC = "tgrad_step effective HBM GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the two streaming kernels, from the ncu
-# capture summarised in profiles/cfg3_step_and_refresh_block_cooperative.md (bytes); None where no
+# capture summarised in profiles/cfg3_step_and_refresh_tensor_core_path.md (bytes); None where no
 # capture exists for the workload.  (back_tail: 304.1 MB read + 218.0 MB written -- the rest of the
 # 277 MB it writes is still in L2 when the kernel ends.)
-NCU_TRAFFIC_BYTES = {("cfg3", "proj_tail"): 280.4e6 + 19.6e6, ("cfg3", "back_tail"): 304.1e6 + 218.0e6}
+NCU_TRAFFIC_BYTES = {("cfg3", "proj_tail"): 280.4e6 + 19.0e6, ("cfg3", "back_tail"): 304.1e6 + 218.3e6}
 
 
 def step_bytes(wl: synth.Workload) -> int:
