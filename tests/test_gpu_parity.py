@@ -45,6 +45,30 @@ def test_k_zero_lowrank_only():
         p.step(t)
 
 
+def test_k_equals_numel_sparse_only():
+    # every entry is selected: the residual, its Gram matrices and the core are zero, any orthonormal U^(n) is a valid
+    # factor (so the subspaces are not compared), and the update is the sparse branch alone
+    import dataclasses
+    wl = dataclasses.replace(synth.WORKLOADS["small4"], rho=(1, 1), outlier_frac=(0, 1))
+    assert wl.k == wl.numel
+    p = Pair(wl)
+    g = p.src.gradient(0)
+    p.gst.refresh_subspace(to_device(g, False))
+    orc.oracle_refresh(p.ost, g)
+    assert p.gst.query_status()[0] == 0
+    assert np.array_equal(p.gst.export(B.WHAT_OMEGA), np.arange(wl.numel, dtype=np.uint32))
+    us = p.gst.factors()
+    for u in us:
+        assert H.ortho_defect(u) <= 1e-5
+    p.ost.factors = [u.copy() for u in us]
+    for t in range(3):
+        g = p.src.gradient(t)
+        p.gst.step(p.w_dev, to_device(g, False))
+        p.w_ref = orc.oracle_step(p.ost, p.w_ref, g, refresh=False)
+        p.compare()
+    assert not np.any(p.gst.export(B.WHAT_CORE))
+
+
 def test_topk_ties_bit_exact():
     # tie-heavy quantised gradients, all-equal magnitudes, k in {1, I-1, I}
     shape = (12, 10, 8, 5)
