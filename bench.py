@@ -218,7 +218,8 @@ def run_ours(args, wl):
     grads = [[dev(g) for g in gl] for gl in grads_host]
     w0 = [s.weight() for s in srcs]
     weights = [dev(w) for w in w0]
-    cfgs = [B.make_config(wl.shape, wl.ranks, wl.k, wl.T, lr=wl.lr, half_storage=half, auto_refresh=True)
+    cfgs = [B.make_config(wl.shape, wl.ranks, wl.k, wl.T, lr=wl.lr, half_storage=half, auto_refresh=True,
+                          warm_refresh=True)
             for _ in srcs]
     states = [B.TgradState(c) for c in cfgs]
     stream = torch.cuda.current_stream()
@@ -366,7 +367,7 @@ def run_ours(args, wl):
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{wl.name}: {n_t} x complex {'x'.join(map(str, wl.shape))} "
                                f"({'2xfp16' if half else 'complex64'} W/G), ranks {list(wl.ranks)}, k={wl.k}, T={wl.T}",
-                   "tensors_per_gpu": n_t, "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "tensors_per_gpu": n_t, "warm_refresh": True, "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": f"inputs larger than L2: ring of {ring} gradient buffers of "
                          f"{wl.numel * eb / 1e6:.0f} MB each plus the weight"},
         "steps_per_s": args.steps * world / (ms * 1e-3),

@@ -41,6 +41,7 @@ class TgradConfig(C.Structure):
         ("auto_refresh", C.c_int32),
         ("jacobi_max_sweeps", C.c_int32),
         ("jacobi_tol", C.c_float),
+        ("warm_refresh", C.c_int32),
     ]
 
 
@@ -111,7 +112,7 @@ def _check(s: int, where: str) -> None:
 def make_config(shape: Sequence[int], ranks: Sequence[int], k: int, T: int, lr: float = 1e-3, alpha: float = 1.0,
                 lam: float = 1.0, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
                 weight_decay: float = 0.0, half_storage: bool = False, auto_refresh: bool = True,
-                jacobi_max_sweeps: int = 0, jacobi_tol: float = 0.0) -> TgradConfig:
+                jacobi_max_sweeps: int = 0, jacobi_tol: float = 0.0, warm_refresh: bool = False) -> TgradConfig:
     if len(shape) > MAX_NDIM or len(shape) != len(ranks):
         raise ValueError("bad shape / ranks")
     cfg = TgradConfig()
@@ -128,6 +129,7 @@ def make_config(shape: Sequence[int], ranks: Sequence[int], k: int, T: int, lr: 
     cfg.auto_refresh = 1 if auto_refresh else 0
     cfg.jacobi_max_sweeps = jacobi_max_sweeps
     cfg.jacobi_tol = jacobi_tol
+    cfg.warm_refresh = 1 if warm_refresh else 0
     return cfg
 
 

@@ -201,6 +201,7 @@ struct JacobiFastParams {
   int max_sweeps;
   float tol;
   int* flags;        // flags[0] sticky bits, flags[1 + mode] sweeps used
+  int warm;          // jacobi_vectors_kernel: V holds the basis the matrix was rotated into; the rotations are applied to it in place
 };
 
 // the pair of players (p < q) that meet at table `tb` in stage `stage` of a round robin of m players
@@ -412,6 +413,16 @@ __global__ void __launch_bounds__(JAC_THREADS) jacobi_sweeps_kernel(JacobiFastPa
   for (int i = tid; i < n; i += nt) md.lam[i] = A[(size_t)i * ld + i].x;
 }
 
+// E = 3/2 I - 1/2 G in place: with G = V^H V, V E is one Newton-Schulz step of V towards orthonormal columns
+// (a defect d of V^H V - I becomes O(d^2)); keeps the basis carried from refresh to refresh from drifting.
+__global__ void ns_residual_kernel(cf* __restrict__ G, int n) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n * n) return;
+  const int i = idx / n, j = idx - i * n;
+  const cf g = G[idx];
+  G[idx] = make_float2((i == j ? 1.5f : 0.f) - 0.5f * g.x, -0.5f * g.y);
+}
+
 // NP = pairs per lane (>= n/64), D = stages of the log kept in flight
 template <int NP, int D>
 __global__ void __launch_bounds__(256) jacobi_vectors_kernel(JacobiFastParams P) {
@@ -427,7 +438,7 @@ __global__ void __launch_bounds__(256) jacobi_vectors_kernel(JacobiFastParams P)
   const int m = (n + 1) & ~1, half = m >> 1;
   const int sweeps = P.flags[1 + md.index];
   cf* row = rows + (size_t)warp * P.row_stride;
-  for (int j = lane; j < n; j += 32) row[j] = make_float2(j == i_row ? 1.f : 0.f, 0.f);
+  for (int j = lane; j < n; j += 32) row[j] = P.warm ? md.V[(size_t)i_row * n + j] : make_float2(j == i_row ? 1.f : 0.f, 0.f);
   __syncwarp();
   // the log is replayed D stages at a time, the next D already in flight
   const float4* lg = md.log;

@@ -31,11 +31,11 @@ inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 
 struct Layout {
   // persistent block
-  size_t p_flags, p_omega, p_slab, p_factor[TGRAD_MAX_NDIM], p_ml, p_vl, p_ms, p_vs, p_u2tab, p_total;
+  size_t p_flags, p_omega, p_slab, p_factor[TGRAD_MAX_NDIM], p_ml, p_vl, p_ms, p_vs, p_u2tab, p_basis[TGRAD_MAX_NDIM], p_total;
   uint32_t nslab, E;          // slabs of the trailing two modes, entries per slab
   // workspace block
   size_t w_ns, w_gs, w_core, w_nl, w_bufa, w_bufb, w_sel, w_hist, w_blk, w_gram[TGRAD_MAX_NDIM], w_jac[TGRAD_MAX_NDIM],
-      w_v[TGRAD_MAX_NDIM], w_log[TGRAD_MAX_NDIM], w_lam[TGRAD_MAX_NDIM], w_partial, w_total;
+      w_v[TGRAD_MAX_NDIM], w_rot[TGRAD_MAX_NDIM], w_log[TGRAD_MAX_NDIM], w_lam[TGRAD_MAX_NDIM], w_partial, w_total;
   bool jac_fast[TGRAD_MAX_NDIM];    // eigensolver with the matrix in shared memory and a rotation log
   uint64_t numel, P, tsize;   // entries, core entries, entries of the tail-contracted tensor
   uint32_t nblk;              // compaction blocks
@@ -74,6 +74,7 @@ tgrad_status validate(const tgrad_config* c) {
   if (!(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps >= 0.f))
     return TGRAD_ERR_INVALID_ARG;
   if (c->jacobi_max_sweeps < 0 || c->jacobi_tol < 0.f) return TGRAD_ERR_INVALID_ARG;
+  if (c->warm_refresh != 0 && c->warm_refresh != 1) return TGRAD_ERR_INVALID_ARG;
   // limits of this implementation
   if (c->ndim < 3) return TGRAD_ERR_UNSUPPORTED;             // the matrix case is not built
   if (tot >= 4294967296.0L) return TGRAD_ERR_UNSUPPORTED;    // flat indices are uint32
@@ -121,6 +122,11 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
   L.p_vs = o; o = align_up(o + k * 4);
   // operand-fragment table of the compression kernel: 32 lanes x 32 bytes per (8-row tile, 8-column tile) of U^(N-1)
   L.p_u2tab = o; o = align_up(o + (size_t)((c->dims[N - 2] + 7) / 8) * ((c->ranks[N - 2] + 7) / 8) * 1024);
+  // warm-started refresh: the eigenvector basis of each mode's last refresh (modes the rotation-log solver handles)
+  for (int n = 0; n < N; ++n) {
+    L.p_basis[n] = o;
+    if (c->warm_refresh && c->dims[n] <= JAC_FAST_MAX_N) o = align_up(o + (size_t)c->dims[n] * c->dims[n] * 8);
+  }
   L.p_total = o;
   o = 0;
   L.w_ns = o; o = align_up(o + k * 8);
@@ -139,6 +145,7 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
     L.w_gram[n] = o; o = align_up(o + sq);   // A_n, kept for inspection
     L.w_jac[n] = o; o = align_up(o + (size_t)c->dims[n] * (c->dims[n] | 1) * 8);    // working copy the solver diagonalises
     L.w_v[n] = o; o = align_up(o + sq);      // accumulated rotations
+    L.w_rot[n] = o; if (c->warm_refresh) o = align_up(o + sq);   // A_n rotated into the previous basis
     const int sweeps = c->jacobi_max_sweeps > 0 ? c->jacobi_max_sweeps : 30;
     const size_t logb = jac_log_entries((int)c->dims[n], sweeps) * sizeof(float4);
     L.jac_fast[n] = c->dims[n] <= JAC_FAST_MAX_N && logb <= ((size_t)64 << 20);
@@ -162,6 +169,7 @@ struct tgrad_state {
   char* dw;
   int64_t t;
   bool have_subspace;
+  bool basis_valid;     // warm-started refresh: the persistent block holds the bases of a previous refresh
   bool tabs_stale;      // U^(N-1) changed since the compression kernel's fragment table was built
   int sm_count;
   TailPlan tail;
@@ -374,6 +382,18 @@ tgrad_status build_slab_ptr(tgrad_state* s, cudaStream_t st) {
   return TGRAD_OK;
 }
 
+#define TG_TRY(x) do { tgrad_status _s = (x); if (_s != TGRAD_OK) return _s; } while (0)
+
+// out[m][c] = sum_k Aop[m][k] in[k][c] for the small square matrices of the warm-started refresh, in fp32 FMAs:
+// Aop = U (M x K, row-major) or, with conj_t, Aop = U^H for U of K x M.
+tgrad_status small_product(bool conj_t, const cf* in, cf* out, const cf* U, int M, int K, int C, cudaStream_t st) {
+  dim3 grid((unsigned)((C + 31) / 32), (unsigned)((M + MP_BM - 1) / MP_BM), 1);
+  if (conj_t) mode_product_kernel<true, 32><<<grid, MP_THREADS, 0, st>>>(in, out, U, M, K, C, M);
+  else mode_product_kernel<false, 32><<<grid, MP_THREADS, 0, st>>>(in, out, U, M, K, C, K);
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
+}
+
 template <class S>
 tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   const tgrad_config& c = s->cfg;
@@ -435,6 +455,22 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
       fm.log = reinterpret_cast<float4*>(s->dw + L.w_log[m]);
       fm.lam = reinterpret_cast<float*>(s->dw + L.w_lam[m]);
       fm.V = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
+      if (c.warm_refresh) {
+        cf* V = reinterpret_cast<cf*>(s->dp + L.p_basis[m]);
+        fm.V = V;                                       // the solver leaves this refresh's eigenvectors there
+        if (s->basis_valid) {
+          // V <- V (3/2 I - 1/2 V^H V), then A' = V^H A V is what gets diagonalised; its rotations are applied to V
+          cf* t1 = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
+          cf* t2 = reinterpret_cast<cf*>(s->dw + L.w_rot[m]);
+          TG_TRY(small_product(true, V, t1, V, In, In, In, st));          // G = V^H V
+          ns_residual_kernel<<<(In * In + 255) / 256, 256, 0, st>>>(t1, In); TG_LAUNCH_CHECK();
+          TG_TRY(small_product(false, t1, t2, V, In, In, In, st));        // V E
+          if (cudaMemcpyAsync(V, t2, (size_t)In * In * 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return TGRAD_ERR_CUDA;
+          TG_TRY(small_product(false, V, t1, A, In, In, In, st));         // A V
+          TG_TRY(small_product(true, t1, t2, V, In, In, In, st));         // V^H (A V)
+          fm.A = t2;
+        }
+      }
       fm.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
       fm.n = In; fm.r = c.ranks[m]; fm.index = m; fm.row0 = fp.total_rows;
       fp.total_rows += In;
@@ -459,6 +495,7 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   }
   if (fp.nmodes) {
     fp.max_sweeps = max_sweeps; fp.tol = tol; fp.flags = flags;
+    fp.warm = (c.warm_refresh && s->basis_valid) ? 1 : 0;
     // the sweeps: modes whose matrix fits in shared memory in one launch, the larger ones (matrix in L2) in another
     JacobiFastParams fs = fp, fg = fp;
     fs.nmodes = fg.nmodes = 0;
@@ -479,6 +516,7 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   }
   s->have_subspace = true;
   s->tabs_stale = true;
+  if (c.warm_refresh) s->basis_valid = true;
   return TGRAD_OK;
 }
 
@@ -503,7 +541,6 @@ tgrad_status mode_product(bool conj_t, const cf* in, cf* out, const cf* U, uint6
   return TGRAD_OK;
 }
 
-#define TG_TRY(x) do { tgrad_status _s = (x); if (_s != TGRAD_OK) return _s; } while (0)
 #define TG_MARK(i) do { if (evs) cudaEventRecord(evs[i], st); } while (0)
 
 tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t st) {
@@ -666,7 +703,7 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
   memset(st, 0, sizeof(*st));
   st->cfg = *cfg; st->L = L;
   st->dp = static_cast<char*>(d_persistent); st->dw = static_cast<char*>(d_workspace);
-  st->t = 0; st->have_subspace = false; st->tabs_stale = true;
+  st->t = 0; st->have_subspace = false; st->tabs_stale = true; st->basis_valid = false;
   int dev = 0, sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }

@@ -40,7 +40,7 @@ def storage_exact(x: np.ndarray, half: bool) -> np.ndarray:
 
 
 class Pair:
-    def __init__(self, wl: synth.Workload, tensor_id=0, **over):
+    def __init__(self, wl: synth.Workload, tensor_id=0, warm_refresh=False, **over):
         self.wl = wl
         self.src = synth.GradientSource(wl, tensor_id)
         kw = dict(lr=wl.lr, alpha=1.0, lam=1.0, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
@@ -48,7 +48,8 @@ class Pair:
         self.half = wl.half_storage
         self.ocfg = orc.OracleConfig(shape=wl.shape, ranks=wl.ranks, k=wl.k, T=wl.T, half_storage=self.half, **kw)
         self.ost = orc.OracleState(self.ocfg)
-        self.gcfg = B.make_config(wl.shape, wl.ranks, wl.k, wl.T, half_storage=self.half, auto_refresh=False, **kw)
+        self.gcfg = B.make_config(wl.shape, wl.ranks, wl.k, wl.T, half_storage=self.half, auto_refresh=False,
+                                  warm_refresh=warm_refresh, **kw)
         self.gst = B.TgradState(self.gcfg)
         w0 = storage_exact(self.src.weight(), self.half)
         self.w_ref = w0
@@ -192,11 +193,12 @@ class SampledChecker:
     """Refresh + steps at full size, checked on sampled outputs and on everything that is
     element-wise (both Adam updates), using the GPU's own exported inputs for each stage."""
 
-    def __init__(self, wl: synth.Workload, tensor_id=0, n_samples=6, seed=0):
+    def __init__(self, wl: synth.Workload, tensor_id=0, n_samples=6, seed=0, warm_refresh=False):
         self.wl = wl
         self.half = wl.half_storage
         self.src = synth.GradientSource(wl, tensor_id)
-        self.cfg = B.make_config(wl.shape, wl.ranks, wl.k, wl.T, lr=wl.lr, half_storage=self.half, auto_refresh=False)
+        self.cfg = B.make_config(wl.shape, wl.ranks, wl.k, wl.T, lr=wl.lr, half_storage=self.half, auto_refresh=False,
+                                 warm_refresh=warm_refresh)
         self.st = B.TgradState(self.cfg)
         self.w = storage_exact(self.src.weight(), self.half)
         self.w_dev = to_device(self.w, self.half)
@@ -239,11 +241,11 @@ class SampledChecker:
             assert od <= TOL_ORTHO, (n, od)
         return r
 
-    def step(self):
+    def step(self, refresh=False):
         wl, t = self.wl, self.t
         g = storage_exact(self.src.gradient(t), self.half)
         g_dev = to_device(g, self.half)
-        if t % wl.T == 0:
+        if t % wl.T == 0 or refresh:
             r = self.refresh(g, g_dev)
         else:
             r = orc.residual(g, self.omega)

@@ -29,6 +29,17 @@ def test_trajectory_cfg1_full():
     print("cfg1", p.report)
 
 
+@pytest.mark.parametrize("name", ["small4", "ragged4", "odd32", "cfg1"])
+def test_trajectory_warm_refresh(name):
+    # every refresh after the first starts the eigensolver from the previous eigenvectors: same subspaces, same
+    # orthonormality, same trajectory tolerances
+    wl = synth.WORKLOADS[name]
+    p = Pair(wl, warm_refresh=True)
+    for t in range(max(wl.steps, 3 * wl.T + 1)):
+        p.step(t)
+    print(name, p.report)
+
+
 def test_alpha_lambda_weight_decay():
     wl = synth.WORKLOADS["small4"]
     p = Pair(wl, alpha=0.25, lam=0.5, weight_decay=0.1, lr=1e-2)
