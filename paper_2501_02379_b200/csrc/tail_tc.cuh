@@ -113,7 +113,7 @@ __device__ __forceinline__ void tc_issue_load(const unsigned char* gbase, unsign
 // RAT = ceil(ra/8); KS = k-steps of stage 1 (>= tc_ksteps(B)).
 // ---------------------------------------------------------------------------------------------
 
-__host__ inline bool proj_tc_geom(int A, int B, int rat, uint32_t nslab, int ntw, int PJ_WARPS, uint32_t smem_per_block, TcGeom& g) {
+__host__ inline bool proj_tc_geom(int A, int B, int rat, uint32_t nslab, int ntw, int PJ_WARPS, uint32_t smem_per_block, TcGeom& g) {   // PJ_WARPS: warps per block
   if (A % 8) return false;
   const int tiles = A / 8;
   // tps = warps per slab, each with ntw row tiles; spi = slabs per group
@@ -154,16 +154,24 @@ __global__ void proj_u2tab_kernel(const cf* __restrict__ Ua, int A, int ra, int 
   tab[2 * idx + 1] = make_float4(l0.x, l0.y, l1.x, l1.y);
 }
 
-template <int RAT, int KS, int NTW, int PJ_WARPS>
-__global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW <= 2 ? 4 : 3)) proj_tail_tc_kernel(const void* __restrict__ g, TailTcParams P) {
+constexpr int PJ_WARPS = 4;
+
+// TW = warps per slab (row tiles of a slab / NTW): 4, 2 or 1, so a group has PJ_WARPS / TW slabs
+template <int RAT, int KS, int NTW, int TW>
+__global__ void __launch_bounds__(32 * PJ_WARPS, NTW <= 2 ? 4 : 3) proj_tail_tc_kernel(const void* __restrict__ g, TailTcParams P) {
   griddep_chain();
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int PJ_THREADS = 32 * PJ_WARPS;
   const TailParams& p = P.p;
   const TcGeom& G = P.g;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t = lane & 3;
-  const int B = p.B, ra = p.ra, rb = p.rb, twoB = 2 * B, nbuf = G.nbuf, spi = G.spi, tw = G.tps;
-  const uint32_t E = p.E, nslab = p.nslab, ngroups = G.ngroups, gstride = gridDim.x;
+  constexpr int tw = TW, spi = PJ_WARPS / TW;
+  // an odd KS fixes B = 4 (KS - 1) + 1 and NTW * TW fixes the rows of a slab, so that every offset into a slab
+  // is an immediate
+  const int B = (KS & 1) ? 4 * (KS - 1) + 1 : p.B;
+  const int ra = p.ra, rb = p.rb, twoB = 2 * B, nbuf = G.nbuf;
+  const uint32_t E = (KS & 1) ? (uint32_t)(8 * NTW * TW * (4 * (KS - 1) + 1)) : p.E;
+  const uint32_t nslab = p.nslab, ngroups = G.ngroups, gstride = gridDim.x;
   const int q = warp / tw, wt = warp - q * tw;
   constexpr int REDW = RAT * 128;                       // floats of one warp's partial: [8 RAT][8] complex
   float* red = reinterpret_cast<float*>(smem + G.off_aux);   // [2][PJ_WARPS][REDW]
@@ -238,6 +246,7 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, PJ_WARPS == 8 ? 2 : (NTW <= 2 ?
       if (o_src[i] >= 0 && up * spi + o_q[i] < nslab) {
         const float* src = rp + o_src[i];
         float acc = src[0];
+#pragma unroll
         for (int w = 1; w < tw; ++w) acc += src[(size_t)w * REDW];
         tg_[o_dst[i]] = acc;
       }

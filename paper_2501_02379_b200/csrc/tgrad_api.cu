@@ -220,21 +220,23 @@ tgrad_status tail_any(const tgrad_state* s, int op, void* ptr, const TailParams&
                                       : tail_dispatch<StoreC32H>(op, s->tail, ptr, p, st);
 }
 
-template <int RAT, int KS, int NTW, int W>
+template <int RAT, int KS, int NTW, int TW>
 tgrad_status tc_proj_op2(int op, const TailPlan& tp, const void* g, const TailTcParams& P, cudaStream_t st) {
   if (op == 0) {
-    return cudaFuncSetAttribute(proj_tail_tc_kernel<RAT, KS, NTW, W>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(proj_tail_tc_kernel<RAT, KS, NTW, TW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)tp.gproj.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
   }
-  launch_chained(proj_tail_tc_kernel<RAT, KS, NTW, W>, dim3(tp.grid_proj), dim3(32 * W), tp.gproj.total, st, g, P);
+  launch_chained(proj_tail_tc_kernel<RAT, KS, NTW, TW>, dim3(tp.grid_proj), dim3(32 * PJ_WARPS), tp.gproj.total, st, g, P);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
 template <int RAT, int KS>
 tgrad_status tc_proj_op(int op, const TailPlan& tp, const void* g, const TailTcParams& P, cudaStream_t st) {
-  if (tp.pjw == 8) return tc_proj_op2<RAT, KS, 1, 8>(op, tp, g, P, st);
-  if (tp.ntw == 4) return tc_proj_op2<RAT, KS, 4, 4>(op, tp, g, P, st);
-  return tp.ntw == 2 ? tc_proj_op2<RAT, KS, 2, 4>(op, tp, g, P, st) : tc_proj_op2<RAT, KS, 1, 4>(op, tp, g, P, st);
+  // (row tiles per warp, warps per slab): 64 rows -> (2, 4), 32 rows -> (4, 1), 16 rows -> (2, 1)
+  if (tp.ntw == 4 && tp.gproj.tps == 1) return tc_proj_op2<RAT, KS, 4, 1>(op, tp, g, P, st);
+  if (tp.ntw == 2 && tp.gproj.tps == 4) return tc_proj_op2<RAT, KS, 2, 4>(op, tp, g, P, st);
+  if (tp.ntw == 2 && tp.gproj.tps == 1) return tc_proj_op2<RAT, KS, 2, 1>(op, tp, g, P, st);
+  return TGRAD_ERR_UNSUPPORTED;
 }
 template <int RAT, int NS>
 tgrad_status tc_back_op2(int op, const TailPlan& tp, void* w, const TailTcParams& P, cudaStream_t st) {
@@ -334,7 +336,7 @@ tgrad_status plan_tail(tgrad_state* s) {
     // 8 warps with one tile each: 101 against 122 us on 128x128x64x33)
     tp.pjw = 4; tp.ntw = (A == 64) ? 2 : (A == 32 ? 4 : 2);
     tp.back_ns = ((uint64_t)A * B * 8 <= 8192) ? 2 : 1;      // small slabs: two per warp and iteration
-    const int pj_blocks = tp.pjw == 8 ? 2 : (tp.ntw <= 2 ? 4 : 3);     // resident blocks per SM
+    const int pj_blocks = tp.ntw <= 2 ? 4 : 3;     // resident blocks per SM
     const uint32_t pj_smem = (227u * 1024u) / pj_blocks - 1024u;
     if (proj_tc_geom(A, B, rat, (uint32_t)S, tp.ntw, tp.pjw, pj_smem, tp.gproj) && tail_tc_geom(true, A, B, rat, (uint32_t)S, tp.back_ns, tp.gback)) {
       const uint32_t cap = 2u * (uint32_t)s->sm_count, pcap = (uint32_t)pj_blocks * (uint32_t)s->sm_count;
