@@ -558,23 +558,26 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
       // ---- stage 1: Y'[a][(c, jb)] for rows r0 and r1; hi*hi, lo*hi and hi*lo accumulate separately ----
       float d1[2][3][4];
 #pragma unroll
-      for (int c = 0; c < 2; ++c)
-#pragma unroll
-        for (int m = 0; m < 3; ++m)
-#pragma unroll
-          for (int i = 0; i < 4; ++i) d1[c][m][i] = 0.f;
-#pragma unroll
       for (int ks = 0; ks < KS2; ++ks) {
         float trh, trl, tih, til;
         split_tf32(tv[i][ks].x, trh, trl); split_tf32(tv[i][ks].y, tih, til);
         const float* a = ua[ks];
         // A = (Ua[r0].re, Ua[r1].re, Ua[r0].im, Ua[r1].im);  re tile: B = (Tr, -Ti);  im tile: B = (Ti, Tr)
-        mma_tf32(d1[0][0], a[0], a[1], a[2], a[3], trh, -tih);
-        mma_tf32(d1[0][1], a[4], a[5], a[6], a[7], trh, -tih);
-        mma_tf32(d1[0][2], a[0], a[1], a[2], a[3], trl, -til);
-        mma_tf32(d1[1][0], a[0], a[1], a[2], a[3], tih, trh);
-        mma_tf32(d1[1][1], a[4], a[5], a[6], a[7], tih, trh);
-        mma_tf32(d1[1][2], a[0], a[1], a[2], a[3], til, trl);
+        if (ks == 0) {
+          mma_tf32_z(d1[0][0], a[0], a[1], a[2], a[3], trh, -tih);
+          mma_tf32_z(d1[0][1], a[4], a[5], a[6], a[7], trh, -tih);
+          mma_tf32_z(d1[0][2], a[0], a[1], a[2], a[3], trl, -til);
+          mma_tf32_z(d1[1][0], a[0], a[1], a[2], a[3], tih, trh);
+          mma_tf32_z(d1[1][1], a[4], a[5], a[6], a[7], tih, trh);
+          mma_tf32_z(d1[1][2], a[0], a[1], a[2], a[3], til, trl);
+        } else {
+          mma_tf32(d1[0][0], a[0], a[1], a[2], a[3], trh, -tih);
+          mma_tf32(d1[0][1], a[4], a[5], a[6], a[7], trh, -tih);
+          mma_tf32(d1[0][2], a[0], a[1], a[2], a[3], trl, -til);
+          mma_tf32(d1[1][0], a[0], a[1], a[2], a[3], tih, trh);
+          mma_tf32(d1[1][1], a[4], a[5], a[6], a[7], tih, trh);
+          mma_tf32(d1[1][2], a[0], a[1], a[2], a[3], til, trl);
+        }
       }
       // Y' as stage-2 A fragments: a0 = d[0] (row g, jb), a1 = d[2] (row g+8, jb), a2 = d[1] (row g, jb+1), a3 = d[3]
       float yh[2][4], yl[2][4];
@@ -588,10 +591,10 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
 #pragma unroll 3
       for (int nb = 0; nb < nbt; ++nb) {
         const float4 fr = ubf[(nb * 2 + 0) * 32 + lane], fi = ubf[(nb * 2 + 1) * 32 + lane];
-        float dh[4] = {0.f, 0.f, 0.f, 0.f}, dl[4] = {0.f, 0.f, 0.f, 0.f}, dx[4] = {0.f, 0.f, 0.f, 0.f};
-        mma_tf32(dh, yh[0][0], yh[0][2], yh[0][1], yh[0][3], fr.x, fr.y);
-        mma_tf32(dl, yl[0][0], yl[0][2], yl[0][1], yl[0][3], fr.x, fr.y);
-        mma_tf32(dx, yh[0][0], yh[0][2], yh[0][1], yh[0][3], fr.z, fr.w);
+        float dh[4], dl[4], dx[4];
+        mma_tf32_z(dh, yh[0][0], yh[0][2], yh[0][1], yh[0][3], fr.x, fr.y);
+        mma_tf32_z(dl, yl[0][0], yl[0][2], yl[0][1], yl[0][3], fr.x, fr.y);
+        mma_tf32_z(dx, yh[0][0], yh[0][2], yh[0][1], yh[0][3], fr.z, fr.w);
         mma_tf32(dh, yh[1][0], yh[1][2], yh[1][1], yh[1][3], fi.x, fi.y);
         mma_tf32(dl, yl[1][0], yl[1][2], yl[1][1], yl[1][3], fi.x, fi.y);
         mma_tf32(dx, yh[1][0], yh[1][2], yh[1][1], yh[1][3], fi.z, fi.w);
