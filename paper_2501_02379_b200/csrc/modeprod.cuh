@@ -157,7 +157,6 @@ __device__ __forceinline__ void mt_split(float x, float& hi, float& lo) {
 template <bool CONJ_T, int NT>
 __global__ void __launch_bounds__(MT_THREADS) mode_product_tc_kernel(const cf* __restrict__ in, cf* __restrict__ out,
                                                                      const cf* __restrict__ U, int M, int K, int C, int r_n) {
-  griddep_chain();
   constexpr int BC = 32 * NT, LDX = BC + 4;      // X tile row length: rows 4 slots apart in the 16 bank pairs
   __shared__ __align__(16) float4 As[2][MT_BM][MT_LDA];   // (re.hi, im.hi, re.lo, im.lo) of Aop[m][k]
   __shared__ __align__(16) cf Xs[2][MT_BK][LDX];
@@ -224,7 +223,8 @@ __global__ void __launch_bounds__(MT_THREADS) mode_product_tc_kernel(const cf* _
 #pragma unroll
       for (int i = 0; i < 4; ++i) tot[mt][nt][i] = 0.f;
 
-  fetch_a(0);
+  fetch_a(0);                 // U only: in flight while the previous kernel drains
+  griddep_chain();
   load_x(0, 0);
   stash_a(0);
   int buf = 0;
@@ -305,9 +305,9 @@ __global__ void __launch_bounds__(SW_THREADS) core_sandwich_tc_kernel(const cf* 
                                                                       const cf* __restrict__ g_s, cf* __restrict__ m_s,
                                                                       float* __restrict__ v_s, cf* __restrict__ n_s, uint32_t ks,
                                                                       uint32_t nblk_core, AdamScalars a) {
-  griddep_chain();
   extern __shared__ __align__(16) unsigned char swm[];
   if (blockIdx.x >= nblk_core) {
+    griddep_chain();
     const uint32_t i = (blockIdx.x - nblk_core) * SW_THREADS + threadIdx.x;
     if (i < ks) {
       cf m = m_s[i]; float v = v_s[i];
@@ -322,13 +322,14 @@ __global__ void __launch_bounds__(SW_THREADS) core_sandwich_tc_kernel(const cf* 
   cf* Us = Xs + (size_t)I1p * SWT_LDX;                 // [I1p][ldu], zero padded
   cf* Cs = Us + (size_t)I1p * ldu;                     // [r1p][SWT_LDX]: the core block, then N
   const int c0 = blockIdx.x * SW_CB;
-  for (int idx = tid; idx < I1p * SW_CB; idx += SW_THREADS) {
-    const int i = idx / SW_CB, cc = idx - i * SW_CB;
-    Xs[i * SWT_LDX + cc] = (i < I1 && c0 + cc < C) ? X[(size_t)i * C + c0 + cc] : make_float2(0.f, 0.f);
-  }
   for (int idx = tid; idx < I1p * (ldu - 4); idx += SW_THREADS) {
     const int i = idx / (ldu - 4), j = idx - i * (ldu - 4);
     Us[i * ldu + j] = (i < I1 && j < r1) ? U1[(size_t)i * r1 + j] : make_float2(0.f, 0.f);
+  }
+  griddep_chain();            // U1 alone was read so far; X is the previous kernel's output
+  for (int idx = tid; idx < I1p * SW_CB; idx += SW_THREADS) {
+    const int i = idx / SW_CB, cc = idx - i * SW_CB;
+    Xs[i * SWT_LDX + cc] = (i < I1 && c0 + cc < C) ? X[(size_t)i * C + c0 + cc] : make_float2(0.f, 0.f);
   }
   __syncthreads();
   // ---- core[j][c] = sum_i conj(U1[i][j]) X[i][c]: rows (j, re|im), k = (i, re|im) ----

@@ -109,9 +109,11 @@ __device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1,
 // soon as every block of this grid has got this far.  Both are no-ops in a kernel launched the ordinary way.
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-// What every kernel of the step starts with: nothing in global memory is touched before the predecessor is done,
-// so only the launch itself and the scheduling of the blocks overlap with the predecessor's tail.
-__device__ __forceinline__ void griddep_chain() { griddep_launch_dependents(); griddep_wait(); }
+// What every kernel of the step runs before it touches anything a kernel of the same step writes.  The wait comes
+// first, so that a kernel's successor is not scheduled before the kernel's own predecessor has completed: code that
+// a kernel runs before this call therefore overlaps with its immediate predecessor only, and may read what earlier
+// launches wrote (the factor matrices, which only a refresh changes) but nothing of the step, and write nothing.
+__device__ __forceinline__ void griddep_chain() { griddep_wait(); griddep_launch_dependents(); }
 
 // 16-byte read-only load that the compiler neither hoists out of a loop nor merges with its repeats.
 __device__ __forceinline__ float4 ld_nc_f4_volatile(const float4* p) {

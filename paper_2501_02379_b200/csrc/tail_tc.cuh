@@ -159,7 +159,6 @@ constexpr int PJ_WARPS = 4;
 // TW = warps per slab (row tiles of a slab / NTW): 4, 2 or 1, so a group has PJ_WARPS / TW slabs
 template <int RAT, int KS, int NTW, int TW>
 __global__ void __launch_bounds__(32 * PJ_WARPS, NTW <= 2 ? 4 : 3) proj_tail_tc_kernel(const void* __restrict__ g, TailTcParams P) {
-  griddep_chain();
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int PJ_THREADS = 32 * PJ_WARPS;
   const TailParams& p = P.p;
@@ -214,6 +213,7 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, NTW <= 2 ? 4 : 3) proj_tail_tc_
     fence_mbar_init();
   }
   __syncthreads();
+  griddep_chain();            // so far only Ub was read: the tables are built while the previous kernel drains
   if (tid == 0) {
     uint32_t u = blockIdx.x;
     for (int i = 0; i < nbuf && u < ngroups; ++i, u += gstride) tc_issue_load(gb, smem, G, bars, u, i, nslab);
@@ -413,7 +413,6 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, NTW <= 2 ? 4 : 3) proj_tail_tc_
 // ---------------------------------------------------------------------------------------------
 template <int RAT, int NS>
 __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __restrict__ w, TailTcParams P) {
-  griddep_chain();
   extern __shared__ __align__(128) unsigned char smem[];
   const TailParams& p = P.p;
   const TcGeom& G = P.g;
@@ -461,6 +460,7 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
     fence_mbar_init();
   }
   __syncthreads();
+  griddep_chain();            // so far only Ua and Ub were read: the operand tables are built while the previous kernel drains
   if (tid == 0) {
     uint32_t u = blockIdx.x;
     for (int i = 0; i < la && u < ngroups; ++i, u += gstride) tc_issue_load(wb, smem, G, bars, u, i, nslab);
