@@ -158,7 +158,7 @@ constexpr int PJ_WARPS = 4;
 
 // TW = warps per slab (row tiles of a slab / NTW): 4, 2 or 1, so a group has PJ_WARPS / TW slabs
 template <int RAT, int KS, int NTW, int TW>
-__global__ void __launch_bounds__(32 * PJ_WARPS, NTW <= 2 ? 4 : 3) proj_tail_tc_kernel(const void* __restrict__ g, TailTcParams P) {
+__global__ void __launch_bounds__(32 * PJ_WARPS, 4) proj_tail_tc_kernel(const void* __restrict__ g, TailTcParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
   constexpr int PJ_THREADS = 32 * PJ_WARPS;
   const TailParams& p = P.p;

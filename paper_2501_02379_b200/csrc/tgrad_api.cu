@@ -336,7 +336,7 @@ tgrad_status plan_tail(tgrad_state* s) {
     // 8 warps with one tile each: 101 against 122 us on 128x128x64x33)
     tp.pjw = 4; tp.ntw = (A == 64) ? 2 : (A == 32 ? 4 : 2);
     tp.back_ns = ((uint64_t)A * B * 8 <= 8192) ? 2 : 1;      // small slabs: two per warp and iteration
-    const int pj_blocks = tp.ntw <= 2 ? 4 : 3;     // resident blocks per SM
+    const int pj_blocks = 4;     // resident blocks per SM
     const uint32_t pj_smem = (227u * 1024u) / pj_blocks - 1024u;
     if (proj_tc_geom(A, B, rat, (uint32_t)S, tp.ntw, tp.pjw, pj_smem, tp.gproj) && tail_tc_geom(true, A, B, rat, (uint32_t)S, tp.back_ns, tp.gback)) {
       const uint32_t cap = 2u * (uint32_t)s->sm_count, pcap = (uint32_t)pj_blocks * (uint32_t)s->sm_count;
