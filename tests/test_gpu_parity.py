@@ -168,6 +168,36 @@ def test_export_import_resume_bitwise():
     assert a.query_status()[1] == b.query_status()[1] == total
 
 
+def test_factors_imported_mid_run_take_effect():
+    # a state that has already stepped (so every table derived from the factors exists) gets new factors through the
+    # C ABI; its next step must equal, bit for bit, that of a fresh state given the same factors from the start
+    wl = synth.WORKLOADS["odd32"]                # 32 x 17 slabs: the tensor-core streaming kernels
+    src = synth.GradientSource(wl)
+    cfg = B.make_config(wl.shape, wl.ranks, wl.k, wl.T, auto_refresh=False)
+    a = B.TgradState(cfg)
+    wa = to_device(src.weight(), False)
+    a.refresh_subspace(to_device(src.gradient(0), False))
+    for t in range(2):
+        a.step(wa, to_device(src.gradient(t), False))
+    rng = np.random.default_rng(5)
+    new_u = [H.random_orthonormal(rng, i, r).astype(np.complex64) for i, r in zip(wl.shape, wl.ranks)]
+    for n, u in enumerate(new_u):
+        a.import_(B.WHAT_FACTOR_BASE + n, u)
+    b = B.TgradState(B.make_config(wl.shape, wl.ranks, wl.k, wl.T, auto_refresh=False))
+    for w in (B.WHAT_OMEGA, B.WHAT_M_L, B.WHAT_V_L, B.WHAT_M_S, B.WHAT_V_S):
+        b.import_(w, a.export(w))
+    for n, u in enumerate(new_u):
+        b.import_(B.WHAT_FACTOR_BASE + n, u)
+    b.set_step(2)
+    wb = wa.clone()
+    g = src.gradient(2)
+    a.step(wa, to_device(g, False))
+    b.step(wb, to_device(g, False))
+    assert torch.equal(wa, wb)
+    for w in (B.WHAT_M_L, B.WHAT_V_L, B.WHAT_CORE):
+        assert np.array_equal(a.export(w), b.export(w))
+
+
 def test_batched_matches_single():
     wl = synth.WORKLOADS["small4"]
     srcs = [synth.GradientSource(wl, i) for i in range(3)]
