@@ -332,8 +332,8 @@ tgrad_status plan_tail(tgrad_state* s) {
   const double dec = 1.0 - (double)c.lr * (double)c.weight_decay;
   if (c.wg_dtype == TGRAD_C64 && (A == 16 || A == 32 || A == 64) && rat <= 2 && rb <= 8 && ks && dec > 0.0) {
     tp.rat = rat; tp.ks = ks;
-    // compression kernel: blocks of 4 warps; two row tiles per warp for 64-row slabs (measured faster than
-    // 8 warps with one tile each: 101 against 122 us on 128x128x64x33)
+    // compression kernel: blocks of 4 warps; two row tiles per warp for 64-row and 16-row slabs, four for 32-row
+    // slabs (measured: two tiles per warp there, two warps per slab, 218 against 200 us on 64x64x32x32x17)
     tp.pjw = 4; tp.ntw = (A == 64) ? 2 : (A == 32 ? 4 : 2);
     tp.back_ns = ((uint64_t)A * B * 8 <= 8192) ? 2 : 1;      // small slabs: two per warp and iteration
     const int pj_blocks = 4;     // resident blocks per SM
@@ -601,8 +601,8 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   TG_MARK(1);
   // the chain on the small tensor: compression of modes N-2 .. 2, then mode 1 + Adam + mode 1 in one
   // launch (or three when the first mode is too large for it), then reconstruction of modes 2 .. N-2
-  // (the fused launch does its two products with fp32 FMAs: beyond 64 M complex multiply-adds per product the
-  //  tensor-core GEMM launches win even with the extra round trips)
+  // (the fused launch holds all of U^(1) and a 16-column block in shared memory and serialises its two products:
+  //  beyond 64 M complex multiply-adds per product separate GEMM launches win even with the extra round trips)
   uint64_t c_first = (uint64_t)ra * rb;
   for (int q = 1; q <= N - 3; ++q) c_first *= c.ranks[q];
   const bool fused = c.dims[0] <= SW_MAX_I && c.ranks[0] <= SW_MAX_R &&
