@@ -192,9 +192,9 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
       }
 }
 
-// Sum the split-K partials, always in the same order (four interleaved running sums per entry, then
-// those four in order): deterministic.  Mirrors the upper triangle.
-constexpr int GRR_E = 64, GRR_G = 4;     // entries per block, split groups
+// Sum the split-K partials, always in the same order (sixteen interleaved running sums per entry, then
+// those in order): deterministic.  Mirrors the upper triangle.
+constexpr int GRR_E = 64, GRR_G = 16;    // entries per block, split groups
 __global__ void __launch_bounds__(GRR_E * GRR_G) gram_reduce_kernel(const cf* __restrict__ partial, int splits, int In,
                                                                    cf* __restrict__ A) {
   __shared__ cf part[GRR_G][GRR_E];
