@@ -41,20 +41,30 @@ __global__ void __launch_bounds__(512) sel_hist_kernel(const void* __restrict__ 
   const uint32_t prefix = st->prefix;
   const uint32_t hi_mask = (pass == 0) ? 0u : (0xffffffffu << (shift + bits));
   bool bad = false;
-  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  constexpr int UN = 4;                       // entries per thread and iteration: their loads are issued together
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x * UN;
   // block-uniform loop bound, so every warp stays converged for the warp votes below
-  for (uint64_t b0 = (uint64_t)blockIdx.x * blockDim.x; b0 < n; b0 += stride) {
-    const uint64_t i = b0 + threadIdx.x;
-    const bool valid = i < n;
-    uint32_t key = valid ? mag_key(S::load(g, i)) : 0u;
-    if (pass == 0 && (key & 0x7f800000u) == 0x7f800000u) bad = true;
-    bool in = valid && (key & hi_mask) == prefix;
-    uint32_t d = (key >> shift) & (nb - 1u);
-    // warp-aggregated shared atomics: gradients crowd into a few exponent bins
-    unsigned act = __ballot_sync(0xffffffffu, in);
-    if (in) {
-      unsigned peers = __match_any_sync(act, d);
-      if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&sh[d], (uint32_t)__popc(peers));
+  for (uint64_t b0 = (uint64_t)blockIdx.x * blockDim.x * UN; b0 < n; b0 += stride) {
+    uint32_t keys[UN];
+    bool valid[UN];
+#pragma unroll
+    for (int j = 0; j < UN; ++j) {
+      const uint64_t i = b0 + (uint64_t)j * blockDim.x + threadIdx.x;
+      valid[j] = i < n;
+      keys[j] = valid[j] ? mag_key(S::load(g, i)) : 0u;
+    }
+#pragma unroll
+    for (int j = 0; j < UN; ++j) {
+      const uint32_t key = keys[j];
+      if (pass == 0 && (key & 0x7f800000u) == 0x7f800000u) bad = true;
+      bool in = valid[j] && (key & hi_mask) == prefix;
+      uint32_t d = (key >> shift) & (nb - 1u);
+      // warp-aggregated shared atomics: gradients crowd into a few exponent bins
+      unsigned act = __ballot_sync(0xffffffffu, in);
+      if (in) {
+        unsigned peers = __match_any_sync(act, d);
+        if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&sh[d], (uint32_t)__popc(peers));
+      }
     }
   }
   __syncthreads();
