@@ -117,6 +117,48 @@ __global__ void __launch_bounds__(MP_THREADS) mode_product_kernel(const cf* __re
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same product for few output rows (M <= 8) and slices whose K C entries fit in shared memory: the 32-row
+// tensor-core tiles would be mostly padding there.  A block walks over slices o;
+// the slice [K][C] and Aop sit in shared memory, a thread owns outputs (m, c) and sums over k in fp32.
+// ---------------------------------------------------------------------------------------------
+constexpr int MS_THREADS = 256;
+__host__ __device__ inline size_t mode_small_smem(int M, int K, int C) { return ((size_t)K * C + (size_t)M * K) * sizeof(cf); }
+
+template <bool CONJ_T>
+__global__ void __launch_bounds__(MS_THREADS) mode_product_small_kernel(const cf* __restrict__ in, cf* __restrict__ out,
+                                                                        const cf* __restrict__ U, int M, int K, int C,
+                                                                        int r_n, int O) {
+  extern __shared__ __align__(16) unsigned char msm[];
+  cf* Xs = reinterpret_cast<cf*>(msm);           // [K][C]
+  cf* As = Xs + (size_t)K * C;                   // [M][K]
+  const int tid = threadIdx.x;
+  for (int idx = tid; idx < M * K; idx += MS_THREADS) {
+    const int m = idx / K, k = idx - m * K;
+    cf v;
+    if (CONJ_T) { const cf u = U[(size_t)k * r_n + m]; v = make_float2(u.x, -u.y); }
+    else v = U[(size_t)m * r_n + k];
+    As[idx] = v;
+  }
+  griddep_chain();            // the factor alone was read so far
+  const int KC = K * C, MC = M * C;
+  for (int o = blockIdx.x; o < O; o += gridDim.x) {
+    const cf* xin = in + (size_t)o * KC;
+    for (int idx = tid; idx < KC; idx += MS_THREADS) Xs[idx] = xin[idx];
+    __syncthreads();
+    cf* xout = out + (size_t)o * MC;
+    for (int idx = tid; idx < MC; idx += MS_THREADS) {
+      const int m = idx / C, c = idx - m * C;
+      const cf* a = As + (size_t)m * K;
+      cf acc = make_float2(0.f, 0.f);
+#pragma unroll 4
+      for (int k = 0; k < K; ++k) cfma(acc, a[k], Xs[k * C + c]);
+      xout[idx] = acc;
+    }
+    __syncthreads();
+  }
+}
+
 // AdamUpdate of Algorithm 1 on the Tucker core (entries [0, n)) and, when the streaming kernel only
 // gathered them, on the ks sparse values (entries [n, n + ks)): moments in place, N_L / N_S out.
 __global__ void adam_kernel(const cf* __restrict__ core, cf* __restrict__ m_l, float* __restrict__ v_l,

@@ -95,6 +95,9 @@ WORKLOADS: Dict[str, Workload] = {
                  outlier_frac=(1, 100), outlier_scale=20.0, noise="laplace", noise_scale=0.05),
         Workload("odd32", 96, (5, 7, 32, 17), (3, 3, 8, 5), (1, 25), 3, 5,
                  outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.05),
+        # a 5-way tensor whose middle mode product has many small slices (the shared-memory fp32 product kernel)
+        Workload("small5b", 97, (8, 9, 6, 16, 9), (3, 3, 3, 4, 3), (1, 50), 3, 5,
+                 outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.05),
         # the five benchmark configurations
         Workload("cfg1", 1, (32, 32, 16, 9), (8, 8, 4, 3), (1, 100), 5, 20,
                  outliers_equal_k=True, outlier_scale=20.0, noise_scale=0.01, lr=1e-3),

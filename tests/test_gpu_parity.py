@@ -12,7 +12,7 @@ from tests.parity import Pair, to_device, from_device
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name", ["tiny4", "small4", "small5", "ragged4", "small3", "odd4", "odd32"])
+@pytest.mark.parametrize("name", ["tiny4", "small4", "small5", "ragged4", "small3", "odd4", "odd32", "small5b"])
 def test_trajectory_small(name):
     wl = synth.WORKLOADS[name]
     p = Pair(wl)
