@@ -411,13 +411,16 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, 4) proj_tail_tc_kernel(const vo
 // decayed dense update that follows leaves exactly eta*lambda*N_S), then each warp updates its
 // rows in place and stores them with one bulk copy.
 // ---------------------------------------------------------------------------------------------
-template <int RAT, int NS>
+// NBT > 0: the number of column tiles (tc_ksteps(B)) is built in and the loop over them unrolled; an odd NBT also
+// fixes B = 4 (NBT - 1) + 1, so that every offset into a slab is an immediate.  NBT = 0: both at run time
+template <int RAT, int NS, int NBT>
 __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __restrict__ w, TailTcParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
   const TailParams& p = P.p;
   const TcGeom& G = P.g;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t = lane & 3;
-  const int B = p.B, ra = p.ra, rb = p.rb, twoB = 2 * B, nbuf = G.nbuf, spi = G.spi, tps = G.tps, nbt = G.nbt;
+  const int B = (NBT & 1) ? 4 * (NBT - 1) + 1 : p.B, nbt = NBT ? NBT : G.nbt;
+  const int ra = p.ra, rb = p.rb, twoB = 2 * B, nbuf = G.nbuf, spi = G.spi, tps = G.tps;
   const uint32_t E = p.E, nslab = p.nslab, ngroups = G.ngroups, gstride = gridDim.x;
   const int q = warp / tps, am = 16 * (warp - q * tps);
   const int r0 = am + gq, r1 = r0 + 8;
@@ -588,7 +591,8 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
       // ---- stage 2, one column tile at a time, applied to the slab right away ----
       float* w0row = ws + (size_t)r0 * twoB;
       float* w1row = ws + (size_t)r1 * twoB;
-#pragma unroll 3
+      constexpr int NB_UNROLL = NBT ? NBT : 3;
+#pragma unroll NB_UNROLL
       for (int nb = 0; nb < nbt; ++nb) {
         const float4 fr = ubf[(nb * 2 + 0) * 32 + lane], fi = ubf[(nb * 2 + 1) * 32 + lane];
         float dh[4], dl[4], dx[4];

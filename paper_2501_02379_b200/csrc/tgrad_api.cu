@@ -238,19 +238,30 @@ tgrad_status tc_proj_op(int op, const TailPlan& tp, const void* g, const TailTcP
   if (tp.ntw == 2 && tp.gproj.tps == 1) return tc_proj_op2<RAT, KS, 2, 1>(op, tp, g, P, st);
   return TGRAD_ERR_UNSUPPORTED;
 }
-template <int RAT, int NS>
+template <int RAT, int NS, int NBT>
 tgrad_status tc_back_op2(int op, const TailPlan& tp, void* w, const TailTcParams& P, cudaStream_t st) {
   if (op == 0) {
-    return cudaFuncSetAttribute(back_tail_tc_kernel<RAT, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(back_tail_tc_kernel<RAT, NS, NBT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)tp.gback.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
   }
-  launch_chained(back_tail_tc_kernel<RAT, NS>, dim3(tp.grid_back), dim3(TC_THREADS), tp.gback.total, st, w, P);
+  launch_chained(back_tail_tc_kernel<RAT, NS, NBT>, dim3(tp.grid_back), dim3(TC_THREADS), tp.gback.total, st, w, P);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
+template <int RAT, int NS>
+tgrad_status tc_back_op1(int op, const TailPlan& tp, void* w, const TailTcParams& P, cudaStream_t st) {
+  // the common tile counts (trailing extents 16, 17, 32, 33 and those that pad to them) are built in
+  switch (tp.gback.nbt) {
+    case 4: return tc_back_op2<RAT, NS, 4>(op, tp, w, P, st);
+    case 5: return tc_back_op2<RAT, NS, 5>(op, tp, w, P, st);
+    case 8: return tc_back_op2<RAT, NS, 8>(op, tp, w, P, st);
+    case 9: return tc_back_op2<RAT, NS, 9>(op, tp, w, P, st);
+    default: return tc_back_op2<RAT, NS, 0>(op, tp, w, P, st);
+  }
+}
 template <int RAT>
 tgrad_status tc_back_op(int op, const TailPlan& tp, void* w, const TailTcParams& P, cudaStream_t st) {
-  return tp.back_ns == 2 ? tc_back_op2<RAT, 2>(op, tp, w, P, st) : tc_back_op2<RAT, 1>(op, tp, w, P, st);
+  return tp.back_ns == 2 ? tc_back_op1<RAT, 2>(op, tp, w, P, st) : tc_back_op1<RAT, 1>(op, tp, w, P, st);
 }
 template <int RAT, int RBT>
 tgrad_status th_proj_op(int op, const TailPlan& tp, const void* g, const TailHParams& P, cudaStream_t st) {
