@@ -32,7 +32,7 @@ FALLBACK_HBM_GBS = 6650.0
 # capture summarised in profiles/cfg3_step_and_refresh_tensor_core_path.md (bytes); None where no
 # capture exists for the workload.  (back_tail: 304.1 MB read + 218.0 MB written -- the rest of the
 # 277 MB it writes is still in L2 when the kernel ends.)
-NCU_TRAFFIC_BYTES = {("cfg3", "proj_tail"): 280.4e6 + 19.3e6, ("cfg3", "back_tail"): 304.1e6 + 217.9e6}
+NCU_TRAFFIC_BYTES = {("cfg3", "proj_tail"): 280.4e6 + 19.1e6, ("cfg3", "back_tail"): 304.1e6 + 218.2e6}
 
 
 def step_bytes(wl: synth.Workload) -> int:
