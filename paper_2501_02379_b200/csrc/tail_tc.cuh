@@ -463,11 +463,14 @@ __global__ void __launch_bounds__(TC_THREADS, 2) back_tail_tc_kernel(void* __res
     fence_mbar_init();
   }
   __syncthreads();
-  griddep_chain();            // so far only Ua and Ub were read: the operand tables are built while the previous kernel drains
+  // Before the dependency wait: the operand tables above (Ua, Ub) and the first loads of W.  W was last written by
+  // this kernel's launch of the previous step (or by the caller before this step), which completed before any
+  // kernel of this step got past its own wait; nothing of this step writes it before this kernel does.
   if (tid == 0) {
     uint32_t u = blockIdx.x;
     for (int i = 0; i < la && u < ngroups; ++i, u += gstride) tc_issue_load(wb, smem, G, bars, u, i, nslab);
   }
+  griddep_chain();
   const bool sparse = p.k > 0;
   int b0 = 0, b1 = 0, n0 = 0, n1 = 0;
   uint32_t pom = 0; cf pn = make_float2(0.f, 0.f);
