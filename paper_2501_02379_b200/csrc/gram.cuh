@@ -30,7 +30,8 @@ __device__ __forceinline__ float gr_tf32(float x) { return __uint_as_float((__fl
 
 constexpr size_t GR_SMEM = 2 * 2 * GR_T * GR_LD * sizeof(cf);      // two stages of (Xa, Xb)
 
-template <class S, bool SPLIT>
+// FULL: I_n is a multiple of the tile, so no sub-tile of a warp is empty and the MMA loop has no branches
+template <class S, bool SPLIT, bool FULL>
 __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void* __restrict__ g, int In, uint32_t O, uint32_t C,
                                                                   uint32_t chunks_total, uint32_t chunks_per_split,
                                                                   cf* __restrict__ partial) {
@@ -56,9 +57,9 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
   // which 16-row / 8-column sub-tiles of this warp hold any row of A
   bool mok[2], nok[4];
 #pragma unroll
-  for (int mt = 0; mt < 2; ++mt) mok[mt] = a0 + wm * 32 + mt * 16 < In;
+  for (int mt = 0; mt < 2; ++mt) mok[mt] = FULL || a0 + wm * 32 + mt * 16 < In;
 #pragma unroll
-  for (int nt = 0; nt < 4; ++nt) nok[nt] = b0 + wn * 32 + nt * 8 < In;
+  for (int nt = 0; nt < 4; ++nt) nok[nt] = FULL || b0 + wn * 32 + nt * 8 < In;
   float are[2][4][4], aim[2][4][4];
 #pragma unroll
   for (int mt = 0; mt < 2; ++mt)
@@ -149,13 +150,13 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
       }
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt) {
-        if (!nok[nt]) continue;
+        if (!FULL && !nok[nt]) continue;
         const cf y = widen(XB[wn * 32 + nt * 8 + gq][kc]);
         const float yh0 = HALF ? y.x : gr_tf32(y.x), yh1 = HALF ? y.y : gr_tf32(y.y);
         const float yl0 = y.x - yh0, yl1 = y.y - yh1;
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
-          if (!mok[mt]) continue;
+          if (!FULL && !mok[mt]) continue;
           mma_tf32(are[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], yh0, yh1);
           mma_tf32(aim[mt][nt], ah[mt][0], ah[mt][1], ah[mt][2], ah[mt][3], -yh1, yh0);
           if (DOSPLIT) {

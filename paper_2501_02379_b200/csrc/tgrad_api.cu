@@ -453,12 +453,13 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
     cf* A = reinterpret_cast<cf*>(s->dw + L.w_gram[m]);
     dim3 grid(T * T, L.gram_splits[m]);
     // long contractions average the TF32 input rounding away; short ones get the split-precision products
-    if (O * C >= 16384)
-      gram_partial_kernel<S, false><<<grid, GR_THREADS, GR_SMEM, st>>>(d_grad, In, (uint32_t)O, (uint32_t)C, L.gram_chunks[m],
-                                                                 L.gram_cps[m], partial);
-    else
-      gram_partial_kernel<S, true><<<grid, GR_THREADS, GR_SMEM, st>>>(d_grad, In, (uint32_t)O, (uint32_t)C, L.gram_chunks[m],
-                                                                L.gram_cps[m], partial);
+    const bool full = (In % GR_T) == 0;
+#define TG_GRAM(SPLIT_, FULL_)                                                                                      \
+  gram_partial_kernel<S, SPLIT_, FULL_><<<grid, GR_THREADS, GR_SMEM, st>>>(d_grad, In, (uint32_t)O, (uint32_t)C,    \
+                                                                          L.gram_chunks[m], L.gram_cps[m], partial)
+    if (O * C >= 16384) { if (full) TG_GRAM(false, true); else TG_GRAM(false, false); }
+    else { if (full) TG_GRAM(true, true); else TG_GRAM(true, false); }
+#undef TG_GRAM
     TG_LAUNCH_CHECK();
     gram_reduce_kernel<<<(In * In + GRR_E - 1) / GRR_E, GRR_E * GRR_G, 0, st>>>(partial, L.gram_splits[m], In, A); TG_LAUNCH_CHECK();
     if (L.jac_fast[m]) {
@@ -737,11 +738,16 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
   s = plan_tail(st);
   if (s != TGRAD_OK) { delete st; return s; }
   {
-    cudaError_t e1 = cudaFuncSetAttribute(gram_partial_kernel<StoreC64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GR_SMEM);
-    cudaError_t e2 = cudaFuncSetAttribute(gram_partial_kernel<StoreC64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GR_SMEM);
-    cudaError_t e3 = cudaFuncSetAttribute(gram_partial_kernel<StoreC32H, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GR_SMEM);
-    cudaError_t e4 = cudaFuncSetAttribute(gram_partial_kernel<StoreC32H, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GR_SMEM);
-    if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || e4 != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
+    bool ok = true;
+#define TG_GRAM_ATTR(S_, SPLIT_, FULL_)                                                                       \
+  ok = ok && cudaFuncSetAttribute(gram_partial_kernel<S_, SPLIT_, FULL_>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                  (int)GR_SMEM) == cudaSuccess
+    TG_GRAM_ATTR(StoreC64, false, false); TG_GRAM_ATTR(StoreC64, false, true);
+    TG_GRAM_ATTR(StoreC64, true, false); TG_GRAM_ATTR(StoreC64, true, true);
+    TG_GRAM_ATTR(StoreC32H, false, false); TG_GRAM_ATTR(StoreC32H, false, true);
+    TG_GRAM_ATTR(StoreC32H, true, false); TG_GRAM_ATTR(StoreC32H, true, true);
+#undef TG_GRAM_ATTR
+    if (!ok) { delete st; return TGRAD_ERR_CUDA; }
   }
   if (cfg->dims[0] <= SW_MAX_I && cfg->ranks[0] <= SW_MAX_R &&
       cudaFuncSetAttribute(core_sandwich_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
