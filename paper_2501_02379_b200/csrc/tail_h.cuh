@@ -318,14 +318,16 @@ struct TailHBParams {
   int* flags;
 };
 
-template <int RAT, int RBT>
+// NBT > 0 (odd): the number of column tiles is built in, which fixes B = 4 (NBT - 1) + 1; a warp's share of the tile
+// loop is unrolled and every offset into a row is an immediate.  NBT = 0: both at run time.
+template <int RAT, int RBT, int NBT>
 __global__ void __launch_bounds__(512, 1) back_tail_h_kernel(void* __restrict__ w, TailHBParams P) {
   griddep_chain();
   extern __shared__ __align__(128) unsigned char smem[];
   const TailParams& p = P.p;
   const TailHBGeom& G = P.g;
   const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t = lane & 3;
-  const int A = p.A, B = p.B, ra = p.ra, rb = p.rb, nbuf = G.nbuf, nbt = G.nbt;
+  const int A = p.A, B = NBT ? 4 * (NBT - 1) + 1 : p.B, ra = p.ra, rb = p.rb, nbuf = G.nbuf, nbt = NBT ? NBT : G.nbt;
   constexpr int KS2 = 2 * RAT;
   const uint32_t E = p.E, nslab = p.nslab, gstride = gridDim.x;
   const int mtile = warp >> 1, am = 16 * mtile, r0 = am + gq, r1 = r0 + 8;
@@ -443,14 +445,22 @@ __global__ void __launch_bounds__(512, 1) back_tail_h_kernel(void* __restrict__ 
 #pragma unroll
           for (int i = 0; i < 4; ++i) split_tf32(d1[c][jt][i], yh[c][jt][i], yl[c][jt][i]);
       // ---- stage 2, one column tile at a time, applied to the slab right away ----
+      constexpr int NB_UNROLL = NBT ? (NBT + 1) / 2 : 1;
+#pragma unroll NB_UNROLL
       for (int nb = nb0; nb < nb1; ++nb) {
-        float dh[4] = {0.f, 0.f, 0.f, 0.f}, dl[4] = {0.f, 0.f, 0.f, 0.f}, dx[4] = {0.f, 0.f, 0.f, 0.f};
+        float dh[4], dl[4], dx[4];
 #pragma unroll
         for (int jt = 0; jt < RBT; ++jt) {
           const float4 fr = ubf[((nb * RBT + jt) * 2 + 0) * 32 + lane], fi = ubf[((nb * RBT + jt) * 2 + 1) * 32 + lane];
-          mma_tf32(dh, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.x, fr.y);
-          mma_tf32(dl, yl[0][jt][0], yl[0][jt][2], yl[0][jt][1], yl[0][jt][3], fr.x, fr.y);
-          mma_tf32(dx, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.z, fr.w);
+          if (jt == 0) {
+            mma_tf32_z(dh, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.x, fr.y);
+            mma_tf32_z(dl, yl[0][jt][0], yl[0][jt][2], yl[0][jt][1], yl[0][jt][3], fr.x, fr.y);
+            mma_tf32_z(dx, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.z, fr.w);
+          } else {
+            mma_tf32(dh, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.x, fr.y);
+            mma_tf32(dl, yl[0][jt][0], yl[0][jt][2], yl[0][jt][1], yl[0][jt][3], fr.x, fr.y);
+            mma_tf32(dx, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.z, fr.w);
+          }
           mma_tf32(dh, yh[1][jt][0], yh[1][jt][2], yh[1][jt][1], yh[1][jt][3], fi.x, fi.y);
           mma_tf32(dl, yl[1][jt][0], yl[1][jt][2], yl[1][jt][1], yl[1][jt][3], fi.x, fi.y);
           mma_tf32(dx, yh[1][jt][0], yh[1][jt][2], yh[1][jt][1], yh[1][jt][3], fi.z, fi.w);

@@ -280,15 +280,21 @@ tgrad_status th_dispatch(int op, const TailPlan& tp, const void* g, const TailHP
   return TGRAD_ERR_UNSUPPORTED;
 }
 
-template <int RAT, int RBT>
-tgrad_status th_back_op(int op, const TailPlan& tp, void* w, const TailHBParams& P, cudaStream_t st) {
+template <int RAT, int RBT, int NBT>
+tgrad_status th_back_op2(int op, const TailPlan& tp, void* w, const TailHBParams& P, cudaStream_t st) {
   if (op == 0) {
-    return cudaFuncSetAttribute(back_tail_h_kernel<RAT, RBT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(back_tail_h_kernel<RAT, RBT, NBT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)tp.ghb.total) == cudaSuccess ? TGRAD_OK : TGRAD_ERR_CUDA;
   }
-  launch_chained(back_tail_h_kernel<RAT, RBT>, dim3(tp.grid_hb), dim3(32 * tp.ghb.nwarps), tp.ghb.total, st, w, P);
+  launch_chained(back_tail_h_kernel<RAT, RBT, NBT>, dim3(tp.grid_hb), dim3(32 * tp.ghb.nwarps), tp.ghb.total, st, w, P);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
+}
+template <int RAT, int RBT>
+tgrad_status th_back_op(int op, const TailPlan& tp, void* w, const TailHBParams& P, cudaStream_t st) {
+  // rows of 65 entries (17 column tiles) have their own instance with the tile loop unrolled
+  if (tp.ghb.nbt == 17) return th_back_op2<RAT, RBT, 17>(op, tp, w, P, st);
+  return th_back_op2<RAT, RBT, 0>(op, tp, w, P, st);
 }
 tgrad_status thb_dispatch(int op, const TailPlan& tp, void* w, const TailHBParams& P, cudaStream_t st) {
 #define TG_HCASE(RAT_, RBT_) if (tp.h_rat == RAT_ && tp.h_rbt == RBT_) return th_back_op<RAT_, RBT_>(op, tp, w, P, st);
