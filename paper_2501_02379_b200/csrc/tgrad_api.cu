@@ -470,7 +470,7 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
     gram_reduce_kernel<<<(In * In + GRR_E - 1) / GRR_E, GRR_E * GRR_G, 0, st>>>(partial, L.gram_splits[m], In, A); TG_LAUNCH_CHECK();
     if (L.jac_fast[m]) {
       JacobiFastMode& fm = fp.mode[fp.nmodes++];
-      fm.A = A;
+      fm.A = A; fm.A0 = A;
       fm.work = reinterpret_cast<cf*>(s->dw + L.w_jac[m]);
       fm.log = reinterpret_cast<float4*>(s->dw + L.w_log[m]);
       fm.lam = reinterpret_cast<float*>(s->dw + L.w_lam[m]);
@@ -483,7 +483,9 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
           cf* t1 = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
           cf* t2 = reinterpret_cast<cf*>(s->dw + L.w_rot[m]);
           TG_TRY(small_product(true, V, t1, V, In, In, In, st));          // G = V^H V
-          ns_residual_kernel<<<(In * In + 255) / 256, 256, 0, st>>>(t1, In); TG_LAUNCH_CHECK();
+          int* bad = flags + JAC_BAD_BASIS + m;
+          if (cudaMemsetAsync(bad, 0, sizeof(int), st) != cudaSuccess) return TGRAD_ERR_CUDA;
+          ns_residual_kernel<<<(In * In + 255) / 256, 256, 0, st>>>(t1, In, bad); TG_LAUNCH_CHECK();
           TG_TRY(small_product(false, t1, t2, V, In, In, In, st));        // V E
           if (cudaMemcpyAsync(V, t2, (size_t)In * In * 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return TGRAD_ERR_CUDA;
           TG_TRY(small_product(false, V, t1, A, In, In, In, st));         // A V

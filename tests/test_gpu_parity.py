@@ -227,6 +227,29 @@ def test_nonfinite_sets_flag():
     assert flags & B.FLAG_NONFINITE
 
 
+def test_warm_refresh_recovers_from_a_nonfinite_gradient():
+    # a refresh on a gradient with a NaN leaves a useless eigenvector basis behind; the next warm-started refresh must
+    # notice and start from the identity, so that its factors are those of the new (finite) gradient
+    wl = synth.WORKLOADS["ragged4"]
+    src = synth.GradientSource(wl)
+    st = B.TgradState(B.make_config(wl.shape, wl.ranks, wl.k, wl.T, auto_refresh=False, warm_refresh=True))
+    st.refresh_subspace(to_device(src.gradient(0), False))
+    g = src.gradient(1).copy()
+    g.reshape(-1)[7] = np.nan
+    st.refresh_subspace(to_device(g, False))
+    assert st.query_status()[0] & B.FLAG_NONFINITE
+    g2 = src.gradient(2)
+    st.refresh_subspace(to_device(g2, False))
+    ost = orc.OracleState(orc.OracleConfig(shape=wl.shape, ranks=wl.ranks, k=wl.k, T=wl.T, half_storage=False, lr=1e-3,
+                                           alpha=1.0, lam=1.0, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0))
+    orc.oracle_refresh(ost, g2)
+    assert np.array_equal(st.export(B.WHAT_OMEGA), ost.omega)
+    for ug, uo in zip(st.factors(), ost.factors):
+        assert np.all(np.isfinite(ug))
+        assert H.max_sin_angle(ug, uo) <= 1e-3
+        assert H.ortho_defect(ug) <= 1e-5
+
+
 def test_jacobi_cap_sets_flag_not_hang():
     wl = synth.WORKLOADS["small4"]
     g = synth.GradientSource(wl).gradient(0)
