@@ -28,10 +28,12 @@ from paper_2501_02379_b200 import replicas, synth  # noqa: E402
 METRIC = "tgrad_step effective HBM GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the two streaming kernels, from the ncu
-# capture summarised in profiles/cfg3_step_and_refresh_tensor_core_path.md (bytes); None where no
-# capture exists for the workload.  (back_tail: 304.1 MB read + 218.0 MB written -- the rest of the
-# 277 MB it writes is still in L2 when the kernel ends.)
+NOMINAL_HBM_GBS = 8000.0      # the nominal HBM3e figure fractions are also quoted against
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the two streaming kernels as one ncu capture
+# of this build's kernels counted them (bytes); None where no capture of the current kernel exists.
+# (back_tail: 304.1 MB read + 218.2 MB written -- the rest of the 277 MB it writes is still in L2 when the
+# kernel ends.)
 NCU_TRAFFIC_BYTES = {("cfg3", "proj_tail"): 280.4e6 + 19.1e6, ("cfg3", "back_tail"): 304.1e6 + 218.2e6}
 
 
@@ -126,9 +128,10 @@ def oracle_sample(wl: synth.Workload, budget_s: float, n_steps: int):
     slices of mode 1 (ranks clipped to the sample's extents), sized for the time budget."""
     import dataclasses
     from oracle import tgrad_oracle as orc
-    # oracle speed is roughly 5e6 entries/s per step on a few cores; size the sample for the budget
-    per_step = budget_s / max(1, n_steps + 1)
-    entries = max(200_000, int(4.0e6 * per_step))
+    # a non-refresh oracle step handles roughly 1.5e7 entries per second on 8 cores and its refresh costs about
+    # a dozen steps; size the sample for the budget (the whole tensor where that fits)
+    per_step = budget_s / max(1, n_steps + 12)
+    entries = max(200_000, int(1.2e7 * per_step))
     rest = wl.numel // wl.shape[0]
     i1 = int(min(wl.shape[0], max(4, entries // rest)))
     shape = (i1,) + tuple(wl.shape[1:])
@@ -162,6 +165,15 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
+def config_of(wl: synth.Workload, world: int, ring: int):
+    eb = 4 if wl.half_storage else 8
+    return {"workload": wl.name, "tensors_per_gpu": wl.n_tensors, "shape": list(wl.shape), "ranks": list(wl.ranks),
+            "k": wl.k, "T": wl.T, "storage": "2xfp16" if wl.half_storage else "complex64", "warm_refresh": True,
+            "parallelism": "replicas only" if world > 1 else "single GPU",
+            "l2": f"inputs larger than L2: ring of {ring} gradient buffers of {wl.numel * eb / 1e6:.0f} MB each "
+                  f"plus the weight"}
+
+
 def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -179,7 +191,8 @@ def run_reference(args, wl):
         "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus, "steps": len(timed),
         "warmup": args.warmup, "ms_per_step": 1e3 * total / len(timed), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "shape": list(wl.shape), "sample_shape": list(sub.shape)},
+        "config": config_of(wl, 1, args.ring),
+        "sample_shape": list(sub.shape),
         "steps_per_s": len(timed) / total,
         "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -221,6 +234,8 @@ def run_ours(args, wl):
     cfgs = [B.make_config(wl.shape, wl.ranks, wl.k, wl.T, lr=wl.lr, half_storage=half, auto_refresh=True,
                           warm_refresh=True)
             for _ in srcs]
+    if wl.T < 2:
+        raise SystemExit("the benchmark separates refresh steps from the others: T >= 2")
     states = [B.TgradState(c) for c in cfgs]
     stream = torch.cuda.current_stream()
 
@@ -259,36 +274,52 @@ def run_ours(args, wl):
     ms = replicas.max_over_ranks(ms, dist, "cuda")
     flags = [s.query_status()[0] for s in states]
 
-    # ---- non-refresh steps alone, then their per-stage device times (events on the launching stream) ----
+    # ---- non-refresh steps alone, for at least a second of device time so that the clock sampler sees the
+    #      GPU under this load (runs of T-1 steps; the counter is set back to 1 before each run, which keeps
+    #      them off the refresh schedule and changes nothing but the bias-correction scalars) ----
     st0 = states[0]
-    while t % wl.T == 0:
-        one_step(t); t += 1
-    n_stage_steps = min(30, max(1, (wl.T - (t % wl.T) - 1) // 2))
-    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e2.record(stream)
-    for _ in range(n_stage_steps):
-        states[0].step(weights[0], grads[0][t % ring], stream); t += 1
-    e3.record(stream)
-    torch.cuda.synchronize()
-    nonrefresh_ms = e2.elapsed_time(e3) / n_stage_steps
+    sampler.active = True
+    run_len = min(wl.T - 1, 200)
+    nonrefresh_total_ms, nonrefresh_steps = 0.0, 0
+    while nonrefresh_total_ms < args.min_clock_ms and nonrefresh_steps < 20000:
+        st0.set_step(1)
+        e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e2.record(stream)
+        for _ in range(run_len):
+            st0.step(weights[0], grads[0][t % ring], stream); t += 1
+        e3.record(stream)
+        torch.cuda.synchronize()
+        nonrefresh_total_ms += e2.elapsed_time(e3); nonrefresh_steps += run_len
+    sampler.active = False
+    nonrefresh_ms = nonrefresh_total_ms / nonrefresh_steps
+    # ---- per-stage device times (events on the launching stream between the stages) ----
+    n_stage_steps = min(30, run_len)
+    st0.set_step(1)
     st0.set_stage_timing(True)                       # the events between the stages add a few microseconds per stage
     for _ in range(n_stage_steps):
-        states[0].step(weights[0], grads[0][t % ring], stream); t += 1
+        st0.step(weights[0], grads[0][t % ring], stream); t += 1
     torch.cuda.synchronize()
     stage_ms, n_rec = st0.stage_times(stream)
     st0.set_stage_timing(False)
     # the counter of tensor 0 ran ahead of the others; irrelevant from here on
     stage_us = {name: 1e3 * v / max(1, n_rec) for name, v in zip(B.STAGE_NAMES, stage_ms)}
 
-    # ---- one refresh step timed alone ----
-    e4, e5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    e4.record(stream)
-    last_refresh = ((t - 1) // wl.T) * wl.T                        # a gradient other than the last refresh's, so that a
-    states[0].refresh_subspace(grads[0][(last_refresh + 1) % ring], stream)   # warm start meets a changed matrix
-    e5.record(stream)
-    torch.cuda.synchronize()
-    refresh_ms = e4.elapsed_time(e5)
+    # ---- steps that carry a refresh (t mod T = 0), timed alone: each on another gradient than the refresh
+    #      before it, so that the warm start of the eigensolver meets a changed matrix ----
+    refresh_step_list = []
+    for i in range(3):
+        st0.set_step(wl.T)
+        e4, e5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e4.record(stream)
+        st0.step(weights[0], grads[0][(i + 1) % ring], stream)
+        e5.record(stream)
+        torch.cuda.synchronize()
+        refresh_step_list.append(e4.elapsed_time(e5))
+    refresh_step_ms = float(np.median(refresh_step_list))
+    refresh_ms = refresh_step_ms - nonrefresh_ms
+    amortised_ms = ((wl.T - 1) * nonrefresh_ms + refresh_step_ms) / wl.T
+    flags += [st0.query_status()[0]]
 
     # ---- end to end with host buffers: W and G go up, W comes back, every step ----
     n_e2e = max(1, min(args.steps, args.e2e_steps))
@@ -354,6 +385,8 @@ def run_ours(args, wl):
         if dist is not None:
             dist.destroy_process_group()
         return
+    if any(flags):
+        raise SystemExit(f"sticky device flags set during the benchmark: {flags}")
     bstep = step_bytes(wl) * n_t
     value = bstep * args.steps * world / (ms * 1e-3) / 1e9
     e2e_val = bstep * n_e2e * world / (e2e_ms * 1e-3) / 1e9
@@ -366,17 +399,22 @@ def run_ours(args, wl):
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{wl.name}: {n_t} x complex {'x'.join(map(str, wl.shape))} "
-                               f"({'2xfp16' if half else 'complex64'} W/G), ranks {list(wl.ranks)}, k={wl.k}, T={wl.T}",
-                   "tensors_per_gpu": n_t, "warm_refresh": True, "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "l2": f"inputs larger than L2: ring of {ring} gradient buffers of "
-                         f"{wl.numel * eb / 1e6:.0f} MB each plus the weight"},
+        "config": config_of(wl, world, ring),
         "steps_per_s": args.steps * world / (ms * 1e-3),
         "refreshes_in_timed_region": n_refresh,
         "step_bytes": bstep,
-        "nonrefresh_step_us": 1e3 * nonrefresh_ms, "refresh_us": 1e3 * refresh_ms,
+        # one tensor, from the separately timed regions above: a non-refresh step (mean over >= 1 s), a step that
+        # carries a refresh (median of 3), and the schedule's mean ((T-1) t_step + t_refresh_step) / T
+        "nonrefresh_step_us": 1e3 * nonrefresh_ms, "nonrefresh_steps_timed": nonrefresh_steps,
+        "refresh_step_us": 1e3 * refresh_step_ms, "refresh_us": 1e3 * refresh_ms,
         "nonrefresh_gbs": step_bytes(wl) / (nonrefresh_ms * 1e-3) / 1e9,
         "frac_of_peak_nonrefresh": step_bytes(wl) / (nonrefresh_ms * 1e-3) / 1e9 / peak,
+        "frac_of_nominal_8tbs_nonrefresh": step_bytes(wl) / (nonrefresh_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+        "amortised_ms_per_step": amortised_ms,
+        "amortised_gbs": step_bytes(wl) / (amortised_ms * 1e-3) / 1e9,
+        "frac_of_peak_amortised": step_bytes(wl) / (amortised_ms * 1e-3) / 1e9 / peak,
+        "frac_of_nominal_8tbs_amortised": step_bytes(wl) / (amortised_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+        "peak_gbs": peak, "peak_kind": peak_kind, "nominal_gbs": NOMINAL_HBM_GBS,
         "stage_us": stage_us,
         "clocks": sampler.summary(),
         "e2e": {"value": e2e_val, "unit": "GB/s", "h2d_bytes_per_step": 2 * wl.numel * eb * n_t,
@@ -385,11 +423,12 @@ def run_ours(args, wl):
         "gpu_launches": int(launches),
         "sticky_flags": flags,
         "roofline": {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                     "frac_of_nominal_8tbs": ach / NOMINAL_HBM_GBS,
                      "peak_kind": peak_kind, "bytes_per_launch": sb[dom], "us_per_launch": stage_us[dom],
                      "traffic": traffic},
     }
     if world == 1 and not args.no_cpu_baseline:
-        sub, times, t_refresh = oracle_sample(wl, budget_s=20.0, n_steps=2)
+        sub, times, t_refresh = oracle_sample(wl, budget_s=45.0, n_steps=2)
         tm = float(np.median(times))
         out["cpu_baseline"] = {
             "value": step_bytes(sub) / tm / 1e9, "unit": "GB/s", "cores": blas_threads(), "kind": "oracle",
@@ -412,6 +451,8 @@ def main():
     ap.add_argument("--ring", type=int, default=3, help="distinct gradient buffers cycled through")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-clock-ms", type=float, default=1200.0,
+                    help="device time of the separately timed non-refresh region (the clock sampler runs over it)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

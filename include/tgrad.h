@@ -62,6 +62,10 @@ typedef enum {
 /* sticky device flags reported by tgrad_query_status() */
 #define TGRAD_FLAG_NO_CONVERGE 1   /* the Jacobi eigensolver hit jacobi_max_sweeps */
 #define TGRAD_FLAG_NONFINITE   2   /* a NaN/Inf magnitude was seen while selecting Omega */
+#define TGRAD_FLAG_COPY_TIMEOUT 4  /* a streaming kernel gave up waiting for one of its own asynchronous copies
+                                      (every device-side wait is bounded); the blocks that saw it returned early,
+                                      so W and the moments of that step are undefined.  Not expected in normal
+                                      operation; treat the state as lost */
 
 typedef enum {
   TGRAD_C64 = 0,   /* interleaved 2 x fp32 */
@@ -72,10 +76,12 @@ typedef enum {
 
 /* Hyper-parameters of Algorithm 1 (its "Require" line) plus storage options. */
 typedef struct {
-  int32_t ndim;                     /* N, 3 <= ndim <= TGRAD_MAX_NDIM                          */
+  int32_t ndim;                     /* N, 2 <= ndim <= TGRAD_MAX_NDIM (N = 2: the matrix case,  */
+                                    /* where the Tucker factors are the singular subspaces)     */
   int64_t dims[TGRAD_MAX_NDIM];     /* I_1..I_N, row-major; prod(dims) < 2^32                   */
   int32_t ranks[TGRAD_MAX_NDIM];    /* Tucker ranks, 1 <= r_n <= I_n                            */
-  int64_t k;                        /* |Omega| = ceil(rho*I), computed exactly by the caller    */
+  int64_t k;                        /* |Omega| = ceil(rho*I), computed exactly by the caller;   */
+                                    /* k < 2^31                                                 */
   int32_t T;                        /* subspace change frequency, >= 1                          */
   float lr;                         /* eta                                                      */
   float alpha;                      /* scale of the reconstructed low-rank update               */
@@ -115,7 +121,17 @@ enum {
  * Counts follow the state inventory of Algorithm 1 (its initialisation
  * statements) and of the appendix "Parameter Complexity Analysis":
  * prod(r_n) core-shaped entries for each low-rank moment, sum I_n r_n factor
- * entries, k indices and k entries for each sparse moment. */
+ * entries, k indices and k entries for each sparse moment.
+ * The sizes do not depend on the device the state will run on.
+ *
+ * Limits of this implementation; a configuration outside them returns
+ * TGRAD_ERR_UNSUPPORTED here and from tgrad_init_state:
+ *   prod(dims) < 2^32 (flat indices are uint32) and k < 2^31;
+ *   every I_n <= 1024 (size of the on-device eigensolver);
+ *   r_N <= 32 (rank of the last mode);
+ *   one trailing slab of I_{N-1} x I_N entries, with the operand tables of
+ *   its two mode products, must fit in the 227 KB of shared memory of one SM
+ *   (roughly I_{N-1} * (I_N + r_N) complex64 entries <= 28,000). */
 tgrad_status tgrad_state_bytes(const tgrad_config* cfg, size_t* persistent_bytes, size_t* workspace_bytes);
 
 /* Algorithm 1 initialisation: t <- 0, M_L, V_L, M_S, V_S <- 0 (enqueued on
@@ -191,6 +207,8 @@ const char* tgrad_status_string(tgrad_status s);
  * exits.  That fixes the largest input: numel <= TGRAD_NOALLOC_MAX_NUMEL,
  * otherwise TGRAD_ERR_TOO_LARGE and nothing is enqueued.
  *
+ * d_grad, d_omega and d_values must be 16-byte aligned, like the pointers of
+ * the other entry points (TGRAD_ERR_INVALID_ARG otherwise, nothing enqueued).
  * d_grad:   device, numel entries of wg_dtype (tgrad_dtype), read only.
  * d_omega:  device, out, k x uint32: the flat indices of the k entries of
  *           largest |g|^2 (fp32 re*re + im*im without fused multiply-add),

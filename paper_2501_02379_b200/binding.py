@@ -21,7 +21,7 @@ STAGE_NAMES = ["proj_tail", "proj_chain", "mode1_adam", "back_chain", "back_tail
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BUFFER_TOO_SMALL, ERR_CUDA, ERR_NO_CONVERGE, ERR_NONFINITE, ERR_BAD_STATE = range(8)
 ERR_TOO_LARGE = 8
 NOALLOC_MAX_NUMEL = 1 << 26
-FLAG_NO_CONVERGE, FLAG_NONFINITE = 1, 2
+FLAG_NO_CONVERGE, FLAG_NONFINITE, FLAG_COPY_TIMEOUT = 1, 2, 4
 C64, C32H = 0, 1
 WHAT_OMEGA, WHAT_M_L, WHAT_V_L, WHAT_M_S, WHAT_V_S, WHAT_CORE, WHAT_N_L, WHAT_N_S = 1, 2, 3, 4, 5, 6, 7, 8
 WHAT_GRAM_BASE, WHAT_FACTOR_BASE = 32, 64

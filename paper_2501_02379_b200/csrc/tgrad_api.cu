@@ -28,6 +28,7 @@ constexpr int kStages = 5;   // proj_tail, proj_chain, adam_core, back_chain, ba
 constexpr int kTimingRing = 64;
 
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+constexpr size_t kSmemMax = 227 * 1024;   // dynamic shared memory a block may ask for
 
 struct Layout {
   // persistent block
@@ -76,8 +77,8 @@ tgrad_status validate(const tgrad_config* c) {
   if (c->jacobi_max_sweeps < 0 || c->jacobi_tol < 0.f) return TGRAD_ERR_INVALID_ARG;
   if (c->warm_refresh != 0 && c->warm_refresh != 1) return TGRAD_ERR_INVALID_ARG;
   // limits of this implementation
-  if (c->ndim < 3) return TGRAD_ERR_UNSUPPORTED;             // the matrix case is not built
   if (tot >= 4294967296.0L) return TGRAD_ERR_UNSUPPORTED;    // flat indices are uint32
+  if (c->k >= ((int64_t)1 << 31)) return TGRAD_ERR_UNSUPPORTED;   // slots of Omega are addressed with int
   for (int n = 0; n < c->ndim; ++n)
     if (c->dims[n] > JAC_MAX_N) return TGRAD_ERR_UNSUPPORTED;
   if (c->ranks[c->ndim - 1] > 32) return TGRAD_ERR_UNSUPPORTED;
@@ -100,10 +101,31 @@ void plan_gram(const tgrad_config* c, int n, int sm, uint32_t& chunks, uint32_t&
   chunks = (uint32_t)total; cps = (uint32_t)per; splits = (int)((total + per - 1) / per);
 }
 
-tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
-  tgrad_status s = validate(c);
+// The configuration the kernels see.  A matrix (N = 2, where the Tucker decomposition is the matrix SVD) is handled as
+// the 3-way tensor I_1 x 1 x I_2 with ranks (r_1, 1, r_2): the unit mode's factor is the 1 x 1 identity, so every
+// stage computes exactly what Algorithm 1 computes for the matrix.  map[n] = internal mode of the caller's mode n.
+tgrad_status internal_config(const tgrad_config* ext, tgrad_config& in, int* map) {
+  tgrad_status s = validate(ext);
   if (s != TGRAD_OK) return s;
+  in = *ext;
+  for (int n = 0; n < TGRAD_MAX_NDIM; ++n) map[n] = n;
+  if (ext->ndim == 2) {
+    in.ndim = 3;
+    in.dims[0] = ext->dims[0]; in.dims[1] = 1; in.dims[2] = ext->dims[1];
+    in.ranks[0] = ext->ranks[0]; in.ranks[1] = 1; in.ranks[2] = ext->ranks[1];
+    map[0] = 0; map[1] = 2;
+  }
+  return TGRAD_OK;
+}
+
+tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
   const int N = c->ndim;
+  {
+    // a trailing slab and the operand tables of its two products must fit in the shared memory of one SM
+    const int A = (int)c->dims[N - 2], B = (int)c->dims[N - 1], ra = c->ranks[N - 2], rb = c->ranks[N - 1];
+    if (tail_blk_geom(A, B, ra, rb, false).total > kSmemMax || tail_blk_geom(A, B, ra, rb, true).total > kSmemMax)
+      return TGRAD_ERR_UNSUPPORTED;
+  }
   uint64_t numel = 1, P = 1;
   for (int n = 0; n < N; ++n) { numel *= (uint64_t)c->dims[n]; P *= (uint64_t)c->ranks[n]; }
   L.numel = numel; L.P = P;
@@ -163,7 +185,9 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
 }  // namespace
 
 struct tgrad_state {
-  tgrad_config cfg;
+  tgrad_config cfg;     // as the kernels see it (a matrix carries a unit mode in the middle)
+  int ext_ndim;         // the caller's N
+  int mode_map[TGRAD_MAX_NDIM];   // caller's mode -> mode of cfg
   Layout L;
   char* dp;
   char* dw;
@@ -715,7 +739,13 @@ extern "C" {
 tgrad_status tgrad_state_bytes(const tgrad_config* cfg, size_t* persistent_bytes, size_t* workspace_bytes) {
   if (!persistent_bytes || !workspace_bytes) return TGRAD_ERR_INVALID_ARG;
   Layout L;
-  tgrad_status s = compute_layout(cfg, L, 148);
+  tgrad_config ic; int map[TGRAD_MAX_NDIM];
+  tgrad_status s = internal_config(cfg, ic, map);
+  if (s != TGRAD_OK) return s;
+  // The split-K plan of the Gram kernels (part of the workspace size) is made for 148 SMs whatever the device:
+  // the sizes a configuration needs are then the same on every machine, and the kernels only need a plan, not
+  // the best one.
+  s = compute_layout(&ic, L, 148);
   if (s != TGRAD_OK) return s;
   *persistent_bytes = L.p_total;
   *workspace_bytes = L.w_total;
@@ -727,8 +757,12 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
   if (!out) return TGRAD_ERR_INVALID_ARG;
   *out = nullptr;
   Layout L;
-  tgrad_status s = compute_layout(cfg, L, 148);
+  tgrad_config ic; int map[TGRAD_MAX_NDIM];
+  tgrad_status s = internal_config(cfg, ic, map);
   if (s != TGRAD_OK) return s;
+  s = compute_layout(&ic, L, 148);
+  if (s != TGRAD_OK) return s;
+  cfg = &ic;
   if (!d_persistent || !d_workspace) return TGRAD_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(d_persistent) & 255) || (reinterpret_cast<uintptr_t>(d_workspace) & 255))
     return TGRAD_ERR_INVALID_ARG;
@@ -737,6 +771,8 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
   if (!st) return TGRAD_ERR_INVALID_ARG;
   memset(st, 0, sizeof(*st));
   st->cfg = *cfg; st->L = L;
+  st->ext_ndim = (ic.ndim == 3 && map[1] == 2) ? 2 : ic.ndim;
+  for (int n = 0; n < TGRAD_MAX_NDIM; ++n) st->mode_map[n] = map[n];
   st->dp = static_cast<char*>(d_persistent); st->dw = static_cast<char*>(d_workspace);
   st->t = 0; st->have_subspace = false; st->tabs_stale = true; st->basis_valid = false;
   int dev = 0, sm = 0;
@@ -813,7 +849,7 @@ tgrad_status tgrad_query_status(tgrad_state* st, void* cuda_stream, int32_t* sti
   if (cudaStreamSynchronize(stream) != cudaSuccess) return TGRAD_ERR_CUDA;
   if (sticky_flags) *sticky_flags = host[0];
   if (t) *t = st->t;
-  if (sweeps) for (int n = 0; n < st->cfg.ndim; ++n) sweeps[n] = host[1 + n];
+  if (sweeps) for (int n = 0; n < st->ext_ndim; ++n) sweeps[n] = host[1 + st->mode_map[n]];
   return TGRAD_OK;
 }
 
@@ -828,8 +864,8 @@ static tgrad_status locate(tgrad_state* st, int32_t what, bool for_import, char*
     case TGRAD_WHAT_V_S: *ptr = st->dp + L.p_vs; *bytes = k * 4; return TGRAD_OK;
     default: break;
   }
-  if (what >= TGRAD_WHAT_FACTOR_BASE && what < TGRAD_WHAT_FACTOR_BASE + c.ndim) {
-    int n = what - TGRAD_WHAT_FACTOR_BASE;
+  if (what >= TGRAD_WHAT_FACTOR_BASE && what < TGRAD_WHAT_FACTOR_BASE + st->ext_ndim) {
+    int n = st->mode_map[what - TGRAD_WHAT_FACTOR_BASE];
     *ptr = st->dp + L.p_factor[n]; *bytes = (size_t)c.dims[n] * c.ranks[n] * 8; return TGRAD_OK;
   }
   if (for_import) return TGRAD_ERR_INVALID_ARG;
@@ -839,8 +875,8 @@ static tgrad_status locate(tgrad_state* st, int32_t what, bool for_import, char*
     case TGRAD_WHAT_N_S: *ptr = st->dw + L.w_ns; *bytes = k * 8; return TGRAD_OK;
     default: break;
   }
-  if (what >= TGRAD_WHAT_GRAM_BASE && what < TGRAD_WHAT_GRAM_BASE + c.ndim) {
-    int n = what - TGRAD_WHAT_GRAM_BASE;
+  if (what >= TGRAD_WHAT_GRAM_BASE && what < TGRAD_WHAT_GRAM_BASE + st->ext_ndim) {
+    int n = st->mode_map[what - TGRAD_WHAT_GRAM_BASE];
     *ptr = st->dw + L.w_gram[n]; *bytes = (size_t)c.dims[n] * c.dims[n] * 8; return TGRAD_OK;
   }
   return TGRAD_ERR_INVALID_ARG;
@@ -1019,6 +1055,8 @@ extern "C" tgrad_status tgrad_select_topk_noalloc(const void* d_grad, int64_t nu
   if (wg_dtype != TGRAD_C64 && wg_dtype != TGRAD_C32H) return TGRAD_ERR_INVALID_ARG;
   if ((uint64_t)numel > kNaMaxNumel) return TGRAD_ERR_TOO_LARGE;
   if (!d_grad || (k > 0 && (!d_omega || !d_values))) return TGRAD_ERR_INVALID_ARG;
+  // the kernels read the gradient with vector loads and write index / value pairs: same rule as the other calls
+  if (!aligned16(d_grad) || (k > 0 && (!aligned16(d_omega) || !aligned16(d_values)))) return TGRAD_ERR_INVALID_ARG;
   if (k == 0) return TGRAD_OK;
   NoAllocScratch* sc = nullptr;
   int sm = 0;

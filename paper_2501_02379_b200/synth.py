@@ -98,6 +98,21 @@ WORKLOADS: Dict[str, Workload] = {
         # a 5-way tensor whose middle mode product has many small slices (the shared-memory fp32 product kernel)
         Workload("small5b", 97, (8, 9, 6, 16, 9), (3, 3, 3, 4, 3), (1, 50), 3, 5,
                  outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.05),
+        # shapes that reach the kernels only the largest configuration would otherwise run: 65-entry rows of a
+        # 128-row slab stored as fp16 with trailing ranks (32, 16); a leading extent whose Gram matrix is too large
+        # for the eigensolver's shared-memory path (161..256) and one beyond its rotation-log path (> 256, which
+        # also takes the first mode out of the fused launch); a trailing extent (19) whose tile count is not built in
+        Workload("half65", 98, (3, 4, 128, 65), (2, 3, 32, 16), (1, 100), 3, 5,
+                 outlier_frac=(1, 200), outlier_scale=20.0, noise_scale=0.02, half_storage=True),
+        Workload("lead200", 99, (200, 6, 8, 5), (4, 3, 3, 2), (1, 50), 3, 5,
+                 outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.02),
+        Workload("lead300", 100, (300, 5, 8, 5), (4, 3, 3, 2), (1, 50), 3, 5,
+                 outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.02),
+        Workload("tail19", 101, (5, 6, 16, 19), (3, 3, 4, 3), (1, 50), 3, 5,
+                 outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.05),
+        # the matrix case (N = 2)
+        Workload("mat2", 102, (96, 80), (12, 10), (1, 50), 3, 7,
+                 outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.02),
         # the five benchmark configurations
         Workload("cfg1", 1, (32, 32, 16, 9), (8, 8, 4, 3), (1, 100), 5, 20,
                  outliers_equal_k=True, outlier_scale=20.0, noise_scale=0.01, lr=1e-3),

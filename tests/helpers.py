@@ -31,6 +31,30 @@ def rel_err(a, b, floor_frac=FLOOR_FRAC):
     return float(np.max(np.abs(a - b) / den))
 
 
+FLOOR_CONTRACT = 1e-3
+
+
+def below_floor_fraction(b, floor_frac=FLOOR_CONTRACT):
+    """Share of the reference entries smaller than tau = floor_frac * rms(b)."""
+    b = np.asarray(b).reshape(-1).astype(np.complex128)
+    if b.size == 0:
+        return 0.0
+    rms = np.sqrt(np.mean(np.abs(b) ** 2))
+    return float(np.mean(np.abs(b) < floor_frac * rms))
+
+
+def tightest_floor_log2(a, b, tol=1e-4, lo=5, hi=16):
+    """Largest j in [lo, hi] such that rel_err(a, b, 2^-j) <= tol (the error is monotone in the floor);
+    lo - 1 if even 2^-lo fails."""
+    best = lo - 1
+    for j in range(lo, hi + 1):
+        if rel_err(a, b, 2.0 ** -j) <= tol:
+            best = j
+        else:
+            break
+    return best
+
+
 def fro_err(a, b):
     a = np.asarray(a).reshape(-1).astype(np.complex128)
     b = np.asarray(b).reshape(-1).astype(np.complex128)

@@ -16,7 +16,8 @@ from paper_2501_02379_b200 import synth
 from tests import helpers as H
 
 TOL_FLOAT = 1e-4       # max relative error, entries measured against max(|ref|, 2^-5 rms(ref)); see helpers.rel_err
-TOL_FRO = 5e-6         # and the whole array: ||a - b||_F / ||b||_F (split-TF32 products carry 2^-21 relative error)
+TOL_FRO = 5e-6         # and the whole array: ||a - b||_F / ||b||_F (split-TF32 products carry 2^-21 relative error
+                       # each, and an entry passes through up to 2 N of them)
 TOL_ANGLE = 1e-3       # largest principal-angle sine of a refreshed factor
 TOL_ORTHO = 1e-5       # max |U^H U - I|
 
@@ -58,6 +59,25 @@ class Pair:
 
     def _note(self, name, val):
         self.report[name] = max(self.report.get(name, 0.0), float(val))
+
+    def _note_min(self, name, val):
+        self.report[name] = min(self.report.get(name, 1e9), float(val))
+
+    def sync_oracle_from_gpu(self):
+        """Snapshot parity: the oracle takes over the whole exported GPU state (counter, Omega, factors, all
+        four moments, weight), so that its next step starts from exactly what the GPU's next step starts from."""
+        gst, ost = self.gst, self.ost
+        flags, t, _ = gst.query_status()
+        assert flags == 0, f"sticky flags {flags}"
+        ost.t = t
+        ost.factors = gst.factors()
+        ost.m_l, ost.v_l = gst.export(B.WHAT_M_L), gst.export(B.WHAT_V_L)
+        if self.wl.k > 0:
+            ost.omega = gst.export(B.WHAT_OMEGA)
+            ost.m_s, ost.v_s = gst.export(B.WHAT_M_S), gst.export(B.WHAT_V_S)
+        else:
+            ost.omega = np.zeros(0, np.uint32)
+        self.w_ref = from_device(self.w_dev, self.half)
 
     def refresh(self, g: np.ndarray, g_dev: torch.Tensor):
         before = g_dev.clone()
@@ -122,6 +142,15 @@ class Pair:
             e = H.rel_err(a, b)
             self._note(name, e)
             assert e <= TOL_FLOAT, f"{name}: max relative error {e} at t={ost.t - 1}"
+            # the same metric at the floor 1e-3 rms: asserted where the quantity is element-wise (the sparse
+            # moments), reported for the contracted quantities together with the tightest passing floor
+            e3 = H.rel_err(a, b, H.FLOOR_CONTRACT)
+            self._note(name + "@1e-3", e3)
+            if name in ("m_s", "v_s"):
+                assert e3 <= TOL_FLOAT, f"{name}: max relative error {e3} at the 1e-3 rms floor"
+            elif a.size <= (1 << 22):
+                self._note_min(name + "_floor_log2", H.tightest_floor_log2(a, b, TOL_FLOAT))
+                self._note(name + "_below_1e-3", H.below_floor_fraction(b))
             f = H.fro_err(a, b)
             self._note(name + "_fro", f)
             assert f <= TOL_FRO, f"{name}: Frobenius error {f} at t={ost.t - 1}"
@@ -137,9 +166,10 @@ class Pair:
             assert frac >= 0.999, f"only {frac} of the fp16 weights are bit-identical"
             self.w_ref = w_gpu          # follow the GPU's rounding so one-ulp choices do not compound
         else:
-            e = H.rel_err(w_gpu, self.w_ref)
-            self._note("w", e)
-            assert e <= TOL_FLOAT, f"weights: max relative error {e}"
+            e = H.rel_err(w_gpu, self.w_ref, H.FLOOR_CONTRACT)
+            self._note("w@1e-3", e)
+            assert e <= TOL_FLOAT, f"weights: max relative error {e} at the 1e-3 rms floor"
+        assert gst.query_status()[0] == 0, "sticky device flags after a step"
 
 
 # ---------------------------------------------------------------------------------------------
@@ -189,11 +219,36 @@ def gram_entry(r: np.ndarray, n: int, a: int, b: int):
     return complex(orc.mode_gram(sub, n)[0, 1])
 
 
-class SampledChecker:
-    """Refresh + steps at full size, checked on sampled outputs and on everything that is
-    element-wise (both Adam updates), using the GPU's own exported inputs for each stage."""
+def full_core_by_slices(r: np.ndarray, factors) -> np.ndarray:
+    """R x_1 U1^H ... x_N UN^H in complex128 without a complex128 copy of R: the leading mode is summed slice by
+    slice (linearity), and inside a slice the modes are contracted last-first with the oracle's mode product
+    (mode products commute; the oracle's pins check that on small tensors)."""
+    uh = [np.conj(np.asarray(u, dtype=np.complex128)).T for u in factors]
+    core = np.zeros([u.shape[1] for u in factors], dtype=np.complex128)
+    nd = r.ndim - 1
+    for i1 in range(r.shape[0]):
+        x = np.asarray(r[i1], dtype=np.complex128)
+        for n in range(nd - 1, -1, -1):
+            x = orc.mode_n_product(x, uh[n + 1], n)
+        core += uh[0][:, i1].reshape((-1,) + (1,) * nd) * x[None]
+    return core
 
-    def __init__(self, wl: synth.Workload, tensor_id=0, n_samples=6, seed=0, warm_refresh=False):
+
+def dense_update_slab(n_l: np.ndarray, factors, lead):
+    """The trailing A x B slab at leading indices `lead` of N_L x_1 U1 ... x_N UN: one reconstruction call of the
+    oracle on factors whose leading modes are cut down to the wanted row."""
+    fs = [np.ascontiguousarray(u[i:i + 1, :]) for u, i in zip(factors, lead)] + list(factors[len(lead):])
+    return orc.tucker_reconstruct(n_l, fs).reshape(factors[-2].shape[0], factors[-1].shape[0])
+
+
+class SampledChecker:
+    """Refresh + steps at a size where a full oracle step is out of reach (the 545 M-entry configuration): Omega
+    by its defining properties, sampled Gram entries, the factors against an eigen-decomposition of the exported
+    Gram matrices, the whole compressed gradient, both Adam updates in full, and the updated weight on whole
+    slabs (first slabs, every slab of the last leading index -- which holds the partly filled last round of the
+    streaming kernels -- and random ones), every entry compared."""
+
+    def __init__(self, wl: synth.Workload, tensor_id=0, n_samples=6, n_random_slabs=64, seed=0, warm_refresh=False):
         self.wl = wl
         self.half = wl.half_storage
         self.src = synth.GradientSource(wl, tensor_id)
@@ -204,6 +259,7 @@ class SampledChecker:
         self.w_dev = to_device(self.w, self.half)
         self.rng = np.random.default_rng(seed)
         self.n_samples = n_samples
+        self.n_random_slabs = n_random_slabs
         self.t = 0
         self.m_l = np.zeros(wl.ranks, np.complex64); self.v_l = np.zeros(wl.ranks, np.float32)
         self.m_s = np.zeros(wl.k, np.complex64); self.v_s = np.zeros(wl.k, np.float32)
@@ -241,6 +297,16 @@ class SampledChecker:
             assert od <= TOL_ORTHO, (n, od)
         return r
 
+    def _slab_list(self):
+        wl = self.wl
+        lead_shape = wl.shape[:-2]
+        nslab = int(np.prod(lead_shape))
+        per_last = nslab // lead_shape[0]
+        picks = set(range(min(4, nslab)))
+        picks.update(range(nslab - per_last, nslab))                    # every slab of the last leading index
+        picks.update(int(x) for x in self.rng.integers(0, nslab, self.n_random_slabs))
+        return sorted(picks), lead_shape
+
     def step(self, refresh=False):
         wl, t = self.wl, self.t
         g = storage_exact(self.src.gradient(t), self.half)
@@ -252,15 +318,14 @@ class SampledChecker:
         self.st.step(self.w_dev, g_dev)
         torch.cuda.synchronize()
         st = self.st
-        # compressed gradient: sampled entries against the definition
+        assert st.query_status()[0] == 0
+        # compressed gradient: every entry
         core = st.export(B.WHAT_CORE)
-        rms = float(np.sqrt(np.mean(np.abs(core.astype(np.complex128)) ** 2)))
-        for _ in range(self.n_samples):
-            j = tuple(int(self.rng.integers(0, rr)) for rr in wl.ranks)
-            want = core_entry(r, self.factors, j)
-            err = abs(complex(core[j]) - want) / max(abs(want), H.FLOOR_FRAC * rms)
-            self._note("core", err)
-            assert err <= TOL_FLOAT, (j, err)
+        want_core = full_core_by_slices(r, self.factors)
+        e = H.rel_err(core, want_core); self._note("core", e); assert e <= TOL_FLOAT, ("core", e)
+        f = H.fro_err(core, want_core); self._note("core_fro", f); assert f <= TOL_FRO, ("core", f)
+        self._note("core@1e-3", H.rel_err(core, want_core, H.FLOOR_CONTRACT))
+        del r
         # both Adam updates in full (element-wise), from the GPU's own compressed inputs
         n_l, self.m_l, self.v_l = orc.adam_update(core, self.m_l, self.v_l, 0.9, 0.999, 1e-8, t)
         for name, a, b in (("n_l", st.export(B.WHAT_N_L), n_l), ("m_l", st.export(B.WHAT_M_L), self.m_l),
@@ -271,33 +336,40 @@ class SampledChecker:
         n_s_gpu = st.export(B.WHAT_N_S)
         for name, a, b in (("n_s", n_s_gpu, n_s), ("m_s", st.export(B.WHAT_M_S), self.m_s),
                            ("v_s", st.export(B.WHAT_V_S), self.v_s)):
-            e = H.rel_err(a, b); self._note(name, e); assert e <= TOL_FLOAT, (name, e)
-        # weights: sampled entries inside and outside Omega
+            e = H.rel_err(a, b, H.FLOOR_CONTRACT); self._note(name, e); assert e <= TOL_FLOAT, (name, e)
+        # weights: whole slabs, every entry
         w_new = from_device(self.w_dev, self.half)
         n_l_gpu = st.export(B.WHAT_N_L)
         lr = float(np.float32(wl.lr))
         om = self.omega.astype(np.int64)
-        picks = list(self.rng.integers(0, wl.numel, self.n_samples)) + list(om[self.rng.integers(0, om.size, 3)] if om.size else [])
-        w_rms = float(np.sqrt(np.mean(np.abs(self.w.astype(np.complex128)) ** 2)))
-        for flat in picks:
-            idx = np.unravel_index(int(flat), wl.shape)
-            d = dense_update_entry(n_l_gpu, self.factors, idx)
-            want = np.complex128(self.w[idx]) - lr * d
+        slabs, lead_shape = self._slab_list()
+        E = wl.shape[-2] * wl.shape[-1]
+        n_checked = n_same = 0
+        w_rms = float(np.sqrt(np.mean(np.abs(self.w[tuple(0 for _ in lead_shape)].astype(np.complex128)) ** 2)))
+        for s_ in slabs:
+            lead = np.unravel_index(s_, lead_shape)
+            d = dense_update_slab(n_l_gpu, self.factors, lead)
+            want = self.w[lead].astype(np.complex128) - lr * d
+            j0, j1 = np.searchsorted(om, [s_ * E, (s_ + 1) * E])
+            loc = om[j0:j1] - s_ * E
             if self.half:
-                want = complex(np.float16(want.real)) + 1j * complex(np.float16(want.imag)).real
-            pos = np.searchsorted(om, flat)
-            if pos < om.size and om[pos] == flat:
-                want = want - lr * complex(n_s_gpu[pos])
-                if self.half:
-                    want = complex(np.float16(want.real)) + 1j * complex(np.float16(want.imag)).real
-            got = complex(w_new[idx])
-            if self.half:
-                ulp = max(np.spacing(np.float16(abs(want.real))), np.spacing(np.float16(abs(want.imag))))
-                assert abs(got - want) <= 1.01 * float(ulp) * np.sqrt(2), (idx, got, want)
+                want = synth.from_half_pairs(synth.to_half_pairs(want.astype(np.complex64))).astype(np.complex128)
+                wf = want.reshape(-1)
+                wf[loc] = wf[loc] - lr * n_s_gpu[j0:j1].astype(np.complex128)
+                a = synth.to_half_pairs(w_new[lead]).view(np.int16).astype(np.int32)
+                b = synth.to_half_pairs(want.astype(np.complex64)).view(np.int16).astype(np.int32)
+                dd = np.abs(a - b)
+                assert dd.max() <= 1, (lead, int(dd.max()))
+                n_checked += dd.size; n_same += int((dd == 0).sum())
             else:
-                err = abs(got - want) / max(abs(want), H.FLOOR_FRAC * w_rms)
+                wf = want.reshape(-1)
+                wf[loc] = wf[loc] - lr * n_s_gpu[j0:j1].astype(np.complex128)
+                err = np.max(np.abs(w_new[lead] - want) / np.maximum(np.abs(want), H.FLOOR_CONTRACT * w_rms))
                 self._note("w", err)
-                assert err <= TOL_FLOAT, (idx, err)
-        # untouched-by-construction invariant: the update is small against |W|
+                assert err <= TOL_FLOAT, (lead, err)
+        if self.half:
+            self._note("w_mismatch_frac", 1.0 - n_same / n_checked)
+            assert n_same >= 0.999 * n_checked
+        self.report["slabs_checked"] = len(slabs)
         self.w = w_new
         self.t += 1

@@ -59,7 +59,7 @@ def test_state_bytes_counts_the_papers_inventory():
 @pytest.mark.parametrize("mutate,status", [
     (lambda c: setattr(c, "ndim", 1), B.ERR_INVALID_ARG),
     (lambda c: setattr(c, "ndim", 9), B.ERR_INVALID_ARG),
-    (lambda c: setattr(c, "ndim", 2), B.ERR_UNSUPPORTED),
+    (lambda c: setattr(c, "ndim", 2), B.OK),                          # the matrix case
     (lambda c: c.ranks.__setitem__(0, 0), B.ERR_INVALID_ARG),
     (lambda c: c.ranks.__setitem__(1, 1000), B.ERR_INVALID_ARG),
     (lambda c: c.dims.__setitem__(2, 0), B.ERR_INVALID_ARG),
@@ -70,6 +70,8 @@ def test_state_bytes_counts_the_papers_inventory():
     (lambda c: setattr(c, "beta1", 1.0), B.ERR_INVALID_ARG),
     (lambda c: setattr(c, "eps", -1.0), B.ERR_INVALID_ARG),
     (lambda c: c.dims.__setitem__(0, 2000), B.ERR_UNSUPPORTED),        # eigensolver size limit
+    (lambda c: (c.dims.__setitem__(3, 40), c.ranks.__setitem__(3, 33)), B.ERR_UNSUPPORTED),   # r_N <= 32
+    (lambda c: (c.dims.__setitem__(2, 600), c.dims.__setitem__(3, 100)), B.ERR_UNSUPPORTED),  # slab > shared memory
 ])
 def test_bad_configs_are_rejected_on_the_host(mutate, status):
     cfg = B.make_config((12, 10, 8, 5), (4, 3, 3, 2), 10, 4)
@@ -82,6 +84,40 @@ def test_too_many_entries_for_uint32_indices():
     cfg = B.make_config((1024, 1024, 1024, 8), (4, 4, 4, 4), 10, 4)
     p, w = C.c_size_t(0), C.c_size_t(0)
     assert B.lib().tgrad_state_bytes(C.byref(cfg), C.byref(p), C.byref(w)) == B.ERR_UNSUPPORTED
+
+
+def test_k_of_two_to_the_31_is_unsupported():
+    # 2^31 <= k <= prod(dims) < 2^32 would overflow the int slot arithmetic of the kernels: refused on the host
+    cfg = B.make_config((1024, 1024, 1024, 3), (4, 4, 4, 3), 1 << 31, 4)
+    p, w = C.c_size_t(0), C.c_size_t(0)
+    assert B.lib().tgrad_state_bytes(C.byref(cfg), C.byref(p), C.byref(w)) == B.ERR_UNSUPPORTED
+    cfg.k = (1 << 31) - 1
+    assert B.lib().tgrad_state_bytes(C.byref(cfg), C.byref(p), C.byref(w)) == B.OK
+
+
+def test_noalloc_entry_point_rejects_misaligned_pointers_without_a_launch():
+    # pointers are plain integers here: the call must return before it touches a device
+    l = B.lib()
+    n0 = B.launch_count()
+    for g, o, v in ((0x1004, 0x2000, 0x3000), (0x1000, 0x2004, 0x3000), (0x1000, 0x2000, 0x3008)):
+        assert l.tgrad_select_topk_noalloc(g, 64, 4, B.C64, o, v, None) == B.ERR_INVALID_ARG
+    assert l.tgrad_select_topk_noalloc(0x1004, 64, 4, B.C32H, 0x2000, 0x3000, None) == B.ERR_INVALID_ARG
+    assert B.launch_count() == n0
+
+
+def test_sticky_flag_names_match_the_header():
+    header = open(os.path.join(ROOT, "include", "tgrad.h")).read()
+    vals = dict(re.findall(r"#define (TGRAD_FLAG_[A-Z_]+)\s+(\d+)", header))
+    assert vals == {"TGRAD_FLAG_NO_CONVERGE": str(B.FLAG_NO_CONVERGE), "TGRAD_FLAG_NONFINITE": str(B.FLAG_NONFINITE),
+                    "TGRAD_FLAG_COPY_TIMEOUT": str(B.FLAG_COPY_TIMEOUT)}
+
+
+def test_state_sizes_of_a_matrix():
+    # N = 2: factors I_1 x r_1 and I_2 x r_2, core r_1 x r_2
+    cfg = B.make_config((96, 80), (12, 10), 77, 4)
+    pb, wb = B.state_bytes(cfg)
+    need = 4 * 77 + 8 * (96 * 12 + 80 * 10) + 12 * 120 + 12 * 77
+    assert need <= pb <= need + 8192 and wb > 0
 
 
 def test_null_and_misaligned_arguments():

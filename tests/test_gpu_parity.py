@@ -12,7 +12,8 @@ from tests.parity import Pair, to_device, from_device
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name", ["tiny4", "small4", "small5", "ragged4", "small3", "odd4", "odd32", "small5b"])
+@pytest.mark.parametrize("name", ["tiny4", "small4", "small5", "ragged4", "small3", "odd4", "odd32", "small5b",
+                                  "half65", "lead200", "lead300", "tail19", "mat2"])
 def test_trajectory_small(name):
     wl = synth.WORKLOADS[name]
     p = Pair(wl)

@@ -261,6 +261,31 @@ def test_real_inputs_full_rank_match_torch_adam():
     assert np.max(np.abs(w.real - p.detach().numpy())) < 2e-6
 
 
+def test_weight_decay_matches_torch_adamw():
+    # Decoupled decay has a definition outside this repository: torch.optim.AdamW multiplies the
+    # parameter by (1 - lr * wd) and then applies the Adam update.  lr * wd = 0.025 is large enough
+    # that decaying after the update, or by (1 - wd), or not at all, misses by far more than the bound.
+    rng = np.random.default_rng(21)
+    shape = (3, 4, 2)
+    lr, wd = 0.05, 0.5
+    w0 = rng.standard_normal(shape).astype(np.float32)
+    grads = [rng.standard_normal(shape).astype(np.float32) for _ in range(8)]
+    p = torch.nn.Parameter(torch.tensor(w0, dtype=torch.float64))
+    opt = torch.optim.AdamW([p], lr=float(np.float32(lr)), betas=(float(np.float32(0.9)), float(np.float32(0.999))),
+                            eps=float(np.float32(1e-8)), weight_decay=float(np.float32(wd)))
+    st = _identity_state(shape, lr, weight_decay=wd)
+    w = w0.astype(np.complex64)
+    for g in grads:
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        w = orc.oracle_step(st, w, g.astype(np.complex64), refresh=False)
+    assert np.max(np.abs(w.imag)) == 0
+    assert np.max(np.abs(w.real - p.detach().numpy())) < 3e-6
+    # the planted mistakes are far outside that bound
+    u = float(np.float32(lr))
+    assert u * u * wd > 1e-4
+
+
 # ---- structure of Algorithm 1 -----------------------------------------------------------------------
 
 def _run(wl_name, steps, **over):
@@ -362,6 +387,30 @@ def test_half_storage_rounds_to_fp16():
     w1 = orc.oracle_step(st, w, g)
     assert np.array_equal(synth.from_half_pairs(synth.to_half_pairs(w1)), w1)
     assert not np.array_equal(w1, w)
+
+
+def test_half_storage_rounds_after_the_dense_update_and_again_at_omega():
+    # Hand-computed case in which rounding once and rounding twice give different fp16 values.
+    # Tensor of shape (2, 1), U1 = [1, 1]^T / sqrt(2), U2 = [1], Omega = {0}, first step (zero moments), so
+    # N_S = g0 / (|g0| + eps) = 1 and N_L = core / (|core| + eps) = 1 (up to 1e-8), and the dense update is
+    # N_L / sqrt(2) on both entries.  With u = 2^-10 (the fp16 spacing in [1, 2)), lr = 0.6 u, lambda = 1 and
+    # alpha = sqrt(2) both updates are 0.6 u:
+    #   entry 0 (in Omega):  1.5 - 0.6u -> fp16 -> 1.5 - u;  (1.5 - u) - 0.6u = 1.5 - 1.6u -> fp16 -> 1.5 - 2u
+    #                        (a single rounding of 1.5 - 1.2u would give 1.5 - u)
+    #   entry 1 (outside):   1.5 - 0.6u -> 1.5 - u
+    # The imaginary parts get no update (the gradient is real) and stay 1.5.
+    u = 2.0 ** -10
+    cfg = orc.OracleConfig(shape=(2, 1), ranks=(1, 1), k=1, T=1000, lr=0.6 * u, alpha=float(np.sqrt(2.0)), lam=1.0,
+                           half_storage=True)
+    st = orc.OracleState(cfg)
+    st.omega = np.array([0], np.uint32)
+    st.factors = [np.array([[1.0], [1.0]], np.complex64) / np.float32(np.sqrt(2.0)), np.ones((1, 1), np.complex64)]
+    w = np.full((2, 1), 1.5 + 1.5j, np.complex64)
+    g = np.array([[8.0], [2.0]], np.complex64)
+    w1 = orc.oracle_step(st, w, g, refresh=False)
+    assert w1[0, 0] == np.complex64(complex(1.5 - 2 * u, 1.5))
+    assert w1[1, 0] == np.complex64(complex(1.5 - u, 1.5))
+    assert float(np.float16(1.5 - 1.2 * u)) == 1.5 - u          # what one rounding would have stored at Omega
 
 
 # ---- state size: the paper's worked example --------------------------------------------------

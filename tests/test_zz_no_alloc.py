@@ -1,4 +1,4 @@
-"""The allocation-free top-k entry point against the regular refresh (run with -m gpu on a B200).
+"""The allocation-free top-k entry point against the regular refresh and the CPU oracle (run with -m gpu on a B200).
 
 Some callers of this library may not allocate device memory while they call it: an allocator
 hook that would re-enter itself, a process whose device memory was handed out in full at
@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import tgrad_oracle as orc
 from paper_2501_02379_b200 import binding as B
 from paper_2501_02379_b200 import synth
 from tests.parity import to_device
@@ -39,6 +40,7 @@ def test_noalloc_topk_matches_refresh_twice_in_a_row():
         got = omega[:k].cpu().numpy().view(np.uint32)
         want = _reference_omega(g_dev, wl.shape, wl.ranks, k)
         assert np.array_equal(got, want)                                   # integer work: bit-exact
+        assert np.array_equal(got, orc.sparse_indices_topk(g, k))          # and what the definition gives
         vals = values[:k].cpu().numpy().view(np.complex64)[:, 0]
         assert np.array_equal(vals, g.reshape(-1)[want.astype(np.int64)])  # a gather: bit-exact
 
