@@ -92,14 +92,13 @@ typedef struct {
   int32_t auto_refresh;             /* 1: tgrad_step refreshes Omega and U^(n) when t % T == 0  */
   int32_t jacobi_max_sweeps;        /* sweep cap of the eigensolver (0 -> default 30)           */
   float jacobi_tol;                 /* off-diagonal tolerance relative to max diag (0 -> 1e-6)  */
-  int32_t warm_refresh;             /* 1: the eigensolver of a refresh starts from the eigenvectors of the
-                                       previous refresh (the paper's "warm restart" of the factors, section
-                                       "Tucker decomposition"): A_n is first rotated into that basis, where it is
-                                       already close to diagonal if the subspace moved little, which saves
-                                       sweeps; the result is the same eigen-decomposition to the same tolerance.
-                                       The I_n x I_n bases are kept in the persistent block (not exported: a
-                                       resumed state starts its first refresh cold).  0: every refresh starts
-                                       from the identity                                                     */
+  int32_t warm_refresh;             /* 1: a refresh starts its eigenvector iteration from the factor matrices
+                                       the state holds (the paper's "warm restart" of the factors, appendix
+                                       "Tensor Decomposition / Implementation") instead of a fixed pseudo-random
+                                       start; if the subspace moved little this saves iterations, and the result
+                                       is the same eigen-decomposition to the same tolerance.  Stored factors
+                                       that are unusable (never set, not finite) are noticed on the device and
+                                       that refresh starts cold.  0: every refresh starts cold               */
 } tgrad_config;
 
 /* Selectors for tgrad_export_state / tgrad_import_state.  FACTOR_BASE + n is

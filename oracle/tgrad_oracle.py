@@ -239,6 +239,27 @@ def oracle_refresh(st: OracleState, grad: np.ndarray) -> None:
     st.factors = tucker_factors(residual(grad, st.omega), cfg.ranks)
 
 
+def weight_update(cfg: OracleConfig, w: np.ndarray, n_l: np.ndarray, n_s: np.ndarray, omega: np.ndarray,
+                  factors: Sequence[np.ndarray]) -> np.ndarray:
+    """The last statements of the loop body of Algorithm 1 ("reconstruct low-rank part", "add scaled sparse
+    tensor", "update weights"), signs flipped as the module docstring says:
+
+        W <- (1 - eta wd) W;  W <- W - eta alpha (N_L x_1 U1 ... x_N UN);  W[Omega] <- W[Omega] - eta lambda N_S
+
+    with one rounding to the storage type after the dense update and one more, at Omega, after the sparse add."""
+    lr = float(np.float32(cfg.lr)); al = float(np.float32(cfg.alpha)); la = float(np.float32(cfg.lam))
+    wd = float(np.float32(cfg.weight_decay))
+    wn = np.asarray(w, dtype=np.complex128)
+    if wd != 0.0:
+        wn = wn * (1.0 - lr * wd)
+    d = tucker_reconstruct(n_l, factors)
+    wn = np.ascontiguousarray(_store_w(wn - (lr * al) * d, cfg.half_storage))
+    flat = wn.reshape(-1)                          # a view of the contiguous array
+    om = np.asarray(omega).astype(np.int64)
+    flat[om] = _store_w(flat[om] - (lr * la) * np.asarray(n_s, dtype=np.complex128), cfg.half_storage)
+    return wn.astype(np.complex64)
+
+
 def oracle_step(st: OracleState, w: np.ndarray, grad: np.ndarray, refresh: Optional[bool] = None) -> np.ndarray:
     """One pass of the loop body of Algorithm 1 for one tensor.
 
@@ -251,7 +272,6 @@ def oracle_step(st: OracleState, w: np.ndarray, grad: np.ndarray, refresh: Optio
     do_refresh = (st.t % cfg.T == 0) if refresh is None else refresh
     if do_refresh:
         oracle_refresh(st, grad)
-    omega = st.omega.astype(np.int64)
     # sparse values, residual, low-rank compression
     g_s = sparse_gather(grad, st.omega).astype(np.complex64)
     core = tucker_compress(residual(grad, st.omega), st.factors).astype(np.complex64)
@@ -259,19 +279,10 @@ def oracle_step(st: OracleState, w: np.ndarray, grad: np.ndarray, refresh: Optio
     n_s, st.m_s, st.v_s = adam_update(g_s, st.m_s, st.v_s, cfg.beta1, cfg.beta2, cfg.eps, st.t)
     n_l, st.m_l, st.v_l = adam_update(core, st.m_l, st.v_l, cfg.beta1, cfg.beta2, cfg.eps, st.t)
     n_s = n_s.astype(np.complex64); n_l = n_l.astype(np.complex64)
-    # reconstruction, scaled sparse add, weight update (signs flipped, see module docstring)
-    lr = float(np.float32(cfg.lr)); al = float(np.float32(cfg.alpha)); la = float(np.float32(cfg.lam))
-    wd = float(np.float32(cfg.weight_decay))
-    wn = np.asarray(w, dtype=np.complex128)
-    if wd != 0.0:
-        wn = wn * (1.0 - lr * wd)
-    d = tucker_reconstruct(n_l, st.factors)
-    wn = np.ascontiguousarray(_store_w(wn - (lr * al) * d, cfg.half_storage))
-    flat = wn.reshape(-1)                          # a view of the contiguous array
-    flat[omega] = _store_w(flat[omega] - (lr * la) * n_s.astype(np.complex128), cfg.half_storage)
+    wn = weight_update(cfg, w, n_l, n_s, st.omega, st.factors)
     st.core, st.n_l, st.g_s, st.n_s = core, n_l, g_s, n_s
     st.t += 1
-    return wn.astype(np.complex64)
+    return wn
 
 
 def state_entries(shape, ranks, k):

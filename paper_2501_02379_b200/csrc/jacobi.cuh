@@ -26,13 +26,18 @@ struct JacobiParams {
   int index[8];     // tensor mode each entry belongs to
   int max_sweeps;
   float tol;
-  int* flags;   // flags[0] sticky bits, flags[1 + mode] sweeps used
+  int* flags;   // flags[0] sticky bits, flags[1 + mode] sweeps used, flags[JAC_SKIP + mode] != 0: nothing to do
 };
+
+// A mode whose factor matrix this refresh has already been produced (by the subspace iteration) is skipped by every
+// kernel of this file.
+constexpr int JAC_SKIP = 16;
 
 struct JacRot { float c, s, gx, gy, npp, nqq; int p, q; };
 
 __global__ void __launch_bounds__(JAC_THREADS) jacobi_kernel(JacobiParams P) {
   const JacobiMode md = P.mode[blockIdx.x];
+  if (P.flags[JAC_SKIP + P.index[blockIdx.x]]) return;
   const int n = md.n, r = md.r;
   cf* __restrict__ A = md.A;
   cf* __restrict__ V = md.V;
@@ -184,8 +189,7 @@ constexpr int JAC_SMEM_MAX_N = 160;      // 160^2 complex64 = 200 KB of shared m
 constexpr int JAC_FAST_MAX_N = 256;      // up to here the same kernel runs with the matrix in global memory (L2)
 
 struct JacobiFastMode {
-  const cf* A;       // n x n input (left untouched); with a warm start, A_n rotated into the previous basis
-  const cf* A0;      // A_n itself: what is diagonalised when the previous basis turns out to be unusable
+  const cf* A;       // n x n input (left untouched)
   cf* work;          // n x (n | 1) working copy in global memory, used when n > JAC_SMEM_MAX_N
   float4* log;       // [sweeps][m-1][m/2] rotations
   float* lam;        // out: n eigenvalues (unsorted)
@@ -201,16 +205,8 @@ struct JacobiFastParams {
   int row_stride;    // jacobi_vectors_kernel: complex entries per warp row buffer (>= largest n)
   int max_sweeps;
   float tol;
-  int* flags;        // flags[0] sticky bits, flags[1 + mode] sweeps used
-  int warm;          // V holds the basis the matrix was rotated into; the rotations are applied to it in place
+  int* flags;        // flags[0] sticky bits, flags[1 + mode] sweeps used, flags[JAC_SKIP + mode]
 };
-
-// Whether mode `index` of this refresh starts from the previous basis: asked for, and the basis passed the check of
-// ns_residual_kernel (flags[JAC_BAD_BASIS + index] stays 0).
-constexpr int JAC_BAD_BASIS = 16;
-__device__ __forceinline__ bool jac_warm(const JacobiFastParams& P, int index) {
-  return P.warm && P.flags[JAC_BAD_BASIS + index] == 0;
-}
 
 // the pair of players (p < q) that meet at table `tb` in stage `stage` of a round robin of m players
 __host__ __device__ inline size_t jac_log_entries(int n, int max_sweeps) {
@@ -294,6 +290,7 @@ template <bool INSMEM>
 __global__ void __launch_bounds__(JAC_THREADS) jacobi_sweeps_kernel(JacobiFastParams P) {
   extern __shared__ __align__(16) unsigned char jsm[];
   const JacobiFastMode md = P.mode[blockIdx.x];
+  if (P.flags[JAC_SKIP + md.index]) return;
   const int n = md.n;
   const int m = (n + 1) & ~1, half = m >> 1;
   cf* A = INSMEM ? reinterpret_cast<cf*>(jsm) : md.work;               // [n][n | 1], upper triangle live
@@ -303,7 +300,7 @@ __global__ void __launch_bounds__(JAC_THREADS) jacobi_sweeps_kernel(JacobiFastPa
   __shared__ float red[32];
   const int tid = threadIdx.x, nt = blockDim.x;
   const int ld = n | 1;      // odd row stride: column accesses (the mirrored half) spread over the banks
-  const cf* Ain = jac_warm(P, md.index) ? md.A : md.A0;
+  const cf* Ain = md.A;
   for (int i = tid; i < n * n; i += nt) { const int r_ = i / n, c_ = i - r_ * n; A[(size_t)r_ * ld + c_] = Ain[i]; }
   __syncthreads();
   float dmax = 0.f;
@@ -422,20 +419,6 @@ __global__ void __launch_bounds__(JAC_THREADS) jacobi_sweeps_kernel(JacobiFastPa
   for (int i = tid; i < n; i += nt) md.lam[i] = A[(size_t)i * ld + i].x;
 }
 
-// E = 3/2 I - 1/2 G in place: with G = V^H V, V E is one Newton-Schulz step of V towards orthonormal columns
-// (a defect d of V^H V - I becomes O(d^2)); keeps the basis carried from refresh to refresh from drifting.
-// Also the check of the carried basis: if G = V^H V is not finite or not close to I (a refresh on a non-finite
-// gradient leaves such a V behind), *bad is set and this refresh diagonalises A_n itself, from the identity.
-__global__ void ns_residual_kernel(cf* __restrict__ G, int n, int* __restrict__ bad) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= n * n) return;
-  const int i = idx / n, j = idx - i * n;
-  const cf g = G[idx];
-  const float dx = g.x - (i == j ? 1.f : 0.f);
-  if (!(fabsf(dx) < 0.25f) || !(fabsf(g.y) < 0.25f)) *bad = 1;          // also catches NaN
-  G[idx] = make_float2((i == j ? 1.5f : 0.f) - 0.5f * g.x, -0.5f * g.y);
-}
-
 // NP = pairs per lane (>= n/64), D = stages of the log kept in flight
 template <int NP, int D>
 __global__ void __launch_bounds__(256) jacobi_vectors_kernel(JacobiFastParams P) {
@@ -447,12 +430,12 @@ __global__ void __launch_bounds__(256) jacobi_vectors_kernel(JacobiFastParams P)
   int mi = 0;
   for (int i = 1; i < P.nmodes; ++i) if (gw >= P.mode[i].row0) mi = i;
   const JacobiFastMode md = P.mode[mi];
+  if (P.flags[JAC_SKIP + md.index]) return;
   const int n = md.n, i_row = gw - md.row0;
   const int m = (n + 1) & ~1, half = m >> 1;
   const int sweeps = P.flags[1 + md.index];
   cf* row = rows + (size_t)warp * P.row_stride;
-  const bool warm = jac_warm(P, md.index);
-  for (int j = lane; j < n; j += 32) row[j] = warm ? md.V[(size_t)i_row * n + j] : make_float2(j == i_row ? 1.f : 0.f, 0.f);
+  for (int j = lane; j < n; j += 32) row[j] = make_float2(j == i_row ? 1.f : 0.f, 0.f);
   __syncwarp();
   // the log is replayed D stages at a time, the next D already in flight
   const float4* lg = md.log;
@@ -501,6 +484,7 @@ __global__ void __launch_bounds__(256) jacobi_vectors_kernel(JacobiFastParams P)
 
 __global__ void __launch_bounds__(JAC_THREADS) jacobi_factors_kernel(JacobiFastParams P) {
   const JacobiFastMode md = P.mode[blockIdx.x];
+  if (P.flags[JAC_SKIP + md.index]) return;
   const int n = md.n, r = md.r;
   const cf* __restrict__ V = md.V;
   __shared__ float lam[JAC_FAST_MAX_N];

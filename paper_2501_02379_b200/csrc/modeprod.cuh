@@ -8,11 +8,11 @@
 // compressing and Aop = U (M = I_n, K = r_n) when reconstructing; U is the
 // I_n x r_n row-major factor matrix in both cases.
 //
-// These tensors are at most a few tens of MB and stay in L2, so the kernel is
-// bound by fp32 FMA issue: a block of 128 threads owns a 32 (m) x 64 (c) output
-// tile, a thread a 4 x 4 complex micro-tile (64 real FMAs per k for 4 shared
-// loads of 16 bytes); the next k-slice is fetched into registers while the
-// current one is being multiplied.
+// These tensors are at most a few tens of MB and stay in L2.  The products run on
+// the tensor cores as split-precision TF32 (mode_product_tc_kernel); products with
+// very few output rows and small slices use an fp32 kernel that keeps a whole slice
+// in shared memory (mode_product_small_kernel); the first mode is fused with the
+// AdamUpdate of the core (core_sandwich_tc_kernel).
 #pragma once
 #include "common.cuh"
 #include "ptx.cuh"
@@ -20,105 +20,8 @@
 
 namespace tg {
 
-constexpr int MP_BM = 32, MP_BK = 16, MP_THREADS = 128;
-
-// MP_BC = 64 (4 x 4 micro-tile) or 32 (4 x 2: twice the blocks, for products with few tiles)
-template <bool CONJ_T, int MP_BC>
-__global__ void __launch_bounds__(MP_THREADS) mode_product_kernel(const cf* __restrict__ in, cf* __restrict__ out,
-                                                                  const cf* __restrict__ U, int M, int K, int C, int r_n) {
-  __shared__ __align__(16) cf As[2][MP_BK][MP_BM];
-  __shared__ __align__(16) cf Bs[2][MP_BK][MP_BC];
-  const int tid = threadIdx.x;
-  constexpr int NC = MP_BC / 16;                   // columns per thread
-  const int tm = tid >> 4, tc = tid & 15;          // 8 x 16 threads: 4 rows (m) x NC cols (c) each
-  const int m0 = blockIdx.y * MP_BM, c0 = blockIdx.x * MP_BC;
-  const size_t o = blockIdx.z;
-  const cf* inb = in + o * (size_t)K * C;
-  constexpr int A_PER = MP_BK * MP_BM / MP_THREADS;   // 4
-  constexpr int B_PER = MP_BK * MP_BC / MP_THREADS;   // 8 or 4
-  cf ra[A_PER], rb[B_PER];
-
-  auto fetch = [&](int k0) {
-#pragma unroll
-    for (int i = 0; i < A_PER; ++i) {
-      const int idx = tid + i * MP_THREADS;
-      int kk, mm;
-      if (CONJ_T) { mm = idx % MP_BM; kk = idx / MP_BM; }   // U[k][m]: m contiguous
-      else { kk = idx % MP_BK; mm = idx / MP_BK; }          // U[m][k]: k contiguous
-      const int m = m0 + mm, k = k0 + kk;
-      cf v = make_float2(0.f, 0.f);
-      if (m < M && k < K) {
-        if (CONJ_T) { cf u = U[(size_t)k * r_n + m]; v = make_float2(u.x, -u.y); }
-        else v = U[(size_t)m * r_n + k];
-      }
-      ra[i] = v;
-    }
-#pragma unroll
-    for (int i = 0; i < B_PER; ++i) {
-      const int idx = tid + i * MP_THREADS;
-      const int cc = idx % MP_BC, kk = idx / MP_BC;
-      const int c = c0 + cc, k = k0 + kk;
-      rb[i] = (c < C && k < K) ? inb[(size_t)k * C + c] : make_float2(0.f, 0.f);
-    }
-  };
-  auto stash = [&](int buf) {
-#pragma unroll
-    for (int i = 0; i < A_PER; ++i) {
-      const int idx = tid + i * MP_THREADS;
-      int kk, mm;
-      if (CONJ_T) { mm = idx % MP_BM; kk = idx / MP_BM; }
-      else { kk = idx % MP_BK; mm = idx / MP_BK; }
-      As[buf][kk][mm] = ra[i];
-    }
-#pragma unroll
-    for (int i = 0; i < B_PER; ++i) {
-      const int idx = tid + i * MP_THREADS;
-      Bs[buf][idx / MP_BC][idx % MP_BC] = rb[i];
-    }
-  };
-
-  cf acc[4][NC];
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-#pragma unroll
-    for (int j = 0; j < NC; ++j) acc[i][j] = make_float2(0.f, 0.f);
-
-  fetch(0);
-  stash(0);
-  __syncthreads();
-  int buf = 0;
-  for (int k0 = 0; k0 < K; k0 += MP_BK) {
-    const bool more = k0 + MP_BK < K;
-    if (more) fetch(k0 + MP_BK);
-#pragma unroll
-    for (int kk = 0; kk < MP_BK; ++kk) {
-      cf a[4], b[NC];
-      load_row_bcast<4>(&As[buf][kk][tm * 4], a);
-      load_row_bcast<NC>(&Bs[buf][kk][tc * NC], b);
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < NC; ++j) cfma(acc[i][j], a[i], b[j]);
-    }
-    if (more) stash(buf ^ 1);
-    __syncthreads();
-    buf ^= 1;
-  }
-  cf* outb = out + o * (size_t)M * C;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int m = m0 + tm * 4 + i;
-    if (m >= M) continue;
-#pragma unroll
-    for (int j = 0; j < NC; ++j) {
-      const int c = c0 + tc * NC + j;
-      if (c < C) outb[(size_t)m * C + c] = acc[i][j];
-    }
-  }
-}
-
 // ---------------------------------------------------------------------------------------------
-// The same product for few output rows (M <= 8) and slices whose K C entries fit in shared memory: the 32-row
+// The product for few output rows (M <= 8) and slices whose K C entries fit in shared memory: the 32-row
 // tensor-core tiles would be mostly padding there.  A block walks over slices o;
 // the slice [K][C] and Aop sit in shared memory, a thread owns outputs (m, c) and sums over k in fp32.
 // ---------------------------------------------------------------------------------------------
@@ -179,7 +82,7 @@ __global__ void adam_kernel(const cf* __restrict__ core, cf* __restrict__ m_l, f
 }
 
 // ---------------------------------------------------------------------------------------------
-// The same product on the tensor cores, split-precision TF32 (hi*hi + lo*hi + hi*lo, fp32
+// The product on the tensor cores, split-precision TF32 (hi*hi + lo*hi + hi*lo, fp32
 // accumulation).  Real formulation with the rows of the output doubled instead of its columns:
 //   [out_re; out_im][m][c] = [[Ar, -Ai], [Ai, Ar]][m][k] . [Xr; Xi][k][c]
 // so that one 8-byte load of the complex entry X[k][c] is a whole B fragment (k = t <-> (k, re),
@@ -369,10 +272,35 @@ __global__ void __launch_bounds__(SW_THREADS) core_sandwich_tc_kernel(const cf* 
     Us[i * ldu + j] = (i < I1 && j < r1) ? U1[(size_t)i * r1 + j] : make_float2(0.f, 0.f);
   }
   griddep_chain();            // U1 alone was read so far; X is the previous kernel's output
-  for (int idx = tid; idx < I1p * SW_CB; idx += SW_THREADS) {
-    const int i = idx / SW_CB, cc = idx - i * SW_CB;
-    Xs[i * SWT_LDX + cc] = (i < I1 && c0 + cc < C) ? X[(size_t)i * C + c0 + cc] : make_float2(0.f, 0.f);
+  {
+    // the X block by asynchronous copies (zero-filled outside the tensor); meanwhile this thread's moments
+    const unsigned char* xb = reinterpret_cast<const unsigned char*>(X);
+    if ((C & 1) == 0) {
+      for (int idx = tid; idx < I1p * (SW_CB / 2); idx += SW_THREADS) {
+        const int i = idx / (SW_CB / 2), cc = 2 * (idx - i * (SW_CB / 2));
+        const bool ok = i < I1 && c0 + cc < C;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(&Xs[i * SWT_LDX + cc])),
+                     "l"(ok ? xb + ((size_t)i * C + c0 + cc) * 8 : xb), "r"(ok ? 16u : 0u) : "memory");
+      }
+    } else {
+      for (int idx = tid; idx < I1p * SW_CB; idx += SW_THREADS) {
+        const int i = idx / SW_CB, cc = idx - i * SW_CB;
+        const bool ok = i < I1 && c0 + cc < C;
+        cp_async8(&Xs[i * SWT_LDX + cc], ok ? xb + ((size_t)i * C + c0 + cc) * 8 : xb, ok ? 8u : 0u);
+      }
+    }
+    cp_async_commit();
   }
+  // moments of the entries this thread updates after the first product (SW_MAX_R * SW_CB / SW_THREADS = 4 at most)
+  constexpr int SW_EPT = SW_MAX_R * SW_CB / SW_THREADS;
+  cf pm[SW_EPT]; float pv[SW_EPT];
+#pragma unroll
+  for (int q = 0; q < SW_EPT; ++q) {
+    const int e = tid + q * SW_THREADS, j = e / SW_CB, cc = e - j * SW_CB;
+    pm[q] = make_float2(0.f, 0.f); pv[q] = 0.f;
+    if (j < r1 && c0 + cc < C) { const size_t idx = (size_t)j * C + c0 + cc; pm[q] = m_l[idx]; pv[q] = v_l[idx]; }
+  }
+  cp_async_wait<0>();
   __syncthreads();
   // ---- core[j][c] = sum_i conj(U1[i][j]) X[i][c]: rows (j, re|im), k = (i, re|im) ----
   for (int tile = warp; tile < (r1p / 8) * 2; tile += SW_THREADS / 32) {
@@ -401,13 +329,15 @@ __global__ void __launch_bounds__(SW_THREADS) core_sandwich_tc_kernel(const cf* 
   }
   __syncthreads();
   // ---- AdamUpdate of the block (rows past r1 are zero and stay zero) ----
-  for (int e = tid; e < r1 * SW_CB; e += SW_THREADS) {
-    const int j = e / SW_CB, cc = e - j * SW_CB;
+#pragma unroll
+  for (int q = 0; q < SW_EPT; ++q) {
+    const int e = tid + q * SW_THREADS, j = e / SW_CB, cc = e - j * SW_CB;
+    if (j >= r1) break;
     cf n = make_float2(0.f, 0.f);
     if (c0 + cc < C) {
       const size_t idx = (size_t)j * C + c0 + cc;
       const cf x = Cs[j * SWT_LDX + cc];
-      cf m = m_l[idx]; float v = v_l[idx];
+      cf m = pm[q]; float v = pv[q];
       n = adam_apply(x, m, v, a);
       m_l[idx] = m; v_l[idx] = v; n_l[idx] = n; core[idx] = x;
     }

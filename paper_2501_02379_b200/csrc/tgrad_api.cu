@@ -14,6 +14,7 @@
 #include "jacobi.cuh"
 #include "modeprod.cuh"
 #include "select.cuh"
+#include "subspace.cuh"
 #include "tail.cuh"
 #include "tail_tc.cuh"
 #include "tail_h.cuh"
@@ -32,11 +33,11 @@ constexpr size_t kSmemMax = 227 * 1024;   // dynamic shared memory a block may a
 
 struct Layout {
   // persistent block
-  size_t p_flags, p_omega, p_slab, p_factor[TGRAD_MAX_NDIM], p_ml, p_vl, p_ms, p_vs, p_u2tab, p_basis[TGRAD_MAX_NDIM], p_total;
+  size_t p_flags, p_omega, p_slab, p_factor[TGRAD_MAX_NDIM], p_ml, p_vl, p_ms, p_vs, p_u2tab, p_total;
   uint32_t nslab, E;          // slabs of the trailing two modes, entries per slab
   // workspace block
   size_t w_ns, w_gs, w_core, w_nl, w_bufa, w_bufb, w_sel, w_hist, w_blk, w_gram[TGRAD_MAX_NDIM], w_jac[TGRAD_MAX_NDIM],
-      w_v[TGRAD_MAX_NDIM], w_rot[TGRAD_MAX_NDIM], w_log[TGRAD_MAX_NDIM], w_lam[TGRAD_MAX_NDIM], w_partial, w_total;
+      w_v[TGRAD_MAX_NDIM], w_log[TGRAD_MAX_NDIM], w_lam[TGRAD_MAX_NDIM], w_partial, w_total;
   bool jac_fast[TGRAD_MAX_NDIM];    // eigensolver with the matrix in shared memory and a rotation log
   uint64_t numel, P, tsize;   // entries, core entries, entries of the tail-contracted tensor
   uint32_t nblk;              // compaction blocks
@@ -144,11 +145,6 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
   L.p_vs = o; o = align_up(o + k * 4);
   // operand-fragment table of the compression kernel: 32 lanes x 32 bytes per (8-row tile, 8-column tile) of U^(N-1)
   L.p_u2tab = o; o = align_up(o + (size_t)((c->dims[N - 2] + 7) / 8) * ((c->ranks[N - 2] + 7) / 8) * 1024);
-  // warm-started refresh: the eigenvector basis of each mode's last refresh (modes the rotation-log solver handles)
-  for (int n = 0; n < N; ++n) {
-    L.p_basis[n] = o;
-    if (c->warm_refresh && c->dims[n] <= JAC_FAST_MAX_N) o = align_up(o + (size_t)c->dims[n] * c->dims[n] * 8);
-  }
   L.p_total = o;
   o = 0;
   L.w_ns = o; o = align_up(o + k * 8);
@@ -166,8 +162,7 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
     size_t sq = (size_t)c->dims[n] * c->dims[n] * 8;
     L.w_gram[n] = o; o = align_up(o + sq);   // A_n, kept for inspection
     L.w_jac[n] = o; o = align_up(o + (size_t)c->dims[n] * (c->dims[n] | 1) * 8);    // working copy the solver diagonalises
-    L.w_v[n] = o; o = align_up(o + sq);      // accumulated rotations
-    L.w_rot[n] = o; if (c->warm_refresh) o = align_up(o + sq);   // A_n rotated into the previous basis
+    L.w_v[n] = o; o = align_up(o + sq);      // accumulated rotations; scratch of the subspace iteration
     const int sweeps = c->jacobi_max_sweeps > 0 ? c->jacobi_max_sweeps : 30;
     const size_t logb = jac_log_entries((int)c->dims[n], sweeps) * sizeof(float4);
     L.jac_fast[n] = c->dims[n] <= JAC_FAST_MAX_N && logb <= ((size_t)64 << 20);
@@ -193,7 +188,7 @@ struct tgrad_state {
   char* dw;
   int64_t t;
   bool have_subspace;
-  bool basis_valid;     // warm-started refresh: the persistent block holds the bases of a previous refresh
+  bool basis_valid;     // the persistent block holds factor matrices (of a refresh or an import) a refresh can start from
   bool tabs_stale;      // U^(N-1) changed since the compression kernel's fragment table was built
   int sm_count;
   TailPlan tail;
@@ -427,16 +422,6 @@ tgrad_status build_slab_ptr(tgrad_state* s, cudaStream_t st) {
 
 #define TG_TRY(x) do { tgrad_status _s = (x); if (_s != TGRAD_OK) return _s; } while (0)
 
-// out[m][c] = sum_k Aop[m][k] in[k][c] for the small square matrices of the warm-started refresh, in fp32 FMAs:
-// Aop = U (M x K, row-major) or, with conj_t, Aop = U^H for U of K x M.
-tgrad_status small_product(bool conj_t, const cf* in, cf* out, const cf* U, int M, int K, int C, cudaStream_t st) {
-  dim3 grid((unsigned)((C + 31) / 32), (unsigned)((M + MP_BM - 1) / MP_BM), 1);
-  if (conj_t) mode_product_kernel<true, 32><<<grid, MP_THREADS, 0, st>>>(in, out, U, M, K, C, M);
-  else mode_product_kernel<false, 32><<<grid, MP_THREADS, 0, st>>>(in, out, U, M, K, C, K);
-  TG_LAUNCH_CHECK();
-  return TGRAD_OK;
-}
-
 template <class S>
 tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   const tgrad_config& c = s->cfg;
@@ -473,7 +458,11 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   cf* partial = reinterpret_cast<cf*>(s->dw + L.w_partial);
   JacobiParams jp; memset(&jp, 0, sizeof(jp));
   JacobiFastParams fp; memset(&fp, 0, sizeof(fp));
+  SubspaceParams sp; memset(&sp, 0, sizeof(sp));
+  size_t sub_bytes = 0;
   int nslow = 0;
+  // no mode's factor is written yet (the eigensolvers below read these words)
+  if (cudaMemsetAsync(flags + SUB_DONE, 0, TGRAD_MAX_NDIM * sizeof(int), st) != cudaSuccess) return TGRAD_ERR_CUDA;
   for (int m = 0; m < N; ++m) {
     uint64_t O = 1, C = 1;
     for (int q = 0; q < m; ++q) O *= c.dims[q];
@@ -492,31 +481,26 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
 #undef TG_GRAM
     TG_LAUNCH_CHECK();
     gram_reduce_kernel<<<(In * In + GRR_E - 1) / GRR_E, GRR_E * GRR_G, 0, st>>>(partial, L.gram_splits[m], In, A); TG_LAUNCH_CHECK();
+    // leading eigenvectors by subspace iteration where the rank leaves room for guard columns ...
+    {
+      int R = 0; bool zsm = false;
+      if (sub_eligible(In, c.ranks[m], R, zsm)) {
+        SubspaceMode& sm_ = sp.mode[sp.nmodes++];
+        sm_.A = A; sm_.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
+        sm_.Zg = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
+        sm_.n = In; sm_.r = c.ranks[m]; sm_.R = R; sm_.index = m; sm_.z_in_smem = zsm ? 1 : 0;
+        const size_t b = sub_smem(In, R, zsm);
+        if (b > sub_bytes) sub_bytes = b;
+      }
+    }
+    // ... and the full Jacobi diagonalisation for every mode (it returns at once where the iteration has delivered)
     if (L.jac_fast[m]) {
       JacobiFastMode& fm = fp.mode[fp.nmodes++];
-      fm.A = A; fm.A0 = A;
+      fm.A = A;
       fm.work = reinterpret_cast<cf*>(s->dw + L.w_jac[m]);
       fm.log = reinterpret_cast<float4*>(s->dw + L.w_log[m]);
       fm.lam = reinterpret_cast<float*>(s->dw + L.w_lam[m]);
       fm.V = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
-      if (c.warm_refresh) {
-        cf* V = reinterpret_cast<cf*>(s->dp + L.p_basis[m]);
-        fm.V = V;                                       // the solver leaves this refresh's eigenvectors there
-        if (s->basis_valid) {
-          // V <- V (3/2 I - 1/2 V^H V), then A' = V^H A V is what gets diagonalised; its rotations are applied to V
-          cf* t1 = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
-          cf* t2 = reinterpret_cast<cf*>(s->dw + L.w_rot[m]);
-          TG_TRY(small_product(true, V, t1, V, In, In, In, st));          // G = V^H V
-          int* bad = flags + JAC_BAD_BASIS + m;
-          if (cudaMemsetAsync(bad, 0, sizeof(int), st) != cudaSuccess) return TGRAD_ERR_CUDA;
-          ns_residual_kernel<<<(In * In + 255) / 256, 256, 0, st>>>(t1, In, bad); TG_LAUNCH_CHECK();
-          TG_TRY(small_product(false, t1, t2, V, In, In, In, st));        // V E
-          if (cudaMemcpyAsync(V, t2, (size_t)In * In * 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return TGRAD_ERR_CUDA;
-          TG_TRY(small_product(false, V, t1, A, In, In, In, st));         // A V
-          TG_TRY(small_product(true, t1, t2, V, In, In, In, st));         // V^H (A V)
-          fm.A = t2;
-        }
-      }
       fm.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
       fm.n = In; fm.r = c.ranks[m]; fm.index = m; fm.row0 = fp.total_rows;
       fp.total_rows += In;
@@ -535,13 +519,17 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   if (k > 0) { scatter_restore_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, g_s, k); TG_LAUNCH_CHECK(); }
   const int max_sweeps = c.jacobi_max_sweeps > 0 ? c.jacobi_max_sweeps : 30;
   const float tol = c.jacobi_tol > 0.f ? c.jacobi_tol : 1e-6f;
+  if (sp.nmodes) {
+    sp.warm = (c.warm_refresh && s->basis_valid) ? 1 : 0;
+    sp.max_sweeps = max_sweeps; sp.tol = tol; sp.flags = flags;
+    subspace_kernel<<<sp.nmodes, SUB_THREADS, sub_bytes, st>>>(sp); TG_LAUNCH_CHECK();
+  }
   if (nslow) {
     jp.max_sweeps = max_sweeps; jp.tol = tol; jp.flags = flags;
     jacobi_kernel<<<nslow, JAC_THREADS, 0, st>>>(jp); TG_LAUNCH_CHECK();
   }
   if (fp.nmodes) {
     fp.max_sweeps = max_sweeps; fp.tol = tol; fp.flags = flags;
-    fp.warm = (c.warm_refresh && s->basis_valid) ? 1 : 0;
     // the sweeps: modes whose matrix fits in shared memory in one launch, the larger ones (matrix in L2) in another
     JacobiFastParams fs = fp, fg = fp;
     fs.nmodes = fg.nmodes = 0;
@@ -562,7 +550,7 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   }
   s->have_subspace = true;
   s->tabs_stale = true;
-  if (c.warm_refresh) s->basis_valid = true;
+  s->basis_valid = true;
   return TGRAD_OK;
 }
 
@@ -796,6 +784,9 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
   if (cfg->dims[0] <= SW_MAX_I && cfg->ranks[0] <= SW_MAX_R &&
       cudaFuncSetAttribute(core_sandwich_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)sandwich_tc_smem(SW_MAX_I, SW_MAX_R)) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
+  if (cudaFuncSetAttribute(subspace_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax) != cudaSuccess) {
+    delete st; return TGRAD_ERR_CUDA;
+  }
   if (cudaFuncSetAttribute(jacobi_sweeps_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)jac_sweeps_smem(JAC_SMEM_MAX_N)) != cudaSuccess) { delete st; return TGRAD_ERR_CUDA; }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -917,7 +908,7 @@ tgrad_status tgrad_import_state(tgrad_state* st, int32_t what, const void* host_
     if (cudaStreamSynchronize(stream) != cudaSuccess) return TGRAD_ERR_CUDA;
   }
   if (what == TGRAD_WHAT_OMEGA || what >= TGRAD_WHAT_FACTOR_BASE) st->have_subspace = true;
-  if (what >= TGRAD_WHAT_FACTOR_BASE) st->tabs_stale = true;
+  if (what >= TGRAD_WHAT_FACTOR_BASE) { st->tabs_stale = true; st->basis_valid = true; }
   return TGRAD_OK;
 }
 
