@@ -148,6 +148,31 @@ def tucker_factors(r: np.ndarray, ranks: Sequence[int]) -> List[np.ndarray]:
     return out
 
 
+def tucker_factors_hooi(r: np.ndarray, ranks: Sequence[int], n_iter: int,
+                        init: Optional[Sequence[np.ndarray]] = None) -> List[np.ndarray]:
+    """TuckerFactors(R, r) with the refinement the paper's implementation applies (Appendix "Tensor Decomposition /
+    Implementation": factors from truncated SVDs of the mode-n unfoldings, then refined iteratively to reduce the
+    Frobenius reconstruction error, optionally restarted from previous factors).
+
+    Higher-order orthogonal iteration: starting from `init` (the truncated-SVD factors of tucker_factors when None),
+    each of the n_iter sweeps visits the modes in order and replaces U^(n) by the r_n leading left singular vectors
+    of the mode-n unfolding of  Y = R x_{m != n} U^(m)H  (every other mode compressed with its current factor, the
+    factors already updated in this sweep included), obtained as eigenvectors of Y_(n) Y_(n)^H, descending,
+    phase-canonicalised, stored as complex64.  n_iter = 0 returns the starting factors.
+    """
+    us = [np.asarray(u, dtype=np.complex64) for u in (init if init is not None else tucker_factors(r, ranks))]
+    x = np.asarray(r, dtype=np.complex128)
+    for _ in range(int(n_iter)):
+        for n, rn in enumerate(ranks):
+            y = x
+            for m, u in enumerate(us):
+                if m != n:
+                    y = mode_n_product(y, np.conj(u.astype(np.complex128)).T, m)
+            w, v = np.linalg.eigh(mode_gram(y, n))
+            us[n] = np.ascontiguousarray(canonical_phase(v[:, ::-1][:, :rn]).astype(np.complex64))
+    return us
+
+
 # --------------------------------------------------------------------------
 # Adam in the compressed space (AdamUpdate of Algorithm 1; UPDATE block of Algorithm 3)
 # --------------------------------------------------------------------------
@@ -200,6 +225,8 @@ class OracleConfig:
     eps: float = 1e-8
     weight_decay: float = 0.0
     half_storage: bool = False      # W and G live as fp16 (re, im) pairs
+    hooi_iters: int = 0             # refinement sweeps of TuckerFactors (0: truncated-SVD factors only)
+    hooi_warm: bool = False         # refinement starts from the factors of the previous refresh when there are any
 
 
 def _store_w(w: np.ndarray, half: bool) -> np.ndarray:
@@ -236,7 +263,12 @@ def oracle_refresh(st: OracleState, grad: np.ndarray) -> None:
     left untouched (nothing in the loop resets them)."""
     cfg = st.cfg
     st.omega = sparse_indices_topk(grad, cfg.k)
-    st.factors = tucker_factors(residual(grad, st.omega), cfg.ranks)
+    res = residual(grad, st.omega)
+    if cfg.hooi_iters > 0:
+        init = st.factors if (cfg.hooi_warm and st.factors is not None) else None
+        st.factors = tucker_factors_hooi(res, cfg.ranks, cfg.hooi_iters, init)
+    else:
+        st.factors = tucker_factors(res, cfg.ranks)
 
 
 def weight_update(cfg: OracleConfig, w: np.ndarray, n_l: np.ndarray, n_s: np.ndarray, omega: np.ndarray,

@@ -124,6 +124,10 @@ WORKLOADS: Dict[str, Workload] = {
                  outlier_frac=(1, 100), outlier_scale=20.0, noise="laplace", noise_scale=0.1),
         Workload("cfg5", 5, (256, 256, 128, 65), (64, 64, 32, 16), (1, 100), 200, 100,
                  outlier_frac=(5, 1000), outlier_scale=30.0, noise_scale=0.02, half_storage=True),
+        # the same slabs, ranks and storage with smaller leading extents (0.3 GB per tensor): the case the
+        # profiler captures of the largest configuration's kernels are taken on
+        Workload("cfg5p", 5, (96, 96, 128, 65), (64, 64, 32, 16), (1, 100), 200, 100,
+                 outlier_frac=(5, 1000), outlier_scale=30.0, noise_scale=0.02, half_storage=True),
     ]
 }
 

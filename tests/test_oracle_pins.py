@@ -209,6 +209,81 @@ def test_gram_identities_and_eigen_residual():
             assert abs(u[i, j].imag) < 1e-6 and u[i, j].real > 0
 
 
+# ---- refinement of the factors (higher-order orthogonal iteration) --------------------------------
+
+def _recon_error(x, us):
+    return float(np.linalg.norm(x - orc.tucker_reconstruct(orc.tucker_compress(x, us), us)))
+
+
+def test_hooi_never_increases_the_reconstruction_error():
+    # each mode update maximises the energy kept given the other factors, so || R - P_U R ||_F cannot grow from sweep
+    # to sweep, and it starts from the truncated-SVD factors' error
+    rng = np.random.default_rng(31)
+    shape, ranks = (7, 6, 5, 4), (3, 2, 2, 2)
+    x = (rng.standard_normal(shape) + 1j * rng.standard_normal(shape)).astype(np.complex64)      # no low-rank structure
+    errs = [_recon_error(x, orc.tucker_factors_hooi(x, ranks, it)) for it in range(5)]
+    assert errs[0] == pytest.approx(_recon_error(x, orc.tucker_factors(x, ranks)), rel=1e-12)
+    for a, b in zip(errs, errs[1:]):
+        assert b <= a * (1 + 1e-6)
+    assert errs[-1] < errs[0] * 0.999          # and on an unstructured tensor the refinement does help
+    for u in orc.tucker_factors_hooi(x, ranks, 3):
+        assert H.ortho_defect(u) < 1e-6
+        for j in range(u.shape[1]):
+            i = np.argmax(np.abs(u[:, j]))
+            assert abs(u[i, j].imag) < 1e-6 and u[i, j].real > 0
+
+
+def test_hooi_fixed_point_on_an_exactly_low_rank_tensor():
+    rng = np.random.default_rng(32)
+    shape, ranks = (8, 7, 6), (3, 2, 2)
+    us = [H.random_orthonormal(rng, i, r) for i, r in zip(shape, ranks)]
+    c = rng.standard_normal(ranks) + 1j * rng.standard_normal(ranks)
+    x = orc.tucker_reconstruct(c, us)
+    f0 = orc.tucker_factors(x, ranks)
+    f2 = orc.tucker_factors_hooi(x, ranks, 2)
+    for a, b, planted in zip(f0, f2, us):
+        assert H.max_sin_angle(b, planted) < 1e-6 and H.max_sin_angle(a, b) < 1e-6
+    assert _recon_error(x, f2) < 1e-6 * np.linalg.norm(x)
+
+
+def test_hooi_on_a_matrix_stays_at_the_svd():
+    rng = np.random.default_rng(33)
+    x = rng.standard_normal((9, 7)) + 1j * rng.standard_normal((9, 7))
+    u, s_, vh = np.linalg.svd(x)
+    f = orc.tucker_factors_hooi(x, (3, 3), 3)
+    assert H.max_sin_angle(f[0], u[:, :3]) < 1e-6
+    assert H.max_sin_angle(f[1], np.conj(vh[:3]).T.conj()) < 1e-6
+
+
+def test_hooi_update_is_the_best_subspace_for_the_other_factors():
+    # the defining property of one mode update: with the other factors fixed, no other orthonormal I_n x r_n matrix
+    # keeps more energy || R x_1 U1^H .. x_N UN^H ||_F
+    rng = np.random.default_rng(34)
+    shape, ranks = (6, 5, 4), (2, 2, 2)
+    x = (rng.standard_normal(shape) + 1j * rng.standard_normal(shape)).astype(np.complex64)
+    us = orc.tucker_factors_hooi(x, ranks, 4)
+    kept = np.linalg.norm(orc.tucker_compress(x, us))
+    for n in range(3):
+        for trial in range(20):
+            alt = list(us)
+            alt[n] = H.random_orthonormal(rng, shape[n], ranks[n])
+            assert np.linalg.norm(orc.tucker_compress(x, alt)) <= kept * (1 + 1e-3)
+
+
+def test_hooi_warm_start_takes_the_previous_factors():
+    wl = synth.WORKLOADS["small4"]
+    src = synth.GradientSource(wl)
+    cfg = orc.OracleConfig(shape=wl.shape, ranks=wl.ranks, k=wl.k, T=2, hooi_iters=1, hooi_warm=True)
+    st = orc.OracleState(cfg)
+    orc.oracle_refresh(st, src.gradient(0))
+    prev = [u.copy() for u in st.factors]
+    g1 = src.gradient(1)
+    orc.oracle_refresh(st, g1)
+    want = orc.tucker_factors_hooi(orc.residual(g1, st.omega), wl.ranks, 1, prev)
+    for a, b in zip(st.factors, want):
+        assert np.array_equal(a, b)
+
+
 # ---- Adam closed forms ----------------------------------------------------------------------------
 
 def test_adam_first_step_is_unit_direction():
