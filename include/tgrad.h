@@ -99,6 +99,15 @@ typedef struct {
                                        is the same eigen-decomposition to the same tolerance.  Stored factors
                                        that are unusable (never set, not finite) are noticed on the device and
                                        that refresh starts cold.  0: every refresh starts cold               */
+  int32_t hooi_iters;               /* refinement sweeps of TuckerFactors after the truncated-SVD factors (higher-
+                                       order orthogonal iteration, the paper's appendix "Tensor Decomposition /
+                                       Implementation"): per sweep and mode, the residual is compressed in every
+                                       other mode with the current factors and U^(n) becomes the leading left
+                                       singular vectors of the result.  0: none.  With warm_refresh = 1 and
+                                       factors in the state, the sweeps start from those factors and the
+                                       truncated-SVD stage is skipped (the warm restart of the decomposition).
+                                       Needs extra workspace, and each trailing slab must still fit in shared
+                                       memory with one of its two factors replaced by the identity            */
 } tgrad_config;
 
 /* Selectors for tgrad_export_state / tgrad_import_state.  FACTOR_BASE + n is
@@ -112,7 +121,9 @@ enum {
   TGRAD_WHAT_CORE = 6,         /* last step's compressed gradient (export only; workspace) */
   TGRAD_WHAT_N_L = 7,          /* last step's normalised core update (export only)         */
   TGRAD_WHAT_N_S = 8,          /* last step's normalised sparse update (export only)       */
-  TGRAD_WHAT_GRAM_BASE = 32,   /* + n: A_n = R_(n) R_(n)^H of the last refresh, I_n x I_n complex64 (export only) */
+  TGRAD_WHAT_GRAM_BASE = 32,   /* + n: the Gram matrix the last refresh took U^(n+1) from, I_n x I_n complex64 (export
+                                  only): A_n = R_(n) R_(n)^H, or with refinement sweeps that of the residual
+                                  compressed in every other mode */
   TGRAD_WHAT_FACTOR_BASE = 64  /* + n */
 };
 

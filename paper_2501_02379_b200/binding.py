@@ -42,6 +42,7 @@ class TgradConfig(C.Structure):
         ("jacobi_max_sweeps", C.c_int32),
         ("jacobi_tol", C.c_float),
         ("warm_refresh", C.c_int32),
+        ("hooi_iters", C.c_int32),
     ]
 
 
@@ -112,7 +113,8 @@ def _check(s: int, where: str) -> None:
 def make_config(shape: Sequence[int], ranks: Sequence[int], k: int, T: int, lr: float = 1e-3, alpha: float = 1.0,
                 lam: float = 1.0, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
                 weight_decay: float = 0.0, half_storage: bool = False, auto_refresh: bool = True,
-                jacobi_max_sweeps: int = 0, jacobi_tol: float = 0.0, warm_refresh: bool = False) -> TgradConfig:
+                jacobi_max_sweeps: int = 0, jacobi_tol: float = 0.0, warm_refresh: bool = False,
+                hooi_iters: int = 0) -> TgradConfig:
     if len(shape) > MAX_NDIM or len(shape) != len(ranks):
         raise ValueError("bad shape / ranks")
     cfg = TgradConfig()
@@ -130,6 +132,7 @@ def make_config(shape: Sequence[int], ranks: Sequence[int], k: int, T: int, lr: 
     cfg.jacobi_max_sweeps = jacobi_max_sweeps
     cfg.jacobi_tol = jacobi_tol
     cfg.warm_refresh = 1 if warm_refresh else 0
+    cfg.hooi_iters = int(hooi_iters)
     return cfg
 
 

@@ -37,7 +37,8 @@ struct Layout {
   uint32_t nslab, E;          // slabs of the trailing two modes, entries per slab
   // workspace block
   size_t w_ns, w_gs, w_core, w_nl, w_bufa, w_bufb, w_sel, w_hist, w_blk, w_gram[TGRAD_MAX_NDIM], w_jac[TGRAD_MAX_NDIM],
-      w_v[TGRAD_MAX_NDIM], w_log[TGRAD_MAX_NDIM], w_lam[TGRAD_MAX_NDIM], w_partial, w_total;
+      w_v[TGRAD_MAX_NDIM], w_log[TGRAD_MAX_NDIM], w_lam[TGRAD_MAX_NDIM], w_partial, w_hooi0, w_hooi1, w_ident, w_total;
+  uint32_t hooi_smem;         // shared memory of the compression kernel when one trailing factor is replaced by the identity
   bool jac_fast[TGRAD_MAX_NDIM];    // eigensolver with the matrix in shared memory and a rotation log
   uint64_t numel, P, tsize;   // entries, core entries, entries of the tail-contracted tensor
   uint32_t nblk;              // compaction blocks
@@ -48,6 +49,7 @@ struct Layout {
 struct TailPlan {
   // general path: one block per slab
   TailBlkGeom bproj, bback;
+  uint32_t hooi_smem;      // shared memory of the compression kernel in a refinement sweep (0: no refinement)
   int grid_bproj, grid_bback;
   // tensor-core fast path (complex64 storage, 16/32/64 slab rows, small trailing ranks)
   bool tc;
@@ -77,6 +79,7 @@ tgrad_status validate(const tgrad_config* c) {
     return TGRAD_ERR_INVALID_ARG;
   if (c->jacobi_max_sweeps < 0 || c->jacobi_tol < 0.f) return TGRAD_ERR_INVALID_ARG;
   if (c->warm_refresh != 0 && c->warm_refresh != 1) return TGRAD_ERR_INVALID_ARG;
+  if (c->hooi_iters < 0 || c->hooi_iters > 64) return TGRAD_ERR_INVALID_ARG;
   // limits of this implementation
   if (tot >= 4294967296.0L) return TGRAD_ERR_UNSUPPORTED;    // flat indices are uint32
   if (c->k >= ((int64_t)1 << 31)) return TGRAD_ERR_UNSUPPORTED;   // slots of Omega are addressed with int
@@ -87,19 +90,26 @@ tgrad_status validate(const tgrad_config* c) {
 }
 
 
-void plan_gram(const tgrad_config* c, int n, int sm, uint32_t& chunks, uint32_t& cps, int& splits) {
-  uint64_t O = 1, C = 1;
-  for (int m = 0; m < n; ++m) O *= c->dims[m];
-  for (int m = n + 1; m < c->ndim; ++m) C *= c->dims[m];
+// Split-K plan of one Gram accumulation: In x In output, contraction over O * C entries per row.
+void plan_gram_dims(int In, uint64_t O, uint64_t C, int sm, uint32_t& chunks, uint32_t& cps, int& splits) {
   uint64_t total = (O * C + GR_KT - 1) / GR_KT;      // the contraction index (o, c) is flattened
-  int T = (int)((c->dims[n] + GR_T - 1) / GR_T);
+  int T = (In + GR_T - 1) / GR_T;
   int tiles = T * (T + 1) / 2;
   uint64_t want = (uint64_t)(6 * sm + tiles - 1) / tiles;
   if (want < 1) want = 1;
   if (want > 1024) want = 1024;
   if (want > total) want = total;
+  if (want < 1) want = 1;
   uint64_t per = (total + want - 1) / want;
+  if (per < 1) per = 1;
   chunks = (uint32_t)total; cps = (uint32_t)per; splits = (int)((total + per - 1) / per);
+  if (splits < 1) splits = 1;
+}
+void plan_gram(const tgrad_config* c, int n, int sm, uint32_t& chunks, uint32_t& cps, int& splits) {
+  uint64_t O = 1, C = 1;
+  for (int m = 0; m < n; ++m) O *= c->dims[m];
+  for (int m = n + 1; m < c->ndim; ++m) C *= c->dims[m];
+  plan_gram_dims((int)c->dims[n], O, C, sm, chunks, cps, splits);
 }
 
 // The configuration the kernels see.  A matrix (N = 2, where the Tucker decomposition is the matrix SVD) is handled as
@@ -173,6 +183,22 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
     if (pb > partial) partial = pb;
   }
   L.w_partial = o; o = align_up(o + partial);
+  // refinement sweeps: two buffers for the tensor compressed in all modes but one, and an identity matrix that
+  // stands in for the factor of the mode that is left alone when that is one of the two trailing modes
+  L.w_hooi0 = L.w_hooi1 = L.w_ident = o; L.hooi_smem = 0;
+  if (c->hooi_iters > 0) {
+    const uint64_t A = (uint64_t)c->dims[N - 2], B = (uint64_t)c->dims[N - 1], ra = c->ranks[N - 2], rb = c->ranks[N - 1];
+    uint64_t per = ra * rb;
+    if (A * rb > per) per = A * rb;
+    if (ra * B > per) per = ra * B;
+    const size_t g1 = tail_blk_geom((int)A, (int)B, (int)A, (int)rb, false).total, g2 = tail_blk_geom((int)A, (int)B, (int)ra, (int)B, false).total;
+    L.hooi_smem = (uint32_t)(g1 > g2 ? g1 : g2);
+    if (L.hooi_smem > kSmemMax) return TGRAD_ERR_UNSUPPORTED;
+    L.w_hooi0 = o; o = align_up(o + (size_t)(S * per) * 8);
+    L.w_hooi1 = o; o = align_up(o + (size_t)(S * per) * 8);
+    const uint64_t mx = A > B ? A : B;
+    L.w_ident = o; o = align_up(o + (size_t)(mx * mx) * 8);
+  }
   L.w_total = o;
   return TGRAD_OK;
 }
@@ -223,7 +249,7 @@ template <class S>
 tgrad_status tail_dispatch(int op, const TailPlan& tp, void* ptr, const TailParams& p, cudaStream_t st) {
   if (op == 0) {
     if (cudaFuncSetAttribute(proj_tail_blk_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)tp.bproj.total) != cudaSuccess) return TGRAD_ERR_CUDA;
+                             (int)(tp.bproj.total > tp.hooi_smem ? tp.bproj.total : tp.hooi_smem)) != cudaSuccess) return TGRAD_ERR_CUDA;
     if (cudaFuncSetAttribute(back_tail_blk_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)tp.bback.total) != cudaSuccess) return TGRAD_ERR_CUDA;
     return TGRAD_OK;
@@ -349,6 +375,7 @@ tgrad_status plan_tail(tgrad_state* s) {
   const size_t kMax = 227 * 1024;
   tp.bproj = tail_blk_geom(A, B, ra, rb, false);
   tp.bback = tail_blk_geom(A, B, ra, rb, true);
+  tp.hooi_smem = s->L.hooi_smem;
   if (tp.bproj.total > kMax || tp.bback.total > kMax) return TGRAD_ERR_UNSUPPORTED;   // a trailing A x B slab does not fit in shared memory
   uint64_t S = s->L.numel / ((uint64_t)A * B);
   {
@@ -422,6 +449,174 @@ tgrad_status build_slab_ptr(tgrad_state* s, cudaStream_t st) {
 
 #define TG_TRY(x) do { tgrad_status _s = (x); if (_s != TGRAD_OK) return _s; } while (0)
 
+tgrad_status mode_product(bool conj_t, const cf* in, cf* out, const cf* U, uint64_t O, int M, int K, uint64_t C,
+                          int r_n, int sm_count, cudaStream_t st);
+
+// A = X_(n) X_(n)^H for a tensor seen as [O][In][C] (storage S), split-K partial sums reduced in a fixed order.
+template <class S>
+tgrad_status launch_gram(tgrad_state* s, const void* x, int In, uint64_t O, uint64_t C, uint32_t chunks, uint32_t cps,
+                         int splits, cf* A, cudaStream_t st) {
+  cf* partial = reinterpret_cast<cf*>(s->dw + s->L.w_partial);
+  const int T = (In + GR_T - 1) / GR_T;
+  dim3 grid(T * T, splits);
+  // long contractions average the TF32 input rounding away; short ones get the split-precision products
+  const bool full = (In % GR_T) == 0;
+#define TG_GRAM(SPLIT_, FULL_)                                                                                   \
+  gram_partial_kernel<S, SPLIT_, FULL_><<<grid, GR_THREADS, GR_SMEM, st>>>(x, In, (uint32_t)O, (uint32_t)C, chunks, \
+                                                                          cps, partial)
+  if (O * C >= 16384) { if (full) TG_GRAM(false, true); else TG_GRAM(false, false); }
+  else { if (full) TG_GRAM(true, true); else TG_GRAM(true, false); }
+#undef TG_GRAM
+  TG_LAUNCH_CHECK();
+  gram_reduce_kernel<<<(In * In + GRR_E - 1) / GRR_E, GRR_E * GRR_G, 0, st>>>(partial, splits, In, A); TG_LAUNCH_CHECK();
+  return TGRAD_OK;
+}
+
+// U^(m) <- eigenvectors of the r_m largest eigenvalues of the Gram matrix stored for mode m, for the listed modes:
+// subspace iteration where the rank leaves room for guard columns (started from the stored factor if `warm`), then
+// the full Jacobi diagonalisation, which returns at once for the modes the iteration has delivered.
+tgrad_status solve_modes(tgrad_state* s, const int* modes, int nm, bool warm, cudaStream_t st) {
+  const tgrad_config& c = s->cfg;
+  const Layout& L = s->L;
+  int* flags = reinterpret_cast<int*>(s->dp + L.p_flags);
+  JacobiParams jp; memset(&jp, 0, sizeof(jp));
+  JacobiFastParams fp; memset(&fp, 0, sizeof(fp));
+  SubspaceParams sp; memset(&sp, 0, sizeof(sp));
+  size_t sub_bytes = 0;
+  int nslow = 0;
+  // no mode's factor is written yet (the eigensolvers below read these words)
+  if (cudaMemsetAsync(flags + SUB_DONE, 0, TGRAD_MAX_NDIM * sizeof(int), st) != cudaSuccess) return TGRAD_ERR_CUDA;
+  for (int i = 0; i < nm; ++i) {
+    const int m = modes[i];
+    const int In = (int)c.dims[m];
+    cf* A = reinterpret_cast<cf*>(s->dw + L.w_gram[m]);
+    {
+      int R = 0; bool zsm = false;
+      if (sub_eligible(In, c.ranks[m], R, zsm)) {
+        SubspaceMode& sm_ = sp.mode[sp.nmodes++];
+        sm_.A = A; sm_.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
+        sm_.Zg = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
+        sm_.n = In; sm_.r = c.ranks[m]; sm_.R = R; sm_.index = m; sm_.z_in_smem = zsm ? 1 : 0;
+        const size_t b = sub_smem(In, R, zsm);
+        if (b > sub_bytes) sub_bytes = b;
+      }
+    }
+    if (L.jac_fast[m]) {
+      JacobiFastMode& fm = fp.mode[fp.nmodes++];
+      fm.A = A;
+      fm.work = reinterpret_cast<cf*>(s->dw + L.w_jac[m]);
+      fm.log = reinterpret_cast<float4*>(s->dw + L.w_log[m]);
+      fm.lam = reinterpret_cast<float*>(s->dw + L.w_lam[m]);
+      fm.V = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
+      fm.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
+      fm.n = In; fm.r = c.ranks[m]; fm.index = m; fm.row0 = fp.total_rows;
+      fp.total_rows += In;
+      if (In > fp.row_stride) fp.row_stride = In;
+    } else {
+      JacobiMode& jm = jp.mode[nslow];
+      jp.index[nslow++] = m;
+      jm.A = reinterpret_cast<cf*>(s->dw + L.w_jac[m]);
+      jm.V = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
+      jm.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
+      jm.n = In; jm.r = c.ranks[m];
+      if (cudaMemcpyAsync(s->dw + L.w_jac[m], A, (size_t)In * In * 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return TGRAD_ERR_CUDA;
+    }
+  }
+  const int max_sweeps = c.jacobi_max_sweeps > 0 ? c.jacobi_max_sweeps : 30;
+  const float tol = c.jacobi_tol > 0.f ? c.jacobi_tol : 1e-6f;
+  if (sp.nmodes) {
+    sp.warm = warm ? 1 : 0;
+    sp.max_sweeps = max_sweeps; sp.tol = tol; sp.flags = flags;
+    subspace_kernel<<<sp.nmodes, SUB_THREADS, sub_bytes, st>>>(sp); TG_LAUNCH_CHECK();
+  }
+  if (nslow) {
+    jp.max_sweeps = max_sweeps; jp.tol = tol; jp.flags = flags;
+    jacobi_kernel<<<nslow, JAC_THREADS, 0, st>>>(jp); TG_LAUNCH_CHECK();
+  }
+  if (fp.nmodes) {
+    fp.max_sweeps = max_sweeps; fp.tol = tol; fp.flags = flags;
+    // the sweeps: modes whose matrix fits in shared memory in one launch, the larger ones (matrix in L2) in another
+    JacobiFastParams fs = fp, fg = fp;
+    fs.nmodes = fg.nmodes = 0;
+    size_t smem_s = 0, smem_g = 0;
+    for (int i = 0; i < fp.nmodes; ++i) {
+      const int n = fp.mode[i].n;
+      if (n <= JAC_SMEM_MAX_N) { fs.mode[fs.nmodes++] = fp.mode[i]; const size_t b = jac_sweeps_smem(n, true); if (b > smem_s) smem_s = b; }
+      else { fg.mode[fg.nmodes++] = fp.mode[i]; const size_t b = jac_sweeps_smem(n, false); if (b > smem_g) smem_g = b; }
+    }
+    if (fg.nmodes) { jacobi_sweeps_kernel<false><<<fg.nmodes, JAC_THREADS, smem_g, st>>>(fg); TG_LAUNCH_CHECK(); }
+    if (fs.nmodes) { jacobi_sweeps_kernel<true><<<fs.nmodes, JAC_THREADS, smem_s, st>>>(fs); TG_LAUNCH_CHECK(); }
+    fp.row_stride = (fp.row_stride + 1) & ~1;
+    const size_t vsm = (size_t)8 * fp.row_stride * sizeof(cf);
+    if (fp.row_stride <= 192) jacobi_vectors_kernel<3, 4><<<(fp.total_rows + 7) / 8, 256, vsm, st>>>(fp);
+    else jacobi_vectors_kernel<4, 2><<<(fp.total_rows + 7) / 8, 256, vsm, st>>>(fp);
+    TG_LAUNCH_CHECK();
+    jacobi_factors_kernel<<<fp.nmodes, JAC_THREADS, 0, st>>>(fp); TG_LAUNCH_CHECK();
+  }
+  return TGRAD_OK;
+}
+
+__global__ void identity_kernel(cf* __restrict__ m, int n) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < n * n) m[idx] = make_float2((idx / n) == (idx % n) ? 1.f : 0.f, 0.f);
+}
+
+// One mode update of the refinement: Y = R x_{q != m} U^(q)H through the general streaming kernel (the two trailing
+// modes, the identity standing in for U^(m) if m is one of them) and the chain of mode products (mode m left out),
+// then A = Y_(m) Y_(m)^H and its leading eigenvectors, started from the current U^(m).  `d_grad` holds the residual
+// (the entries at Omega are zero during a refresh).
+template <class S>
+tgrad_status hooi_mode_update(tgrad_state* s, int m, const void* d_grad, cudaStream_t st) {
+  const tgrad_config& c = s->cfg;
+  const Layout& L = s->L;
+  const int N = c.ndim;
+  const int A = (int)c.dims[N - 2], B = (int)c.dims[N - 1];
+  cf* ident = reinterpret_cast<cf*>(s->dw + L.w_ident);
+  int ra = c.ranks[N - 2], rb = c.ranks[N - 1];
+  const cf* Ua = reinterpret_cast<const cf*>(s->dp + L.p_factor[N - 2]);
+  const cf* Ub = reinterpret_cast<const cf*>(s->dp + L.p_factor[N - 1]);
+  if (m == N - 2) { identity_kernel<<<(A * A + 255) / 256, 256, 0, st>>>(ident, A); TG_LAUNCH_CHECK(); Ua = ident; ra = A; }
+  if (m == N - 1) { identity_kernel<<<(B * B + 255) / 256, 256, 0, st>>>(ident, B); TG_LAUNCH_CHECK(); Ub = ident; rb = B; }
+  TailParams p; memset(&p, 0, sizeof(p));
+  p.A = A; p.B = B; p.Bs = B | 1; p.ra = ra; p.rb = rb; p.ras = ra | 1;
+  p.E = (uint32_t)((uint64_t)A * B); p.nslab = (uint32_t)(L.numel / p.E);
+  p.Ua = Ua; p.Ub = Ub; p.k = 0;
+  cf* cur = reinterpret_cast<cf*>(s->dw + L.w_hooi0);
+  cf* nxt = reinterpret_cast<cf*>(s->dw + L.w_hooi1);
+  p.t = cur;
+  const TailBlkGeom G = tail_blk_geom(A, B, ra, rb, false);
+  {
+    const int per_sm = (int)(kSmemMax / (G.total + 1024));
+    const uint64_t cap = (uint64_t)s->sm_count * (per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm));
+    const unsigned grid = (unsigned)(p.nslab < cap ? p.nslab : cap);
+    proj_tail_blk_kernel<S><<<grid, TB_THREADS, G.total, st>>>(d_grad, p, G); TG_LAUNCH_CHECK();
+  }
+  // leading modes N-3 .. 0, mode m left as it is; the tensor is [d_0 .. d_{N-3}][ra][rb] with d_q shrinking to r_q
+  uint64_t C = (uint64_t)ra * rb;
+  for (int q = N - 3; q >= 0; --q) {
+    if (q == m) { C *= (uint64_t)c.dims[q]; continue; }
+    uint64_t O = 1;
+    for (int z = 0; z < q; ++z) O *= c.dims[z];
+    TG_TRY(mode_product(true, cur, nxt, reinterpret_cast<const cf*>(s->dp + L.p_factor[q]), O, c.ranks[q], (int)c.dims[q],
+                        C, c.ranks[q], s->sm_count, st));
+    C *= (uint64_t)c.ranks[q];
+    cf* tmp = cur; cur = nxt; nxt = tmp;
+  }
+  // Gram matrix over mode m of Y, whose extents are r_q for q != m
+  uint64_t Oy = 1, Cy = 1;
+  for (int q = 0; q < m; ++q) Oy *= (uint64_t)c.ranks[q];
+  for (int q = m + 1; q < N; ++q) Cy *= (uint64_t)c.ranks[q];
+  uint32_t chunks, cps; int splits;
+  plan_gram_dims((int)c.dims[m], Oy, Cy, 148, chunks, cps, splits);
+  if (splits > L.gram_splits[m]) {          // the scratch of the partial sums was sized for the full tensor's plan
+    const uint64_t per = (chunks + (uint64_t)L.gram_splits[m] - 1) / (uint64_t)L.gram_splits[m];
+    cps = (uint32_t)per; splits = (int)((chunks + per - 1) / per);
+  }
+  TG_TRY(launch_gram<StoreC64>(s, cur, (int)c.dims[m], Oy, Cy, chunks, cps, splits, reinterpret_cast<cf*>(s->dw + L.w_gram[m]), st));
+  return solve_modes(s, &m, 1, true, st);
+}
+
 template <class S>
 tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   const tgrad_config& c = s->cfg;
@@ -455,99 +650,28 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
     tgrad_status r = build_slab_ptr(s, st);
     if (r != TGRAD_OK) return r;
   }
-  cf* partial = reinterpret_cast<cf*>(s->dw + L.w_partial);
-  JacobiParams jp; memset(&jp, 0, sizeof(jp));
-  JacobiFastParams fp; memset(&fp, 0, sizeof(fp));
-  SubspaceParams sp; memset(&sp, 0, sizeof(sp));
-  size_t sub_bytes = 0;
-  int nslow = 0;
-  // no mode's factor is written yet (the eigensolvers below read these words)
-  if (cudaMemsetAsync(flags + SUB_DONE, 0, TGRAD_MAX_NDIM * sizeof(int), st) != cudaSuccess) return TGRAD_ERR_CUDA;
-  for (int m = 0; m < N; ++m) {
-    uint64_t O = 1, C = 1;
-    for (int q = 0; q < m; ++q) O *= c.dims[q];
-    for (int q = m + 1; q < N; ++q) C *= c.dims[q];
-    const int In = (int)c.dims[m];
-    const int T = (In + GR_T - 1) / GR_T;
-    cf* A = reinterpret_cast<cf*>(s->dw + L.w_gram[m]);
-    dim3 grid(T * T, L.gram_splits[m]);
-    // long contractions average the TF32 input rounding away; short ones get the split-precision products
-    const bool full = (In % GR_T) == 0;
-#define TG_GRAM(SPLIT_, FULL_)                                                                                      \
-  gram_partial_kernel<S, SPLIT_, FULL_><<<grid, GR_THREADS, GR_SMEM, st>>>(d_grad, In, (uint32_t)O, (uint32_t)C,    \
-                                                                          L.gram_chunks[m], L.gram_cps[m], partial)
-    if (O * C >= 16384) { if (full) TG_GRAM(false, true); else TG_GRAM(false, false); }
-    else { if (full) TG_GRAM(true, true); else TG_GRAM(true, false); }
-#undef TG_GRAM
-    TG_LAUNCH_CHECK();
-    gram_reduce_kernel<<<(In * In + GRR_E - 1) / GRR_E, GRR_E * GRR_G, 0, st>>>(partial, L.gram_splits[m], In, A); TG_LAUNCH_CHECK();
-    // leading eigenvectors by subspace iteration where the rank leaves room for guard columns ...
-    {
-      int R = 0; bool zsm = false;
-      if (sub_eligible(In, c.ranks[m], R, zsm)) {
-        SubspaceMode& sm_ = sp.mode[sp.nmodes++];
-        sm_.A = A; sm_.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
-        sm_.Zg = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
-        sm_.n = In; sm_.r = c.ranks[m]; sm_.R = R; sm_.index = m; sm_.z_in_smem = zsm ? 1 : 0;
-        const size_t b = sub_smem(In, R, zsm);
-        if (b > sub_bytes) sub_bytes = b;
-      }
+  // ---- factor matrices ----
+  // Starting factors: the leading eigenvectors of the mode-n Gram matrices of the residual (truncated SVDs of the
+  // unfoldings).  With refinement sweeps and a warm start, the factors the state holds are the starting point
+  // instead (the "warm restart" of the decomposition) and the full-size Gram matrices are not formed at all.
+  const bool from_stored = c.hooi_iters > 0 && c.warm_refresh && s->basis_valid;
+  if (!from_stored) {
+    int modes[TGRAD_MAX_NDIM];
+    for (int m = 0; m < N; ++m) {
+      uint64_t O = 1, C = 1;
+      for (int q = 0; q < m; ++q) O *= c.dims[q];
+      for (int q = m + 1; q < N; ++q) C *= c.dims[q];
+      TG_TRY(launch_gram<S>(s, d_grad, (int)c.dims[m], O, C, L.gram_chunks[m], L.gram_cps[m], L.gram_splits[m],
+                            reinterpret_cast<cf*>(s->dw + L.w_gram[m]), st));
+      modes[m] = m;
     }
-    // ... and the full Jacobi diagonalisation for every mode (it returns at once where the iteration has delivered)
-    if (L.jac_fast[m]) {
-      JacobiFastMode& fm = fp.mode[fp.nmodes++];
-      fm.A = A;
-      fm.work = reinterpret_cast<cf*>(s->dw + L.w_jac[m]);
-      fm.log = reinterpret_cast<float4*>(s->dw + L.w_log[m]);
-      fm.lam = reinterpret_cast<float*>(s->dw + L.w_lam[m]);
-      fm.V = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
-      fm.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
-      fm.n = In; fm.r = c.ranks[m]; fm.index = m; fm.row0 = fp.total_rows;
-      fp.total_rows += In;
-      if (In > fp.row_stride) fp.row_stride = In;
-    } else {
-      JacobiMode& jm = jp.mode[nslow];
-      jp.index[nslow++] = m;
-      jm.A = reinterpret_cast<cf*>(s->dw + L.w_jac[m]);
-      jm.V = reinterpret_cast<cf*>(s->dw + L.w_v[m]);
-      jm.U = reinterpret_cast<cf*>(s->dp + L.p_factor[m]);
-      jm.n = In; jm.r = c.ranks[m];
-      if (cudaMemcpyAsync(s->dw + L.w_jac[m], A, (size_t)In * In * 8, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-        return TGRAD_ERR_CUDA;
-    }
+    TG_TRY(solve_modes(s, modes, N, c.warm_refresh && s->basis_valid, st));
   }
+  // Refinement (higher-order orthogonal iteration): per sweep and mode, compress the residual in every other mode
+  // with the current factors and take the leading eigenvectors of the mode-n Gram matrix of the result.
+  for (int it = 0; it < c.hooi_iters; ++it)
+    for (int m = 0; m < N; ++m) TG_TRY(hooi_mode_update<S>(s, m, d_grad, st));
   if (k > 0) { scatter_restore_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, g_s, k); TG_LAUNCH_CHECK(); }
-  const int max_sweeps = c.jacobi_max_sweeps > 0 ? c.jacobi_max_sweeps : 30;
-  const float tol = c.jacobi_tol > 0.f ? c.jacobi_tol : 1e-6f;
-  if (sp.nmodes) {
-    sp.warm = (c.warm_refresh && s->basis_valid) ? 1 : 0;
-    sp.max_sweeps = max_sweeps; sp.tol = tol; sp.flags = flags;
-    subspace_kernel<<<sp.nmodes, SUB_THREADS, sub_bytes, st>>>(sp); TG_LAUNCH_CHECK();
-  }
-  if (nslow) {
-    jp.max_sweeps = max_sweeps; jp.tol = tol; jp.flags = flags;
-    jacobi_kernel<<<nslow, JAC_THREADS, 0, st>>>(jp); TG_LAUNCH_CHECK();
-  }
-  if (fp.nmodes) {
-    fp.max_sweeps = max_sweeps; fp.tol = tol; fp.flags = flags;
-    // the sweeps: modes whose matrix fits in shared memory in one launch, the larger ones (matrix in L2) in another
-    JacobiFastParams fs = fp, fg = fp;
-    fs.nmodes = fg.nmodes = 0;
-    size_t smem_s = 0, smem_g = 0;
-    for (int i = 0; i < fp.nmodes; ++i) {
-      const int n = fp.mode[i].n;
-      if (n <= JAC_SMEM_MAX_N) { fs.mode[fs.nmodes++] = fp.mode[i]; const size_t b = jac_sweeps_smem(n, true); if (b > smem_s) smem_s = b; }
-      else { fg.mode[fg.nmodes++] = fp.mode[i]; const size_t b = jac_sweeps_smem(n, false); if (b > smem_g) smem_g = b; }
-    }
-    if (fg.nmodes) { jacobi_sweeps_kernel<false><<<fg.nmodes, JAC_THREADS, smem_g, st>>>(fg); TG_LAUNCH_CHECK(); }
-    if (fs.nmodes) { jacobi_sweeps_kernel<true><<<fs.nmodes, JAC_THREADS, smem_s, st>>>(fs); TG_LAUNCH_CHECK(); }
-    fp.row_stride = (fp.row_stride + 1) & ~1;
-    const size_t vsm = (size_t)8 * fp.row_stride * sizeof(cf);
-    if (fp.row_stride <= 192) jacobi_vectors_kernel<3, 4><<<(fp.total_rows + 7) / 8, 256, vsm, st>>>(fp);
-    else jacobi_vectors_kernel<4, 2><<<(fp.total_rows + 7) / 8, 256, vsm, st>>>(fp);
-    TG_LAUNCH_CHECK();
-    jacobi_factors_kernel<<<fp.nmodes, JAC_THREADS, 0, st>>>(fp); TG_LAUNCH_CHECK();
-  }
   s->have_subspace = true;
   s->tabs_stale = true;
   s->basis_valid = true;

@@ -49,7 +49,7 @@ def storage_exact(x: np.ndarray, half: bool) -> np.ndarray:
 
 
 class Pair:
-    def __init__(self, wl: synth.Workload, tensor_id=0, warm_refresh=False, stagewise_w=False, **over):
+    def __init__(self, wl: synth.Workload, tensor_id=0, warm_refresh=False, stagewise_w=False, hooi_iters=0, **over):
         # stagewise_w: the expected weight is the oracle's weight update applied to the GPU's own normalised
         # updates N_L, N_S (which are themselves checked against the oracle's formula on the GPU's moments, and the
         # moments against the oracle's).  Needed where core entries vanish by construction: for a matrix the
@@ -61,10 +61,11 @@ class Pair:
         kw = dict(lr=wl.lr, alpha=1.0, lam=1.0, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0)
         kw.update(over)
         self.half = wl.half_storage
-        self.ocfg = orc.OracleConfig(shape=wl.shape, ranks=wl.ranks, k=wl.k, T=wl.T, half_storage=self.half, **kw)
+        self.ocfg = orc.OracleConfig(shape=wl.shape, ranks=wl.ranks, k=wl.k, T=wl.T, half_storage=self.half,
+                                     hooi_iters=hooi_iters, hooi_warm=warm_refresh, **kw)
         self.ost = orc.OracleState(self.ocfg)
         self.gcfg = B.make_config(wl.shape, wl.ranks, wl.k, wl.T, half_storage=self.half, auto_refresh=False,
-                                  warm_refresh=warm_refresh, **kw)
+                                  warm_refresh=warm_refresh, hooi_iters=hooi_iters, **kw)
         self.gst = B.TgradState(self.gcfg)
         w0 = storage_exact(self.src.weight(), self.half)
         self.w_ref = w0

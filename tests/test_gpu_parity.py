@@ -52,6 +52,24 @@ def test_trajectory_warm_refresh(name):
     print(name, p.report)
 
 
+@pytest.mark.parametrize("name,warm", [("small4", False), ("ragged4", False), ("odd32", True), ("cfg1", True), ("small5", False)])
+def test_hooi_refinement(name, warm):
+    # TuckerFactors with two refinement sweeps (higher-order orthogonal iteration) on noisier gradients, where the
+    # refined subspaces differ visibly from the truncated-SVD ones; warm: later refreshes start from the stored
+    # factors and skip the truncated-SVD stage
+    import dataclasses
+    wl = dataclasses.replace(synth.WORKLOADS[name], noise_scale=0.1)
+    p = Pair(wl, warm_refresh=warm, hooi_iters=2)
+    for t in range(2 * wl.T + 1):
+        p.step(t)
+    g = p.src.gradient(0)
+    res = orc.residual(g, orc.sparse_indices_topk(g, wl.k))
+    plain, refined = orc.tucker_factors(res, wl.ranks), orc.tucker_factors_hooi(res, wl.ranks, 2)
+    moved = max(H.max_sin_angle(a, b) for a, b in zip(plain, refined))
+    assert moved > 5e-3, f"the refinement barely moves the subspaces here ({moved}): the test would not notice its absence"
+    print("hooi", name, p.report.get("angle"), "moved", moved)
+
+
 def test_alpha_lambda_weight_decay():
     wl = synth.WORKLOADS["small4"]
     p = Pair(wl, alpha=0.25, lam=0.5, weight_decay=0.1, lr=1e-2)
