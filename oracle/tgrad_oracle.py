@@ -60,6 +60,105 @@ def sparse_indices_topk(g: np.ndarray, k: int) -> np.ndarray:
     return np.sort(order[:k]).astype(np.uint32)
 
 
+# ---- the other two sparsification strategies of Section 2.2 ("probabilistic sampling, or uniform random
+#      selection"); the paper names them without defining them, so the definitions below are stated readings ----
+
+_PHILOX_M0, _PHILOX_M1 = np.uint64(0xD2511F53), np.uint64(0xCD9E8D57)
+_PHILOX_W0, _PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+
+
+def philox4x32_10(counter, key):
+    """Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3",
+    SC 2011): counter = four uint32 arrays (or scalars), key = two uint32 scalars; returns four uint32 arrays.
+    Round: (c0, c1, c2, c3) <- (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0)); the key is bumped by
+    the Weyl constants (W0, W1) between rounds."""
+    c = [np.asarray(x, dtype=np.uint64) & np.uint64(0xFFFFFFFF) for x in counter]
+    c = list(np.broadcast_arrays(*c))
+    k0, k1 = int(key[0]) & 0xFFFFFFFF, int(key[1]) & 0xFFFFFFFF
+    mask = np.uint64(0xFFFFFFFF)
+    for _ in range(10):
+        p0 = _PHILOX_M0 * c[0]
+        p1 = _PHILOX_M1 * c[2]
+        c = [(p1 >> np.uint64(32)) ^ c[1] ^ np.uint64(k0), p1 & mask, (p0 >> np.uint64(32)) ^ c[3] ^ np.uint64(k1), p0 & mask]
+        k0 = (k0 + _PHILOX_W0) & 0xFFFFFFFF
+        k1 = (k1 + _PHILOX_W1) & 0xFFFFFFFF
+    return [x.astype(np.uint32) for x in c]
+
+
+def selection_word(numel: int, seed: int, epoch: int) -> np.ndarray:
+    """One 32-bit random word per flat index i for the refresh number `epoch`: the first output word of
+    Philox-4x32-10 with counter (i, epoch, 0, 0) and key (seed mod 2^32, seed div 2^32)."""
+    i = np.arange(numel, dtype=np.uint64)
+    return philox4x32_10((i, np.uint64(epoch), np.uint64(0), np.uint64(0)), (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))[0]
+
+
+_LN2_F = np.float32(0.693147182)
+_SQRT2_F = np.float32(1.41421354)
+_C3, _C5, _C7, _C9 = np.float32(1.0 / 3.0), np.float32(0.2), np.float32(1.0 / 7.0), np.float32(1.0 / 9.0)
+
+
+def neg_log_uniform(word: np.ndarray) -> np.ndarray:
+    """E = -ln(u), u = ((word >> 9) + 1/2) 2^-23 in (0, 1), evaluated in fp32 by a fixed sequence of IEEE operations
+    (no fused multiply-add) so that every implementation gets the same bits: u = m 2^e with m in (sqrt(1/2), sqrt(2)],
+    f = m - 1, s = f / (f + 2), z = s s, ln m = 2 (s + s z (1/3 + z (1/5 + z (1/7 + z / 9)))), ln u = e ln 2 + ln m.
+    An exponential variate of unit rate up to the 1e-7 relative error of the series."""
+    w = np.asarray(word, dtype=np.uint32)
+    u = ((w >> np.uint32(9)).astype(np.float32) + np.float32(0.5)) * np.float32(2.0 ** -23)
+    bits = u.view(np.uint32)
+    e = (bits >> np.uint32(23)).astype(np.int32) - 127
+    m = ((bits & np.uint32(0x7FFFFF)) | np.uint32(0x3F800000)).view(np.float32)
+    big = m > _SQRT2_F
+    m = np.where(big, m * np.float32(0.5), m).astype(np.float32)
+    e = np.where(big, e + 1, e)
+    f = m - np.float32(1.0)
+    s_ = f / (f + np.float32(2.0))
+    z = s_ * s_
+    p = _C9 * z
+    p = p + _C7
+    p = p * z
+    p = p + _C5
+    p = p * z
+    p = p + _C3
+    r = s_ * z
+    r = r * p
+    r = r + s_
+    r = r * np.float32(2.0)
+    ln_u = e.astype(np.float32) * _LN2_F
+    ln_u = ln_u + r
+    return (-ln_u).astype(np.float32)
+
+
+def selection_key(g: np.ndarray, strategy: str, seed: int = 0, epoch: int = 0) -> np.ndarray:
+    """The non-negative fp32 key whose k largest values (ties to the lower flat index) define Omega.
+    topk:  |g|^2 (magnitude_key).
+    randk: the random word itself, as an integer: a uniformly random k-subset, independent of g.
+    probk: |g| / E with E a unit-rate exponential variate per entry -- the k largest of these are a sample of k
+           entries without replacement with probabilities proportional to |g| (the exponential-clocks form of
+           weighted reservoir sampling, Efraimidis and Spirakis 2006); |g| = sqrt of the fp32 key, division in fp32."""
+    if strategy == "topk":
+        return magnitude_key(g).reshape(-1)
+    word = selection_word(int(np.asarray(g).size), seed, epoch)
+    if strategy == "randk":
+        return word
+    if strategy == "probk":
+        w = np.sqrt(magnitude_key(g).reshape(-1))
+        return (w / neg_log_uniform(word)).astype(np.float32)
+    raise ValueError(strategy)
+
+
+def sparse_indices(g: np.ndarray, k: int, strategy: str = "topk", seed: int = 0, epoch: int = 0) -> np.ndarray:
+    """SparseIndices(G, rho, strategy) of Algorithm 1: the k entries with the largest selection_key, ties to the
+    lower flat index, as ascending flat indices."""
+    if strategy == "topk":
+        return sparse_indices_topk(g, k)
+    key = selection_key(g, strategy, seed, epoch)
+    if k < 0 or k > key.size:
+        raise ValueError("k out of range")
+    bits = key.view(np.uint32) if key.dtype == np.float32 else key
+    order = np.argsort(-(bits.astype(np.int64)), kind="stable")
+    return np.sort(order[:k]).astype(np.uint32)
+
+
 def sparse_gather(g: np.ndarray, omega: np.ndarray) -> np.ndarray:
     """Sparse(G, Omega): the values at the stored indices (the per-step
     "create sparse tensor" statement of Algorithm 1)."""
@@ -227,6 +326,12 @@ class OracleConfig:
     half_storage: bool = False      # W and G live as fp16 (re, im) pairs
     hooi_iters: int = 0             # refinement sweeps of TuckerFactors (0: truncated-SVD factors only)
     hooi_warm: bool = False         # refinement starts from the factors of the previous refresh when there are any
+    strategy: str = "topk"          # topk | randk | probk (Section 2.2, sparsification strategies)
+    seed: int = 0                   # of the random strategies
+    composition: str = "us_lr"      # us_lr: Algorithm 1 (sparse first, low rank on the residual);
+                                    # lr_us: low rank first, sparse part taken from G - P_U(G);
+                                    # sum: both applied to the gradient itself and added (Section 2.2 "Residual and
+                                    # composition"; the combination ablation)
 
 
 def _store_w(w: np.ndarray, half: bool) -> np.ndarray:
@@ -258,17 +363,37 @@ class OracleState:
         self.n_s = None
 
 
+def _factors_of(cfg: OracleConfig, x: np.ndarray, prev) -> List[np.ndarray]:
+    if cfg.hooi_iters > 0:
+        init = prev if (cfg.hooi_warm and prev is not None) else None
+        return tucker_factors_hooi(x, cfg.ranks, cfg.hooi_iters, init)
+    return tucker_factors(x, cfg.ranks)
+
+
+def lowrank_residual(cfg: OracleConfig, grad: np.ndarray, factors) -> np.ndarray:
+    """G - P_U(G), P_U(G) = (G x_n U^(n)H) x_n U^(n), rounded to the storage type of the gradient: what the sparse
+    part sees when the low-rank part goes first."""
+    x = np.asarray(grad, dtype=np.complex128)
+    return _store_w(x - tucker_reconstruct(tucker_compress(x, factors), factors), cfg.half_storage).astype(np.complex64)
+
+
 def oracle_refresh(st: OracleState, grad: np.ndarray) -> None:
     """The `t mod T = 0` branch of Algorithm 1: new Omega, residual, new factors.  Moments are
-    left untouched (nothing in the loop resets them)."""
+    left untouched (nothing in the loop resets them).  The first component sees the gradient, the second the
+    residual of the first (composition "sum": both see the gradient)."""
     cfg = st.cfg
-    st.omega = sparse_indices_topk(grad, cfg.k)
-    res = residual(grad, st.omega)
-    if cfg.hooi_iters > 0:
-        init = st.factors if (cfg.hooi_warm and st.factors is not None) else None
-        st.factors = tucker_factors_hooi(res, cfg.ranks, cfg.hooi_iters, init)
+    epoch = st.t // cfg.T
+    if cfg.composition == "us_lr":
+        st.omega = sparse_indices(grad, cfg.k, cfg.strategy, cfg.seed, epoch)
+        st.factors = _factors_of(cfg, residual(grad, st.omega), st.factors)
+    elif cfg.composition == "sum":
+        st.omega = sparse_indices(grad, cfg.k, cfg.strategy, cfg.seed, epoch)
+        st.factors = _factors_of(cfg, np.asarray(grad), st.factors)
+    elif cfg.composition == "lr_us":
+        st.factors = _factors_of(cfg, np.asarray(grad), st.factors)
+        st.omega = sparse_indices(lowrank_residual(cfg, grad, st.factors), cfg.k, cfg.strategy, cfg.seed, epoch)
     else:
-        st.factors = tucker_factors(res, cfg.ranks)
+        raise ValueError(cfg.composition)
 
 
 def weight_update(cfg: OracleConfig, w: np.ndarray, n_l: np.ndarray, n_s: np.ndarray, omega: np.ndarray,
@@ -305,8 +430,18 @@ def oracle_step(st: OracleState, w: np.ndarray, grad: np.ndarray, refresh: Optio
     if do_refresh:
         oracle_refresh(st, grad)
     # sparse values, residual, low-rank compression
-    g_s = sparse_gather(grad, st.omega).astype(np.complex64)
-    core = tucker_compress(residual(grad, st.omega), st.factors).astype(np.complex64)
+    if cfg.composition == "us_lr":
+        g_s = sparse_gather(grad, st.omega).astype(np.complex64)
+        core = tucker_compress(residual(grad, st.omega), st.factors).astype(np.complex64)
+    elif cfg.composition == "sum":
+        g_s = sparse_gather(grad, st.omega).astype(np.complex64)
+        core = tucker_compress(grad, st.factors).astype(np.complex64)
+    else:
+        # low rank first: the core of the gradient itself; the sparse values are those of G - P_U(G), with P_U(G)
+        # rebuilt from the core as stored (fp32)
+        core = tucker_compress(grad, st.factors).astype(np.complex64)
+        low = tucker_reconstruct(core, st.factors).reshape(-1)[st.omega.astype(np.int64)]
+        g_s = (sparse_gather(grad, st.omega).astype(np.complex128) - low).astype(np.complex64)
     # AdamUpdate on both compressed parts
     n_s, st.m_s, st.v_s = adam_update(g_s, st.m_s, st.v_s, cfg.beta1, cfg.beta2, cfg.eps, st.t)
     n_l, st.m_l, st.v_l = adam_update(core, st.m_l, st.v_l, cfg.beta1, cfg.beta2, cfg.eps, st.t)

@@ -488,6 +488,126 @@ def test_half_storage_rounds_after_the_dense_update_and_again_at_omega():
     assert float(np.float16(1.5 - 1.2 * u)) == 1.5 - u          # what one rounding would have stored at Omega
 
 
+# ---- random sparsification strategies and the other composition orders ----------------------------------
+
+def test_philox_known_answers():
+    for line in open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        w = [int(x, 16) for x in line.split()]
+        out = orc.philox4x32_10(w[0:4], w[4:6])
+        assert [int(x.reshape(-1)[0]) for x in out] == w[6:10]
+
+
+def test_randk_is_a_uniform_k_subset_independent_of_the_gradient():
+    rng = np.random.default_rng(40)
+    shape = (16, 16, 8)
+    g1 = (rng.standard_normal(shape) + 1j * rng.standard_normal(shape)).astype(np.complex64)
+    g2 = (g1 * 100).astype(np.complex64)
+    k = 300
+    a = orc.sparse_indices(g1, k, "randk", seed=7, epoch=0)
+    assert a.size == k and np.all(np.diff(a.astype(np.int64)) > 0) and a[-1] < g1.size
+    assert np.array_equal(a, orc.sparse_indices(g2, k, "randk", seed=7, epoch=0))          # does not look at g
+    assert not np.array_equal(a, orc.sparse_indices(g1, k, "randk", seed=7, epoch=1))      # redrawn at each refresh
+    assert not np.array_equal(a, orc.sparse_indices(g1, k, "randk", seed=8, epoch=0))
+    # uniform: over many epochs every position is taken about k / I of the time
+    hits = np.zeros(g1.size)
+    n_ep = 400
+    for ep in range(n_ep):
+        hits[orc.sparse_indices(g1, k, "randk", seed=3, epoch=ep).astype(np.int64)] += 1
+    p = k / g1.size
+    z = (hits - n_ep * p) / np.sqrt(n_ep * p * (1 - p))
+    assert abs(z.mean()) < 0.05 and 0.9 < z.std() < 1.1 and np.abs(z).max() < 5.5
+
+
+def test_exponential_variate_recipe_is_minus_log():
+    w = np.random.default_rng(41).integers(0, 2 ** 32, 200000, dtype=np.uint64).astype(np.uint32)
+    w[:3] = [0, 0xFFFFFFFF, 1 << 31]
+    e = orc.neg_log_uniform(w)
+    u = ((w >> 9).astype(np.float64) + 0.5) * 2.0 ** -23
+    assert e.dtype == np.float32 and np.all(e > 0)
+    assert np.max(np.abs(e + np.log(u)) / -np.log(u)) < 4e-7
+    assert abs(float(e.mean()) - 1.0) < 0.01                                                 # unit-rate exponential
+
+
+def test_probk_samples_proportionally_to_magnitude():
+    # k = 1: the entry with the largest |g| / E wins with probability |g_i| / sum |g| (exponential clocks)
+    g = np.array([1, 2j, -3, 4 - 0j, 0], dtype=np.complex64)
+    counts = np.zeros(5)
+    n = 6000
+    for seed in range(n):
+        counts[int(orc.sparse_indices(g, 1, "probk", seed=seed, epoch=0)[0])] += 1
+    want = np.array([1, 2, 3, 4, 0]) / 10.0
+    assert counts[4] == 0                                                                   # zero magnitude: never drawn first
+    assert np.all(np.abs(counts[:4] / n - want[:4]) < 4 * np.sqrt(want[:4] * (1 - want[:4]) / n))
+    # k = 4 of these five: always the four non-zero entries
+    assert orc.sparse_indices(g, 4, "probk", seed=1, epoch=3).tolist() == [0, 1, 2, 3]
+    # and the key is what the definition says, element by element
+    key = orc.selection_key(g, "probk", seed=5, epoch=2)
+    word = orc.selection_word(5, 5, 2)
+    u = ((word >> 9).astype(np.float64) + 0.5) * 2.0 ** -23
+    assert np.allclose(key[:4], np.abs(g[:4]) / -np.log(u[:4]), rtol=1e-6) and key[4] == 0
+
+
+def _kron_projector(us):
+    """Matrix of P_U on row-major vec(G): kron of U_n U_n^H."""
+    p = np.ones((1, 1), dtype=np.complex128)
+    for u in us:
+        u = u.astype(np.complex128)
+        p = np.kron(p, u @ np.conj(u).T)
+    return p
+
+
+def test_composition_sum_applies_both_parts_to_the_gradient():
+    wl = synth.WORKLOADS["tiny4"]
+    src = synth.GradientSource(wl)
+    g, w0 = src.gradient(0), src.weight()
+    cfg = orc.OracleConfig(shape=wl.shape, ranks=wl.ranks, k=wl.k, T=wl.T, lr=1e-2, composition="sum")
+    st = orc.OracleState(cfg)
+    w1 = orc.oracle_step(st, w0, g)
+    assert np.array_equal(st.omega, orc.sparse_indices_topk(g, wl.k))
+    # factors come from the gradient itself, not from the residual
+    for a, b in zip(st.factors, orc.tucker_factors(g, wl.ranks)):
+        assert H.max_sin_angle(a, b) < 1e-6
+    # first step: N = x / (|x| + eps) on both parts, low-rank part = P_U applied to N_L through the kron projector
+    core = orc.tucker_compress(g, st.factors)
+    n_l = core / (np.abs(core) + 1e-8)
+    dense = orc.tucker_reconstruct(n_l, st.factors).reshape(-1)
+    gs = g.reshape(-1)[st.omega.astype(np.int64)].astype(np.complex128)
+    want = w0.reshape(-1).astype(np.complex128) - 1e-2 * dense
+    want[st.omega.astype(np.int64)] -= 1e-2 * gs / (np.abs(gs) + 1e-8)
+    assert np.max(np.abs(w1.reshape(-1) - want)) < 2e-6
+    assert np.allclose(st.core.reshape(-1), (np.conj(np.kron(np.kron(np.kron(st.factors[0], st.factors[1]), st.factors[2]),
+                                                             st.factors[3]).astype(np.complex128)).T @ g.reshape(-1)), atol=1e-4)
+
+
+def test_composition_lr_us_takes_the_sparse_part_from_the_lowrank_residual():
+    wl = synth.WORKLOADS["tiny4"]
+    src = synth.GradientSource(wl)
+    g, w0 = src.gradient(0), src.weight()
+    cfg = orc.OracleConfig(shape=wl.shape, ranks=wl.ranks, k=wl.k, T=wl.T, lr=1e-2, composition="lr_us")
+    st = orc.OracleState(cfg)
+    w1 = orc.oracle_step(st, w0, g)
+    us = st.factors
+    for a, b in zip(us, orc.tucker_factors(g, wl.ranks)):
+        assert H.max_sin_angle(a, b) < 1e-6
+    # residual through the explicit projector matrix; Omega = its k largest entries by brute force
+    r = (g.reshape(-1).astype(np.complex128) - _kron_projector(us) @ g.reshape(-1).astype(np.complex128)).reshape(wl.shape)
+    assert np.max(np.abs(orc.lowrank_residual(cfg, g, us) - r)) < 1e-6
+    assert st.omega.tolist() == H.brute_topk(orc.lowrank_residual(cfg, g, us), wl.k)
+    assert np.max(np.abs(st.g_s - r.reshape(-1)[st.omega.astype(np.int64)])) < 1e-5
+    # the low-rank part is that of the whole gradient
+    assert np.max(np.abs(st.core - orc.tucker_compress(g, us))) < 1e-5
+    # full ranks: nothing is left for the sparse part, and the step is the low-rank step alone
+    full = orc.OracleConfig(shape=wl.shape, ranks=wl.shape, k=wl.k, T=wl.T, lr=1e-2, composition="lr_us")
+    lo = orc.OracleConfig(shape=wl.shape, ranks=wl.shape, k=0, T=wl.T, lr=1e-2)
+    sa, sb = orc.OracleState(full), orc.OracleState(lo)
+    wa, wb = orc.oracle_step(sa, w0, g), orc.oracle_step(sb, w0, g)
+    assert np.max(np.abs(sa.g_s)) < 1e-5 * np.max(np.abs(g))
+    mask = np.ones(g.size, bool); mask[sa.omega.astype(np.int64)] = False
+    assert np.max(np.abs(wa.reshape(-1)[mask] - wb.reshape(-1)[mask])) < 1e-6
+
+
 # ---- state size: the paper's worked example --------------------------------------------------
 
 def test_state_size_matches_paper_example():
