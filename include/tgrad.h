@@ -108,6 +108,17 @@ typedef struct {
                                        truncated-SVD stage is skipped (the warm restart of the decomposition).
                                        Needs extra workspace, and each trailing slab must still fit in shared
                                        memory with one of its two factors replaced by the identity            */
+  int32_t composition;              /* order of the two parts (Section 2.2 "Residual and composition"):
+                                       0: sparse part first, low-rank part on its residual (Algorithm 1);
+                                       1: low-rank part first, the sparse part selected from and fed with
+                                          G - P_U(G), P_U(G) the low-rank approximation of the gradient;
+                                       2: both parts applied to the gradient itself and added                 */
+  int32_t sparse_strategy;          /* how Omega is chosen at a refresh (Section 2.2 "Unstructured sparse gradient
+                                       tensor"): 0 top-k magnitude; 1 uniform random k-subset; 2 sampling without
+                                       replacement with probabilities proportional to |g|.  1 and 2 rank the
+                                       entries by a key built from one Philox-4x32-10 word per entry (counter =
+                                       flat index, refresh number t / T) and take the k largest                */
+  uint64_t seed;                    /* key of that generator                                                   */
 } tgrad_config;
 
 /* Selectors for tgrad_export_state / tgrad_import_state.  FACTOR_BASE + n is

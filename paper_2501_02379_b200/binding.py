@@ -23,6 +23,8 @@ ERR_TOO_LARGE = 8
 NOALLOC_MAX_NUMEL = 1 << 26
 FLAG_NO_CONVERGE, FLAG_NONFINITE, FLAG_COPY_TIMEOUT = 1, 2, 4
 C64, C32H = 0, 1
+COMPOSITIONS = {"us_lr": 0, "lr_us": 1, "sum": 2}
+STRATEGIES = {"topk": 0, "randk": 1, "probk": 2}
 WHAT_OMEGA, WHAT_M_L, WHAT_V_L, WHAT_M_S, WHAT_V_S, WHAT_CORE, WHAT_N_L, WHAT_N_S = 1, 2, 3, 4, 5, 6, 7, 8
 WHAT_GRAM_BASE, WHAT_FACTOR_BASE = 32, 64
 
@@ -43,6 +45,9 @@ class TgradConfig(C.Structure):
         ("jacobi_tol", C.c_float),
         ("warm_refresh", C.c_int32),
         ("hooi_iters", C.c_int32),
+        ("composition", C.c_int32),
+        ("sparse_strategy", C.c_int32),
+        ("seed", C.c_uint64),
     ]
 
 
@@ -114,7 +119,7 @@ def make_config(shape: Sequence[int], ranks: Sequence[int], k: int, T: int, lr: 
                 lam: float = 1.0, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
                 weight_decay: float = 0.0, half_storage: bool = False, auto_refresh: bool = True,
                 jacobi_max_sweeps: int = 0, jacobi_tol: float = 0.0, warm_refresh: bool = False,
-                hooi_iters: int = 0) -> TgradConfig:
+                hooi_iters: int = 0, composition: str = "us_lr", strategy: str = "topk", seed: int = 0) -> TgradConfig:
     if len(shape) > MAX_NDIM or len(shape) != len(ranks):
         raise ValueError("bad shape / ranks")
     cfg = TgradConfig()
@@ -133,6 +138,9 @@ def make_config(shape: Sequence[int], ranks: Sequence[int], k: int, T: int, lr: 
     cfg.jacobi_tol = jacobi_tol
     cfg.warm_refresh = 1 if warm_refresh else 0
     cfg.hooi_iters = int(hooi_iters)
+    cfg.composition = COMPOSITIONS[composition]
+    cfg.sparse_strategy = STRATEGIES[strategy]
+    cfg.seed = int(seed)
     return cfg
 
 

@@ -16,6 +16,66 @@ struct SelState {
   uint32_t take_eq;  // how many entries with key == thr belong to Omega
 };
 
+// What the entries are ranked by (SparseIndices of Algorithm 1 with one of the sparsification strategies of
+// Section 2.2): 0 top-k magnitude, 1 uniform random selection, 2 probabilistic sampling proportional to |g|.
+struct SelKey {
+  uint32_t seed_lo, seed_hi;   // key of the counter-based generator
+  uint32_t epoch;              // number of the refresh (the sets are redrawn at every refresh)
+  int strategy;
+};
+
+// First output word of Philox-4x32 with 10 rounds (Salmon et al., "Parallel random numbers: as easy as 1, 2, 3") for
+// the counter (i, epoch, 0, 0).
+__device__ __forceinline__ uint32_t sel_word(uint32_t i, const SelKey& kp) {
+  uint32_t c0 = i, c1 = kp.epoch, c2 = 0u, c3 = 0u, k0 = kp.seed_lo, k1 = kp.seed_hi;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+    const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+    c0 = h1 ^ c1 ^ k0; c1 = l1; c2 = h0 ^ c3 ^ k1; c3 = l0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return c0;
+}
+
+// E = -ln(u), u = ((word >> 9) + 1/2) 2^-23: a unit-rate exponential variate.  A fixed sequence of IEEE fp32
+// operations without fused multiply-adds, so that any implementation of the same recipe gets the same bits:
+// u = m 2^e with m in (sqrt(1/2), sqrt(2)], f = m - 1, s = f / (f + 2), z = s s,
+// ln m = 2 (s + s z (1/3 + z (1/5 + z (1/7 + z / 9)))), ln u = e ln 2 + ln m.
+__device__ __forceinline__ float sel_neg_log(uint32_t word) {
+  const float u = __fmul_rn(__fadd_rn((float)(word >> 9), 0.5f), 1.1920928955078125e-07f);   // 2^-23
+  const uint32_t bits = __float_as_uint(u);
+  int e = (int)(bits >> 23) - 127;
+  float m = __uint_as_float((bits & 0x7FFFFFu) | 0x3F800000u);
+  if (m > 1.41421354f) { m = __fmul_rn(m, 0.5f); e += 1; }
+  const float f = __fadd_rn(m, -1.0f);
+  const float sq = __fdiv_rn(f, __fadd_rn(f, 2.0f));
+  const float z = __fmul_rn(sq, sq);
+  float pl = __fmul_rn(0.111111112f, z);
+  pl = __fadd_rn(pl, 0.142857149f);
+  pl = __fmul_rn(pl, z);
+  pl = __fadd_rn(pl, 0.2f);
+  pl = __fmul_rn(pl, z);
+  pl = __fadd_rn(pl, 0.333333343f);
+  float r = __fmul_rn(sq, z);
+  r = __fmul_rn(r, pl);
+  r = __fadd_rn(r, sq);
+  r = __fmul_rn(r, 2.0f);
+  float ln_u = __fmul_rn((float)e, 0.693147182f);
+  ln_u = __fadd_rn(ln_u, r);
+  return -ln_u;
+}
+
+// The key of entry i with value v: its k largest (ties to the lower index) are selected.  Keys are non-negative
+// floats or plain integers, so their bit patterns order like their values.
+__device__ __forceinline__ uint32_t sel_key(cf v, uint32_t i, const SelKey& kp) {
+  if (kp.strategy == 0) return mag_key(v);
+  const uint32_t w = sel_word(i, kp);
+  if (kp.strategy == 1) return w;
+  const float mag = __fsqrt_rn(__uint_as_float(mag_key(v)));
+  return __float_as_uint(__fdiv_rn(mag, sel_neg_log(w)));
+}
+
 // three passes over the 32 key bits: 11 + 11 + 10
 __host__ __device__ inline int sel_bits(int pass) { return pass == 2 ? 10 : 11; }
 __host__ __device__ inline int sel_shift(int pass) { return pass == 0 ? 21 : (pass == 1 ? 10 : 0); }
@@ -32,7 +92,7 @@ __global__ void sel_init_kernel(SelState* st, uint32_t k) {
 template <class S>
 __global__ void __launch_bounds__(512) sel_hist_kernel(const void* __restrict__ g, uint32_t n, int pass,
                                                       const SelState* __restrict__ st, uint32_t* __restrict__ hist,
-                                                      int* __restrict__ flags) {
+                                                      int* __restrict__ flags, SelKey kp) {
   __shared__ uint32_t sh[kSelMaxBins];
   const int bits = sel_bits(pass), shift = sel_shift(pass);
   const uint32_t nb = 1u << bits;
@@ -51,12 +111,15 @@ __global__ void __launch_bounds__(512) sel_hist_kernel(const void* __restrict__ 
     for (int j = 0; j < UN; ++j) {
       const uint64_t i = b0 + (uint64_t)j * blockDim.x + threadIdx.x;
       valid[j] = i < n;
-      keys[j] = valid[j] ? mag_key(S::load(g, i)) : 0u;
+      cf v = make_float2(0.f, 0.f);
+      if (valid[j]) v = S::load(g, i);
+      keys[j] = valid[j] ? sel_key(v, (uint32_t)i, kp) : 0u;
+      // a NaN or an infinity among the magnitudes (the random strategy does not look at them)
+      if (pass == 0 && kp.strategy != 1 && (mag_key(v) & 0x7f800000u) == 0x7f800000u) bad = true;
     }
 #pragma unroll
     for (int j = 0; j < UN; ++j) {
       const uint32_t key = keys[j];
-      if (pass == 0 && (key & 0x7f800000u) == 0x7f800000u) bad = true;
       bool in = valid[j] && (key & hi_mask) == prefix;
       uint32_t d = (key >> shift) & (nb - 1u);
       // warp-aggregated shared atomics: gradients crowd into a few exponent bins
@@ -125,7 +188,7 @@ template <class S>
 __global__ void __launch_bounds__(kChunkThreads) sel_count_kernel(const void* __restrict__ g, uint32_t n,
                                                                   const SelState* __restrict__ st,
                                                                   uint32_t* __restrict__ blk_gt,
-                                                                  uint32_t* __restrict__ blk_eq) {
+                                                                  uint32_t* __restrict__ blk_eq, SelKey kp) {
   __shared__ uint32_t sg[kChunkThreads / 32], se[kChunkThreads / 32];
   const uint32_t thr = st->thr;
   const uint32_t base = blockIdx.x * (uint32_t)kChunk;
@@ -134,7 +197,7 @@ __global__ void __launch_bounds__(kChunkThreads) sel_count_kernel(const void* __
   for (int r = 0; r < kChunk / kChunkThreads; ++r) {
     uint32_t i = base + r * kChunkThreads + threadIdx.x;
     if (i < n) {
-      uint32_t key = mag_key(S::load(g, i));
+      uint32_t key = sel_key(S::load(g, i), i, kp);
       cg += key > thr; ce += key == thr;
     }
   }
@@ -194,7 +257,7 @@ __global__ void __launch_bounds__(kChunkThreads) sel_compact_kernel(const void* 
                                                                     const uint32_t* __restrict__ blk_gt,
                                                                     const uint32_t* __restrict__ blk_eq,
                                                                     uint32_t* __restrict__ omega,
-                                                                    cf* __restrict__ g_s, uint32_t k) {
+                                                                    cf* __restrict__ g_s, uint32_t k, SelKey kp) {
   __shared__ uint32_t wsum[kChunkThreads / 32];
   constexpr int EPT = kChunk / kChunkThreads;   // 8 consecutive entries per thread
   const uint32_t thr = st->thr, take = st->take_eq;
@@ -205,7 +268,7 @@ __global__ void __launch_bounds__(kChunkThreads) sel_compact_kernel(const void* 
 #pragma unroll
   for (int e = 0; e < EPT; ++e) {
     uint32_t i = base + e;
-    if (i < n) { v[e] = S::load(g, i); key[e] = mag_key(v[e]); } else { v[e] = make_float2(0.f, 0.f); key[e] = 0u; }
+    if (i < n) { v[e] = S::load(g, i); key[e] = sel_key(v[e], i, kp); } else { v[e] = make_float2(0.f, 0.f); key[e] = 0u; }
     bool valid = i < n;
     cnt += (valid && key[e] > thr) ? 1u : 0u;
     cnt += (valid && key[e] == thr) ? 0x10000u : 0u;

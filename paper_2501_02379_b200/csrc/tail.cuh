@@ -45,6 +45,8 @@ struct TailParams {
   const uint32_t* omega; // ascending flat indices
   const uint32_t* slab_ptr; // slab_ptr[s] = first Omega slot of slab s (nslab + 1 entries)
   int k;
+  int keep;              // compression: 1 = gather the entries at Omega but leave them in place (the low-rank part sees
+                         // the gradient itself, not the residual of the sparse part)
   cf* m_s; float* v_s;   // sparse moments (proj)
   cf* g_s;               // gathered sparse values (fast path: their Adam update runs in the Adam kernel)
   cf* n_s;               // normalised sparse update: written by proj, read by back
@@ -123,7 +125,7 @@ __global__ void __launch_bounds__(TB_THREADS) proj_tail_blk_kernel(const void* _
         const uint32_t a = loc / B;
         const uint32_t si = a * Bs + (loc - a * B);
         p.g_s[j] = xs[si];
-        xs[si] = make_float2(0.f, 0.f);
+        if (!p.keep) xs[si] = make_float2(0.f, 0.f);
       }
       __syncthreads();
     }

@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(512, 1) proj_tail_h_kernel(const void* __restr
           const uint32_t loc = (first ? pom : p.omega[j]) - base;
           const uint32_t xv = xs[loc];
           p.g_s[j] = __half22float2(*reinterpret_cast<const __half2*>(&xv));
-          xs[loc] = 0u;
+          if (!p.keep) xs[loc] = 0u;
         }
         if (b0 + tid < b1) fence_async_smem();   // the zeroed words were written through the generic proxy; a bulk copy overwrites them later
         b0 = c0; b1 = c1; pom = pomc;

@@ -278,12 +278,12 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, 4) proj_tail_tc_kernel(const vo
       if (jcur < b1) {
         cf* xp = reinterpret_cast<cf*>(xg) + (pom - base);
         p.g_s[jcur] = *xp;
-        *xp = make_float2(0.f, 0.f);
+        if (!p.keep) *xp = make_float2(0.f, 0.f);
       }
       for (int j = jcur + PJ_THREADS; j < b1; j += PJ_THREADS) {   // more entries than threads: not prefetched
         cf* xp = reinterpret_cast<cf*>(xg) + (p.omega[j] - base);
         p.g_s[j] = *xp;
-        *xp = make_float2(0.f, 0.f);
+        if (!p.keep) *xp = make_float2(0.f, 0.f);
       }
     }
     if (__syncthreads_or(!ok)) {

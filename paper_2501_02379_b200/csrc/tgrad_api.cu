@@ -37,7 +37,7 @@ struct Layout {
   uint32_t nslab, E;          // slabs of the trailing two modes, entries per slab
   // workspace block
   size_t w_ns, w_gs, w_core, w_nl, w_bufa, w_bufb, w_sel, w_hist, w_blk, w_gram[TGRAD_MAX_NDIM], w_jac[TGRAD_MAX_NDIM],
-      w_v[TGRAD_MAX_NDIM], w_log[TGRAD_MAX_NDIM], w_lam[TGRAD_MAX_NDIM], w_partial, w_hooi0, w_hooi1, w_ident, w_total;
+      w_v[TGRAD_MAX_NDIM], w_log[TGRAD_MAX_NDIM], w_lam[TGRAD_MAX_NDIM], w_partial, w_hooi0, w_hooi1, w_ident, w_rbuf, w_total;
   uint32_t hooi_smem;         // shared memory of the compression kernel when one trailing factor is replaced by the identity
   bool jac_fast[TGRAD_MAX_NDIM];    // eigensolver with the matrix in shared memory and a rotation log
   uint64_t numel, P, tsize;   // entries, core entries, entries of the tail-contracted tensor
@@ -80,6 +80,7 @@ tgrad_status validate(const tgrad_config* c) {
   if (c->jacobi_max_sweeps < 0 || c->jacobi_tol < 0.f) return TGRAD_ERR_INVALID_ARG;
   if (c->warm_refresh != 0 && c->warm_refresh != 1) return TGRAD_ERR_INVALID_ARG;
   if (c->hooi_iters < 0 || c->hooi_iters > 64) return TGRAD_ERR_INVALID_ARG;
+  if (c->composition < 0 || c->composition > 2 || c->sparse_strategy < 0 || c->sparse_strategy > 2) return TGRAD_ERR_INVALID_ARG;
   // limits of this implementation
   if (tot >= 4294967296.0L) return TGRAD_ERR_UNSUPPORTED;    // flat indices are uint32
   if (c->k >= ((int64_t)1 << 31)) return TGRAD_ERR_UNSUPPORTED;   // slots of Omega are addressed with int
@@ -199,6 +200,9 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
     const uint64_t mx = A > B ? A : B;
     L.w_ident = o; o = align_up(o + (size_t)(mx * mx) * 8);
   }
+  // low-rank-first composition: G - P_U(G) at full size, from which a refresh selects Omega
+  L.w_rbuf = o;
+  if (c->composition == 1) o = align_up(o + (size_t)numel * (c->wg_dtype == TGRAD_C64 ? 8 : 4));
   L.w_total = o;
   return TGRAD_OK;
 }
@@ -557,6 +561,182 @@ tgrad_status solve_modes(tgrad_state* s, const int* modes, int nm, bool warm, cu
   return TGRAD_OK;
 }
 
+// Omega <- the k entries of x with the largest selection keys (ascending), their values into the gather buffer.
+template <class S>
+tgrad_status select_omega(tgrad_state* s, const void* x, cudaStream_t st) {
+  const tgrad_config& c = s->cfg;
+  const Layout& L = s->L;
+  const uint32_t n = (uint32_t)L.numel, k = (uint32_t)c.k;
+  int* flags = reinterpret_cast<int*>(s->dp + L.p_flags);
+  uint32_t* omega = reinterpret_cast<uint32_t*>(s->dp + L.p_omega);
+  cf* g_s = reinterpret_cast<cf*>(s->dw + L.w_gs);
+  SelState* sel = reinterpret_cast<SelState*>(s->dw + L.w_sel);
+  uint32_t* hist = reinterpret_cast<uint32_t*>(s->dw + L.w_hist);
+  uint32_t* blk_gt = reinterpret_cast<uint32_t*>(s->dw + L.w_blk);
+  uint32_t* blk_eq = blk_gt + L.nblk;
+  SelKey kp;
+  kp.seed_lo = (uint32_t)(c.seed & 0xffffffffull); kp.seed_hi = (uint32_t)(c.seed >> 32);
+  kp.epoch = (uint32_t)(s->t / c.T); kp.strategy = c.sparse_strategy;
+  if (cudaMemsetAsync(hist, 0, 3 * kSelMaxBins * 4, st) != cudaSuccess) return TGRAD_ERR_CUDA;
+  sel_init_kernel<<<1, 1, 0, st>>>(sel, k); TG_LAUNCH_CHECK();
+  uint64_t want = ((uint64_t)n + 511) / 512;
+  int hgrid = (int)(want < (uint64_t)s->sm_count * 8 ? want : (uint64_t)s->sm_count * 8);
+  for (int pass = 0; pass < 3; ++pass) {
+    sel_hist_kernel<S><<<hgrid, 512, 0, st>>>(x, n, pass, sel, hist + pass * kSelMaxBins, flags, kp);
+    TG_LAUNCH_CHECK();
+    sel_pick_kernel<<<1, 1024, 0, st>>>(hist + pass * kSelMaxBins, pass, sel); TG_LAUNCH_CHECK();
+  }
+  sel_count_kernel<S><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, kp); TG_LAUNCH_CHECK();
+  sel_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, L.nblk); TG_LAUNCH_CHECK();
+  sel_compact_kernel<S><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, omega, g_s, k, kp);
+  TG_LAUNCH_CHECK();
+  return TGRAD_OK;
+}
+
+// ---- pieces of a step, shared with the refresh of the low-rank-first composition ----
+
+// Geometry, factor and index pointers and the update scalars of the two streaming kernels.
+TailParams tail_params(const tgrad_state* s) {
+  const tgrad_config& c = s->cfg;
+  const Layout& L = s->L;
+  const int N = c.ndim;
+  const int A = (int)c.dims[N - 2], B = (int)c.dims[N - 1], ra = c.ranks[N - 2], rb = c.ranks[N - 1];
+  TailParams p; memset(&p, 0, sizeof(p));
+  p.A = A; p.B = B; p.Bs = B | 1; p.ra = ra; p.rb = rb; p.ras = ra | 1;
+  p.E = (uint32_t)((uint64_t)A * B); p.nslab = (uint32_t)(L.numel / p.E);
+  p.Ua = reinterpret_cast<const cf*>(s->dp + L.p_factor[N - 2]);
+  p.Ub = reinterpret_cast<const cf*>(s->dp + L.p_factor[N - 1]);
+  p.omega = reinterpret_cast<const uint32_t*>(s->dp + L.p_omega);
+  p.slab_ptr = reinterpret_cast<const uint32_t*>(s->dp + L.p_slab);
+  p.k = (int)c.k;
+  p.m_s = reinterpret_cast<cf*>(s->dp + L.p_ms);
+  p.v_s = reinterpret_cast<float*>(s->dp + L.p_vs);
+  p.n_s = reinterpret_cast<cf*>(s->dw + L.w_ns);
+  p.g_s = reinterpret_cast<cf*>(s->dw + L.w_gs);
+  p.s_low = (float)((double)c.lr * (double)c.alpha);
+  p.s_sparse = (float)((double)c.lr * (double)c.lambda);
+  p.decay = (float)(1.0 - (double)c.lr * (double)c.weight_decay);
+  return p;
+}
+
+// Compression of the two trailing modes of the tensor at d_grad into p.t, with the sparse gather if p.k > 0.
+tgrad_status run_proj_tail(tgrad_state* s, const void* d_grad, const TailParams& p, cudaStream_t st) {
+  const Layout& L = s->L;
+  int* flags = reinterpret_cast<int*>(s->dp + L.p_flags);
+  if (s->tail.tc) {
+    TailTcParams mp; mp.flags = flags; mp.s_sparse_pre = 0.f;
+    mp.p = p; mp.g = s->tail.gproj;
+    float4* tab = reinterpret_cast<float4*>(s->dp + L.p_u2tab);
+    if (s->tabs_stale) {
+      const int n_ent = (p.A / 8) * s->tail.rat * 32;
+      proj_u2tab_kernel<<<(n_ent + 127) / 128, 128, 0, st>>>(p.Ua, p.A, p.ra, s->tail.rat, tab);
+      TG_LAUNCH_CHECK();
+      s->tabs_stale = false;
+    }
+    mp.u2tab = tab;
+    return tc_dispatch(1, s->tail, const_cast<void*>(d_grad), mp, st);
+  }
+  if (s->tail.th) {
+    TailHParams hp; hp.p = p; hp.g = s->tail.gh; hp.flags = flags;
+    return th_dispatch(1, s->tail, d_grad, hp, st);
+  }
+  return tail_any(s, 1, const_cast<void*>(d_grad), p, st);
+}
+
+// Reconstruction of the two trailing modes from p.t, fused with the update of the tensor at d_weight:
+// W <- decay W - s_low D, then W[Omega] -= s_sparse N_S if p.k > 0.
+tgrad_status run_back_tail(tgrad_state* s, void* d_weight, const TailParams& p, cudaStream_t st) {
+  int* flags = reinterpret_cast<int*>(s->dp + s->L.p_flags);
+  if (s->tail.tc) {
+    TailTcParams mp; mp.flags = flags; mp.u2tab = nullptr;
+    const tgrad_config& c = s->cfg;
+    mp.s_sparse_pre = (float)((double)c.lr * (double)c.lambda / (1.0 - (double)c.lr * (double)c.weight_decay));
+    mp.p = p; mp.g = s->tail.gback;
+    return tc_dispatch(2, s->tail, d_weight, mp, st);
+  }
+  if (s->tail.thb) {
+    TailHBParams hp; hp.p = p; hp.g = s->tail.ghb; hp.flags = flags;
+    return thb_dispatch(2, s->tail, d_weight, hp, st);
+  }
+  return tail_any(s, 2, d_weight, p, st);
+}
+
+// Whether the first mode's two products and the AdamUpdate of the core run as one launch.
+bool chain_fused(const tgrad_config& c) {
+  const int N = c.ndim;
+  uint64_t c_first = (uint64_t)c.ranks[N - 2] * c.ranks[N - 1];
+  for (int q = 1; q <= N - 3; ++q) c_first *= c.ranks[q];
+  return c.dims[0] <= SW_MAX_I && c.ranks[0] <= SW_MAX_R &&
+         c_first * (uint64_t)c.dims[0] * (uint64_t)c.ranks[0] <= ((uint64_t)64 << 20);
+}
+
+// Compression of modes N-2 .. last (last = 1: the first mode is left for the fused launch; last = 0: down to the
+// core, which lands in the core buffer), starting from the tail-contracted tensor in the first chain buffer.
+// *out = where the result is, *Cout = its trailing extent.
+tgrad_status compress_chain(tgrad_state* s, int last, cf** out, uint64_t* Cout, cudaStream_t st) {
+  const tgrad_config& c = s->cfg;
+  const Layout& L = s->L;
+  const int N = c.ndim;
+  cf* cur = reinterpret_cast<cf*>(s->dw + L.w_bufa);
+  cf* nxt = reinterpret_cast<cf*>(s->dw + L.w_bufb);
+  cf* core = reinterpret_cast<cf*>(s->dw + L.w_core);
+  uint64_t C = (uint64_t)c.ranks[N - 2] * c.ranks[N - 1];
+  for (int m = N - 3; m >= last; --m) {
+    uint64_t O = 1;
+    for (int q = 0; q < m; ++q) O *= c.dims[q];
+    cf* dst = (m == 0) ? core : nxt;
+    TG_TRY(mode_product(true, cur, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[m]), O, c.ranks[m],
+                        (int)c.dims[m], C, c.ranks[m], s->sm_count, st));
+    C *= c.ranks[m];
+    if (m == 0) { cur = core; break; }
+    cf* tmp = cur; cur = nxt; nxt = tmp;
+  }
+  *out = cur; *Cout = C;
+  return TGRAD_OK;
+}
+
+// Reconstruction of modes mfirst .. N-3 (mfirst = 0 from a core-shaped tensor, 1 after the fused launch) into the
+// chain buffers, alternating from buffer `which`; *out = the tensor [I_1 .. I_{N-2}][r_{N-1}][r_N].
+tgrad_status expand_chain(tgrad_state* s, const cf* src, int mfirst, int which, const cf** out, cudaStream_t st) {
+  const tgrad_config& c = s->cfg;
+  const Layout& L = s->L;
+  const int N = c.ndim;
+  cf* bufs[2] = {reinterpret_cast<cf*>(s->dw + L.w_bufa), reinterpret_cast<cf*>(s->dw + L.w_bufb)};
+  uint64_t O = 1;
+  for (int q = 0; q < mfirst; ++q) O *= c.dims[q];
+  for (int m = mfirst; m <= N - 3; ++m) {
+    uint64_t Cm = (uint64_t)c.ranks[N - 2] * c.ranks[N - 1];
+    for (int q = m + 1; q <= N - 3; ++q) Cm *= c.ranks[q];
+    cf* dst = bufs[which];
+    TG_TRY(mode_product(false, src, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[m]), O, (int)c.dims[m],
+                        c.ranks[m], Cm, c.ranks[m], s->sm_count, st));
+    O *= c.dims[m];
+    src = dst; which ^= 1;
+  }
+  *out = src;
+  return TGRAD_OK;
+}
+
+// g_s[j] -= P_U(G)[Omega[j]], with P_U(G) given down to the two trailing modes: t[slab][ja][jb].
+__global__ void lowrank_at_omega_kernel(cf* __restrict__ g_s, const uint32_t* __restrict__ omega, uint32_t k,
+                                        const cf* __restrict__ t, const cf* __restrict__ Ua, const cf* __restrict__ Ub,
+                                        int A, int B, int ra, int rb, uint32_t E) {
+  const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= k) return;
+  const uint32_t w = omega[j], slab = w / E, loc = w - slab * E;
+  const int a = (int)(loc / (uint32_t)B), b = (int)(loc - (uint32_t)a * (uint32_t)B);
+  const cf* ts = t + (size_t)slab * ra * rb;
+  cf acc = make_float2(0.f, 0.f);
+  for (int ja = 0; ja < ra; ++ja) {
+    cf row = make_float2(0.f, 0.f);
+    for (int jb = 0; jb < rb; ++jb) cfma(row, ts[ja * rb + jb], Ub[b * rb + jb]);
+    cfma(acc, row, Ua[a * ra + ja]);
+  }
+  cf v = g_s[j];
+  v.x -= acc.x; v.y -= acc.y;
+  g_s[j] = v;
+}
+
 __global__ void identity_kernel(cf* __restrict__ m, int n) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx < n * n) m[idx] = make_float2((idx / n) == (idx % n) ? 1.f : 0.f, 0.f);
@@ -626,29 +806,15 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   int* flags = reinterpret_cast<int*>(s->dp + L.p_flags);
   uint32_t* omega = reinterpret_cast<uint32_t*>(s->dp + L.p_omega);
   cf* g_s = reinterpret_cast<cf*>(s->dw + L.w_gs);
-  if (k > 0) {
-    SelState* sel = reinterpret_cast<SelState*>(s->dw + L.w_sel);
-    uint32_t* hist = reinterpret_cast<uint32_t*>(s->dw + L.w_hist);
-    uint32_t* blk_gt = reinterpret_cast<uint32_t*>(s->dw + L.w_blk);
-    uint32_t* blk_eq = blk_gt + L.nblk;
-    if (cudaMemsetAsync(hist, 0, 3 * kSelMaxBins * 4, st) != cudaSuccess) return TGRAD_ERR_CUDA;
-    sel_init_kernel<<<1, 1, 0, st>>>(sel, k); TG_LAUNCH_CHECK();
-    uint64_t want = ((uint64_t)n + 511) / 512;
-    int hgrid = (int)(want < (uint64_t)s->sm_count * 8 ? want : (uint64_t)s->sm_count * 8);
-    for (int pass = 0; pass < 3; ++pass) {
-      sel_hist_kernel<S><<<hgrid, 512, 0, st>>>(d_grad, n, pass, sel, hist + pass * kSelMaxBins, flags);
-      TG_LAUNCH_CHECK();
-      sel_pick_kernel<<<1, 1024, 0, st>>>(hist + pass * kSelMaxBins, pass, sel); TG_LAUNCH_CHECK();
+  const int comp = c.composition;
+  // Algorithm 1's order and the additive composition select Omega from the gradient; the former then hands the
+  // residual (entries at Omega zeroed in place, put back below) to the low-rank part
+  if (comp != 1) {
+    if (k > 0) {
+      TG_TRY(select_omega<S>(s, d_grad, st));
+      if (comp == 0) { scatter_zero_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, k); TG_LAUNCH_CHECK(); }
     }
-    sel_count_kernel<S><<<L.nblk, kChunkThreads, 0, st>>>(d_grad, n, sel, blk_gt, blk_eq); TG_LAUNCH_CHECK();
-    sel_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, L.nblk); TG_LAUNCH_CHECK();
-    sel_compact_kernel<S><<<L.nblk, kChunkThreads, 0, st>>>(d_grad, n, sel, blk_gt, blk_eq, omega, g_s, k);
-    TG_LAUNCH_CHECK();
-    scatter_zero_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, k); TG_LAUNCH_CHECK();
-  }
-  {
-    tgrad_status r = build_slab_ptr(s, st);
-    if (r != TGRAD_OK) return r;
+    TG_TRY(build_slab_ptr(s, st));
   }
   // ---- factor matrices ----
   // Starting factors: the leading eigenvectors of the mode-n Gram matrices of the residual (truncated SVDs of the
@@ -671,7 +837,27 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   // with the current factors and take the leading eigenvectors of the mode-n Gram matrix of the result.
   for (int it = 0; it < c.hooi_iters; ++it)
     for (int m = 0; m < N; ++m) TG_TRY(hooi_mode_update<S>(s, m, d_grad, st));
-  if (k > 0) { scatter_restore_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, g_s, k); TG_LAUNCH_CHECK(); }
+  if (k > 0 && comp == 0) { scatter_restore_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, g_s, k); TG_LAUNCH_CHECK(); }
+  if (comp == 1) {
+    // low rank first: R = G - P_U(G) in a buffer of its own (compression of G down to the core, reconstruction down
+    // to the trailing modes, last two modes fused with the subtraction from a copy of G), Omega from R
+    s->tabs_stale = true;                                    // the factors have just changed
+    TailParams p = tail_params(s);
+    p.k = 0; p.keep = 1;
+    p.t = reinterpret_cast<cf*>(s->dw + L.w_bufa);
+    TG_TRY(run_proj_tail(s, d_grad, p, st));
+    cf* cur; uint64_t Cc;
+    TG_TRY(compress_chain(s, 0, &cur, &Cc, st));
+    const cf* tcore;
+    TG_TRY(expand_chain(s, cur, 0, ((N - 2) & 1) ? 0 : 1, &tcore, st));
+    void* rbuf = s->dw + L.w_rbuf;
+    if (cudaMemcpyAsync(rbuf, d_grad, (size_t)L.numel * S::kBytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return TGRAD_ERR_CUDA;
+    p.t = const_cast<cf*>(tcore);
+    p.s_low = 1.0f; p.s_sparse = 0.f; p.decay = 1.0f;
+    TG_TRY(run_back_tail(s, rbuf, p, st));
+    if (k > 0) TG_TRY(select_omega<S>(s, rbuf, st));
+    TG_TRY(build_slab_ptr(s, st));
+  }
   s->have_subspace = true;
   s->tabs_stale = true;
   s->basis_valid = true;
@@ -722,120 +908,64 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
   if (!s->have_subspace) return TGRAD_ERR_BAD_STATE;
   cudaEvent_t* evs = s->timing ? s->ev[s->timing_steps % kTimingRing] : nullptr;
 
-  const int A = (int)c.dims[N - 2], B = (int)c.dims[N - 1], ra = c.ranks[N - 2], rb = c.ranks[N - 1];
-  TailParams p; memset(&p, 0, sizeof(p));
-  p.A = A; p.B = B; p.Bs = B | 1; p.ra = ra; p.rb = rb; p.ras = ra | 1;
-  p.E = (uint32_t)((uint64_t)A * B); p.nslab = (uint32_t)(L.numel / p.E);
-  p.Ua = reinterpret_cast<const cf*>(s->dp + L.p_factor[N - 2]);
-  p.Ub = reinterpret_cast<const cf*>(s->dp + L.p_factor[N - 1]);
-  p.omega = reinterpret_cast<const uint32_t*>(s->dp + L.p_omega);
-  p.slab_ptr = reinterpret_cast<const uint32_t*>(s->dp + L.p_slab);
-  p.k = (int)c.k;
-  p.m_s = reinterpret_cast<cf*>(s->dp + L.p_ms);
-  p.v_s = reinterpret_cast<float*>(s->dp + L.p_vs);
-  p.n_s = reinterpret_cast<cf*>(s->dw + L.w_ns);
-  p.g_s = reinterpret_cast<cf*>(s->dw + L.w_gs);
+  TailParams p = tail_params(s);
   p.adam = adam_scalars(c, s->t);
-  p.s_low = (float)((double)c.lr * (double)c.alpha);
-  p.s_sparse = (float)((double)c.lr * (double)c.lambda);
-  p.decay = (float)(1.0 - (double)c.lr * (double)c.weight_decay);
+  p.keep = c.composition != 0;          // only Algorithm 1's order feeds the low-rank part with the sparse part's residual
   cf* bufa = reinterpret_cast<cf*>(s->dw + L.w_bufa);
-  cf* bufb = reinterpret_cast<cf*>(s->dw + L.w_bufb);
   cf* core = reinterpret_cast<cf*>(s->dw + L.w_core);
   cf* n_l = reinterpret_cast<cf*>(s->dw + L.w_nl);
+  const uint32_t ks = (uint32_t)c.k;
+  const bool lr_first = c.composition == 1;
 
-  // low-rank compression: trailing two modes while streaming G, then modes N-2 .. 1
+  // low-rank compression: trailing two modes while streaming G (with the sparse gather), then modes N-2 .. 1
   TG_MARK(0);
   p.t = bufa;
-  TailTcParams mp;
-  mp.flags = reinterpret_cast<int*>(s->dp + L.p_flags);
-  mp.s_sparse_pre = (float)((double)c.lr * (double)c.lambda / (1.0 - (double)c.lr * (double)c.weight_decay));
-  if (s->tail.tc) {
-    mp.p = p; mp.g = s->tail.gproj;
-    float4* tab = reinterpret_cast<float4*>(s->dp + L.p_u2tab);
-    if (s->tabs_stale) {
-      const int n_ent = (A / 8) * s->tail.rat * 32;
-      proj_u2tab_kernel<<<(n_ent + 127) / 128, 128, 0, st>>>(p.Ua, A, ra, s->tail.rat, tab);
-      TG_LAUNCH_CHECK();
-      s->tabs_stale = false;
-    }
-    mp.u2tab = tab;
-    TG_TRY(tc_dispatch(1, s->tail, d_grad, mp, st));
-  } else if (s->tail.th) {
-    TailHParams hp; hp.p = p; hp.g = s->tail.gh; hp.flags = mp.flags;
-    TG_TRY(th_dispatch(1, s->tail, d_grad, hp, st));
-  } else {
-    TG_TRY(tail_any(s, 1, d_grad, p, st));
-  }
+  TG_TRY(run_proj_tail(s, d_grad, p, st));
   TG_MARK(1);
   // the chain on the small tensor: compression of modes N-2 .. 2, then mode 1 + Adam + mode 1 in one
   // launch (or three when the first mode is too large for it), then reconstruction of modes 2 .. N-2
   // (the fused launch holds all of U^(1) and a 16-column block in shared memory and serialises its two products:
   //  beyond 64 M complex multiply-adds per product separate GEMM launches win even with the extra round trips)
-  uint64_t c_first = (uint64_t)ra * rb;
-  for (int q = 1; q <= N - 3; ++q) c_first *= c.ranks[q];
-  const bool fused = c.dims[0] <= SW_MAX_I && c.ranks[0] <= SW_MAX_R &&
-                     c_first * (uint64_t)c.dims[0] * (uint64_t)c.ranks[0] <= ((uint64_t)64 << 20);
+  const bool fused = !lr_first && chain_fused(c);
   const cf* tprime;
   {
-    cf* cur = bufa; cf* nxt = bufb;
-    uint64_t C = (uint64_t)ra * rb;
-    for (int m = N - 3; m >= (fused ? 1 : 0); --m) {
-      uint64_t O = 1;
-      for (int q = 0; q < m; ++q) O *= c.dims[q];
-      cf* dst = (m == 0) ? core : nxt;
-      TG_TRY(mode_product(true, cur, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[m]), O, c.ranks[m],
-                          (int)c.dims[m], C, c.ranks[m], s->sm_count, st));
-      C *= c.ranks[m];
-      cf* tmp = cur; cur = nxt; nxt = tmp;
-    }
+    cf* cur; uint64_t C;
+    TG_TRY(compress_chain(s, fused ? 1 : 0, &cur, &C, st));
     TG_MARK(2);
-    cf* bufs[2] = {bufa, bufb};
-    int which = ((N - 2) & 1) ? 0 : 1;          // make the last product land in bufa
-    const uint32_t ks = (uint32_t)c.k;
-    const cf* src;
-    int mfirst;
+    int which = ((N - 2) & 1) ? 0 : 1;          // make the last product land in the first buffer
     if (fused) {
       // here cur holds [I_1][C] with C = r_2 .. r_N
+      cf* bufs[2] = {bufa, reinterpret_cast<cf*>(s->dw + L.w_bufb)};
       cf* dst = bufs[which];
       const uint32_t nblk_core = (uint32_t)((C + SW_CB - 1) / SW_CB), nblk_sparse = (ks + SW_THREADS - 1) / SW_THREADS;
-      launch_chained(core_sandwich_tc_kernel, dim3(nblk_core + nblk_sparse), dim3(SW_THREADS), sandwich_tc_smem((int)c.dims[0], c.ranks[0]), st, 
+      launch_chained(core_sandwich_tc_kernel, dim3(nblk_core + nblk_sparse), dim3(SW_THREADS), sandwich_tc_smem((int)c.dims[0], c.ranks[0]), st,
           cur, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[0]), core, reinterpret_cast<cf*>(s->dp + L.p_ml),
           reinterpret_cast<float*>(s->dp + L.p_vl), n_l, (int)c.dims[0], c.ranks[0], (int)C, p.g_s, p.m_s, p.v_s, p.n_s, ks,
           nblk_core, p.adam);
       TG_LAUNCH_CHECK();
-      src = dst; which ^= 1; mfirst = 1;
+      which ^= 1;
+      TG_MARK(3);
+      TG_TRY(expand_chain(s, dst, 1, which, &tprime, st));
     } else {
-      launch_chained(adam_kernel, dim3((unsigned)((L.P + ks + 255) / 256)), dim3(256), 0, st, 
+      if (lr_first && ks > 0) {
+        // the sparse values are those of G - P_U(G): rebuild the low-rank approximation from the core down to the
+        // trailing two modes and subtract its entries at Omega from the gathered ones
+        const cf* tcore;
+        TG_TRY(expand_chain(s, core, 0, which, &tcore, st));
+        lowrank_at_omega_kernel<<<(ks + 127) / 128, 128, 0, st>>>(p.g_s, p.omega, ks, tcore, p.Ua, p.Ub, p.A, p.B, p.ra, p.rb, p.E);
+        TG_LAUNCH_CHECK();
+      }
+      launch_chained(adam_kernel, dim3((unsigned)((L.P + ks + 255) / 256)), dim3(256), 0, st,
           core, reinterpret_cast<cf*>(s->dp + L.p_ml), reinterpret_cast<float*>(s->dp + L.p_vl), n_l, (uint32_t)L.P,
           p.g_s, p.m_s, p.v_s, p.n_s, ks, p.adam);
       TG_LAUNCH_CHECK();
-      src = n_l; mfirst = 0;
+      TG_MARK(3);
+      TG_TRY(expand_chain(s, n_l, 0, which, &tprime, st));
     }
-    TG_MARK(3);
-    uint64_t O = fused ? (uint64_t)c.dims[0] : 1;
-    for (int m = mfirst; m <= N - 3; ++m) {
-      uint64_t Cm = (uint64_t)ra * rb;
-      for (int q = m + 1; q <= N - 3; ++q) Cm *= c.ranks[q];
-      cf* dst = bufs[which];
-      TG_TRY(mode_product(false, src, dst, reinterpret_cast<const cf*>(s->dp + L.p_factor[m]), O, (int)c.dims[m],
-                          c.ranks[m], Cm, c.ranks[m], s->sm_count, st));
-      O *= c.dims[m];
-      src = dst; which ^= 1;
-    }
-    tprime = src;
   }
   TG_MARK(4);
   p.t = const_cast<cf*>(tprime);
-  if (s->tail.tc) {
-    mp.p = p; mp.g = s->tail.gback;
-    TG_TRY(tc_dispatch(2, s->tail, d_weight, mp, st));
-  } else if (s->tail.thb) {
-    TailHBParams hp; hp.p = p; hp.g = s->tail.ghb; hp.flags = mp.flags;
-    TG_TRY(thb_dispatch(2, s->tail, d_weight, hp, st));
-  } else {
-    TG_TRY(tail_any(s, 2, d_weight, p, st));
-  }
+  TG_TRY(run_back_tail(s, d_weight, p, st));
   TG_MARK(5);
   if (s->timing) s->timing_steps++;
   s->t += 1;
@@ -1144,6 +1274,7 @@ template <class S>
 tgrad_status select_noalloc_impl(const void* d_grad, uint32_t n, uint32_t k, uint32_t* d_omega, cf* d_values,
                                  NoAllocScratch* sc, int sm, cudaStream_t st) {
   const uint32_t nblk = (n + kChunk - 1) / kChunk;
+  SelKey kp; kp.seed_lo = kp.seed_hi = kp.epoch = 0u; kp.strategy = 0;     // magnitude top-k
   uint32_t* blk_gt = sc->blk;
   uint32_t* blk_eq = sc->blk + nblk;
   // the histograms and the flag word must start at zero; everything else is overwritten before it is read
@@ -1152,13 +1283,13 @@ tgrad_status select_noalloc_impl(const void* d_grad, uint32_t n, uint32_t k, uin
   const uint64_t want = ((uint64_t)n + 511) / 512;
   const int hgrid = (int)(want < (uint64_t)sm * 8 ? want : (uint64_t)sm * 8);
   for (int pass = 0; pass < 3; ++pass) {
-    sel_hist_kernel<S><<<hgrid, 512, 0, st>>>(d_grad, n, pass, &sc->sel, sc->hist + pass * kSelMaxBins, sc->flags);
+    sel_hist_kernel<S><<<hgrid, 512, 0, st>>>(d_grad, n, pass, &sc->sel, sc->hist + pass * kSelMaxBins, sc->flags, kp);
     TG_LAUNCH_CHECK();
     sel_pick_kernel<<<1, 1024, 0, st>>>(sc->hist + pass * kSelMaxBins, pass, &sc->sel); TG_LAUNCH_CHECK();
   }
-  sel_count_kernel<S><<<nblk, kChunkThreads, 0, st>>>(d_grad, n, &sc->sel, blk_gt, blk_eq); TG_LAUNCH_CHECK();
+  sel_count_kernel<S><<<nblk, kChunkThreads, 0, st>>>(d_grad, n, &sc->sel, blk_gt, blk_eq, kp); TG_LAUNCH_CHECK();
   sel_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, nblk); TG_LAUNCH_CHECK();
-  sel_compact_kernel<S><<<nblk, kChunkThreads, 0, st>>>(d_grad, n, &sc->sel, blk_gt, blk_eq, d_omega, d_values, k);
+  sel_compact_kernel<S><<<nblk, kChunkThreads, 0, st>>>(d_grad, n, &sc->sel, blk_gt, blk_eq, d_omega, d_values, k, kp);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }

@@ -70,6 +70,36 @@ def test_hooi_refinement(name, warm):
     print("hooi", name, p.report.get("angle"), "moved", moved)
 
 
+@pytest.mark.parametrize("name", ["small4", "ragged4", "odd32"])
+@pytest.mark.parametrize("strategy", ["randk", "probk"])
+def test_random_sparsification_strategies(name, strategy):
+    # Omega from one Philox word per entry (uniform k-subset) or from |g| / exponential variate (sampling proportional
+    # to |g|): the same bits on both sides, so the sets are compared exactly, and they change from refresh to refresh
+    wl = synth.WORKLOADS[name]
+    p = Pair(wl, strategy=strategy, seed=0x1234567890ABCDEF)
+    sets = []
+    for t in range(2 * wl.T + 1):
+        p.step(t)
+        if t % wl.T == 0:
+            sets.append(p.gst.export(B.WHAT_OMEGA))
+    assert not np.array_equal(sets[0], sets[1]) and not np.array_equal(sets[1], sets[2])
+    if strategy == "randk":
+        assert not np.array_equal(sets[0], orc.sparse_indices_topk(p.src.gradient(0), wl.k))
+
+
+@pytest.mark.parametrize("name,half", [("small4", False), ("odd32", False), ("ragged4", True), ("small5b", False), ("mat2", False)])
+@pytest.mark.parametrize("composition", ["sum", "lr_us"])
+def test_other_compositions(name, half, composition):
+    # "sum": both parts see the gradient itself; "lr_us": the low-rank part goes first and the sparse part is chosen
+    # from, and fed with, G - P_U(G)
+    import dataclasses
+    wl = dataclasses.replace(synth.WORKLOADS[name], half_storage=half)
+    p = Pair(wl, composition=composition, stagewise_w=(name == "mat2"))
+    for t in range(wl.T + 2):
+        p.step(t)
+    print(composition, name, p.report.get("omega_boundary_entries"), p.report.get("core"), p.report.get("m_s"))
+
+
 def test_alpha_lambda_weight_decay():
     wl = synth.WORKLOADS["small4"]
     p = Pair(wl, alpha=0.25, lam=0.5, weight_decay=0.1, lr=1e-2)
