@@ -12,9 +12,10 @@
  *
  * Conventions
  *  - All tensors are dense, row-major (last index fastest).  TGRAD_C64 stores
- *    each entry as two fp32 (re, im); TGRAD_C32H as two IEEE fp16 (re, im)
- *    (the paper's mixed-precision recipe, Section 2.3: weights and gradients in
- *    half precision, every optimizer state in fp32).
+ *    each entry as two fp32 (re, im); TGRAD_C32H as two IEEE fp16 (re, im) and
+ *    TGRAD_C32B as two bfloat16 (the paper's mixed-precision recipe, Section 2.3:
+ *    weights and gradients in half precision, every optimizer state in fp32; the
+ *    paper does not name the 16-bit format).
  *  - The caller passes grad = d(phi)/dW.  Algorithm 1 is written for
  *    G = -grad and W <- W + eta*Gtilde(G); the library evaluates the same
  *    stages on grad and subtracts, which is bit-identical.
@@ -69,7 +70,8 @@ typedef enum {
 
 typedef enum {
   TGRAD_C64 = 0,   /* interleaved 2 x fp32 */
-  TGRAD_C32H = 1   /* interleaved 2 x IEEE fp16 */
+  TGRAD_C32H = 1,  /* interleaved 2 x IEEE fp16 */
+  TGRAD_C32B = 2   /* interleaved 2 x bfloat16 (general kernels only: no fp16 tensor-core fast path) */
 } tgrad_dtype;
 
 #define TGRAD_MAX_NDIM 8

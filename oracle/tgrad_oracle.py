@@ -324,6 +324,7 @@ class OracleConfig:
     eps: float = 1e-8
     weight_decay: float = 0.0
     half_storage: bool = False      # W and G live as fp16 (re, im) pairs
+    bf16_storage: bool = False      # ... or as bfloat16 pairs (the paper's recipe says "half precision" without naming the format)
     hooi_iters: int = 0             # refinement sweeps of TuckerFactors (0: truncated-SVD factors only)
     hooi_warm: bool = False         # refinement starts from the factors of the previous refresh when there are any
     strategy: str = "topk"          # topk | randk | probk (Section 2.2, sparsification strategies)
@@ -334,8 +335,24 @@ class OracleConfig:
                                     # composition"; the combination ablation)
 
 
-def _store_w(w: np.ndarray, half: bool) -> np.ndarray:
-    """Round a complex128 weight to its storage type and widen it back."""
+def round_to_bfloat16(x: np.ndarray) -> np.ndarray:
+    """float32 values rounded to bfloat16 (8 exponent bits, 7 explicit mantissa bits), nearest, ties to even,
+    returned as float32: the upper 16 bits of the fp32 pattern after adding half a unit of the last kept place
+    (one less on an even keeper)."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    bias = ((u >> np.uint64(16)) & np.uint64(1)) + np.uint64(0x7FFF)
+    r = ((u + bias) & np.uint64(0xFFFF0000)).astype(np.uint32)
+    return r.view(np.float32).reshape(np.shape(x))
+
+
+def _store_w(w: np.ndarray, half, bf16: bool = False) -> np.ndarray:
+    """Round a complex128 weight to its storage type and widen it back.  `half` may be the configuration."""
+    if isinstance(half, OracleConfig):
+        half, bf16 = half.half_storage, half.bf16_storage
+    if bf16:
+        re = round_to_bfloat16(w.real.astype(np.float32)).astype(np.float64)
+        im = round_to_bfloat16(w.imag.astype(np.float32)).astype(np.float64)
+        return re + 1j * im
     if half:
         re = w.real.astype(np.float16).astype(np.float64)
         im = w.imag.astype(np.float16).astype(np.float64)
@@ -374,7 +391,7 @@ def lowrank_residual(cfg: OracleConfig, grad: np.ndarray, factors) -> np.ndarray
     """G - P_U(G), P_U(G) = (G x_n U^(n)H) x_n U^(n), rounded to the storage type of the gradient: what the sparse
     part sees when the low-rank part goes first."""
     x = np.asarray(grad, dtype=np.complex128)
-    return _store_w(x - tucker_reconstruct(tucker_compress(x, factors), factors), cfg.half_storage).astype(np.complex64)
+    return _store_w(x - tucker_reconstruct(tucker_compress(x, factors), factors), cfg).astype(np.complex64)
 
 
 def oracle_refresh(st: OracleState, grad: np.ndarray) -> None:
@@ -410,10 +427,10 @@ def weight_update(cfg: OracleConfig, w: np.ndarray, n_l: np.ndarray, n_s: np.nda
     if wd != 0.0:
         wn = wn * (1.0 - lr * wd)
     d = tucker_reconstruct(n_l, factors)
-    wn = np.ascontiguousarray(_store_w(wn - (lr * al) * d, cfg.half_storage))
+    wn = np.ascontiguousarray(_store_w(wn - (lr * al) * d, cfg))
     flat = wn.reshape(-1)                          # a view of the contiguous array
     om = np.asarray(omega).astype(np.int64)
-    flat[om] = _store_w(flat[om] - (lr * la) * np.asarray(n_s, dtype=np.complex128), cfg.half_storage)
+    flat[om] = _store_w(flat[om] - (lr * la) * np.asarray(n_s, dtype=np.complex128), cfg)
     return wn.astype(np.complex64)
 
 

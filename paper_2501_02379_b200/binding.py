@@ -22,7 +22,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_BUFFER_TOO_SMALL, ERR_CUDA, ERR_NO_CON
 ERR_TOO_LARGE = 8
 NOALLOC_MAX_NUMEL = 1 << 26
 FLAG_NO_CONVERGE, FLAG_NONFINITE, FLAG_COPY_TIMEOUT = 1, 2, 4
-C64, C32H = 0, 1
+C64, C32H, C32B = 0, 1, 2
 COMPOSITIONS = {"us_lr": 0, "lr_us": 1, "sum": 2}
 STRATEGIES = {"topk": 0, "randk": 1, "probk": 2}
 WHAT_OMEGA, WHAT_M_L, WHAT_V_L, WHAT_M_S, WHAT_V_S, WHAT_CORE, WHAT_N_L, WHAT_N_S = 1, 2, 3, 4, 5, 6, 7, 8
@@ -117,7 +117,7 @@ def _check(s: int, where: str) -> None:
 
 def make_config(shape: Sequence[int], ranks: Sequence[int], k: int, T: int, lr: float = 1e-3, alpha: float = 1.0,
                 lam: float = 1.0, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
-                weight_decay: float = 0.0, half_storage: bool = False, auto_refresh: bool = True,
+                weight_decay: float = 0.0, half_storage: bool = False, bf16_storage: bool = False, auto_refresh: bool = True,
                 jacobi_max_sweeps: int = 0, jacobi_tol: float = 0.0, warm_refresh: bool = False,
                 hooi_iters: int = 0, composition: str = "us_lr", strategy: str = "topk", seed: int = 0) -> TgradConfig:
     if len(shape) > MAX_NDIM or len(shape) != len(ranks):
@@ -132,7 +132,7 @@ def make_config(shape: Sequence[int], ranks: Sequence[int], k: int, T: int, lr: 
     cfg.lr, cfg.alpha, cfg.lambda_ = lr, alpha, lam
     cfg.beta1, cfg.beta2, cfg.eps = beta1, beta2, eps
     cfg.weight_decay = weight_decay
-    cfg.wg_dtype = C32H if half_storage else C64
+    cfg.wg_dtype = C32B if bf16_storage else (C32H if half_storage else C64)
     cfg.auto_refresh = 1 if auto_refresh else 0
     cfg.jacobi_max_sweeps = jacobi_max_sweeps
     cfg.jacobi_tol = jacobi_tol

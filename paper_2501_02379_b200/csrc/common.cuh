@@ -1,5 +1,6 @@
 // Shared device helpers for the TensorGRaD step kernels (sm_100a).
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -20,21 +21,39 @@ __device__ __forceinline__ void cfma_conj(cf& acc, cf a, cf b) {
   acc.y = fmaf(a.y, b.x, acc.y); acc.y = fmaf(-a.x, b.y, acc.y);
 }
 
-// Storage adaptors for W and G: interleaved 2 x fp32 or 2 x fp16.
+// Storage adaptors for W and G: interleaved 2 x fp32, 2 x fp16 or 2 x bfloat16.  widen() is exact; narrow() rounds
+// to nearest even (the identity for fp32).
 struct StoreC64 {
   typedef float2 elem;
   static constexpr int kBytes = 8;
+  __device__ static __forceinline__ cf widen(const elem& e) { return e; }
+  __device__ static __forceinline__ cf narrow(cf v) { return v; }
   __device__ static __forceinline__ cf load(const void* p, size_t i) { return reinterpret_cast<const float2*>(p)[i]; }
   __device__ static __forceinline__ void store(void* p, size_t i, cf v) { reinterpret_cast<float2*>(p)[i] = v; }
 };
 struct StoreC32H {
   typedef __half2 elem;
   static constexpr int kBytes = 4;
+  __device__ static __forceinline__ cf widen(const elem& e) { return __half22float2(e); }
+  __device__ static __forceinline__ cf narrow(cf v) { return __half22float2(__floats2half2_rn(v.x, v.y)); }
   __device__ static __forceinline__ cf load(const void* p, size_t i) {
     return __half22float2(reinterpret_cast<const __half2*>(p)[i]);
   }
   __device__ static __forceinline__ void store(void* p, size_t i, cf v) {
     reinterpret_cast<__half2*>(p)[i] = __floats2half2_rn(v.x, v.y);
+  }
+};
+
+struct StoreC32B {
+  typedef __nv_bfloat162 elem;
+  static constexpr int kBytes = 4;
+  __device__ static __forceinline__ cf widen(const elem& e) { return __bfloat1622float2(e); }
+  __device__ static __forceinline__ cf narrow(cf v) { return __bfloat1622float2(__floats2bfloat162_rn(v.x, v.y)); }
+  __device__ static __forceinline__ cf load(const void* p, size_t i) {
+    return __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(p)[i]);
+  }
+  __device__ static __forceinline__ void store(void* p, size_t i, cf v) {
+    reinterpret_cast<__nv_bfloat162*>(p)[i] = __floats2bfloat162_rn(v.x, v.y);
   }
 };
 

@@ -39,8 +39,8 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
   const int ta = blockIdx.x / T, tb = blockIdx.x % T;
   if (ta > tb) return;
   extern __shared__ __align__(16) unsigned char gsm[];
-  // tiles hold the entries as they are stored (fp32 pairs, or fp16 pairs in one word): fp16 values are exact
-  // TF32 operands, so half storage needs neither rounding nor the split products
+  // tiles hold the entries as they are stored (fp32 pairs, or fp16 / bfloat16 pairs in one word): 16-bit values are
+  // exact TF32 operands, so 16-bit storage needs neither rounding nor the split products
   typedef typename S::elem Elem;
   typedef Elem Tile[GR_T][GR_LD];
   Tile* XA = reinterpret_cast<Tile*>(gsm);            // [2]
@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
     const Elem (*Xa)[GR_LD] = XA[st];
     const Elem (*XB)[GR_LD] = diag ? XA[st] : XBs[st];
     auto widen = [](const Elem& e) -> cf {
-      if constexpr (HALF) return __half22float2(e); else return e;
+      return S::widen(e);
     };
 #pragma unroll
     for (int ks = 0; ks < GR_KT / 4; ++ks) {

@@ -259,7 +259,7 @@ __global__ void __launch_bounds__(TB_THREADS) back_tail_blk_kernel(void* __restr
         const uint32_t a = loc / B;
         const uint32_t si = a * Bs + (loc - a * B);
         cf wv = ws[si];
-        if (S::kBytes == 4) wv = __half22float2(__floats2half2_rn(wv.x, wv.y));
+        wv = S::narrow(wv);
         const cf n = p.n_s[j];
         wv.x = fmaf(-p.s_sparse, n.x, wv.x); wv.y = fmaf(-p.s_sparse, n.y, wv.y);
         ws[si] = wv;

@@ -74,7 +74,7 @@ tgrad_status validate(const tgrad_config* c) {
   }
   if (c->k < 0 || (long double)c->k > tot) return TGRAD_ERR_INVALID_ARG;
   if (c->T < 1) return TGRAD_ERR_INVALID_ARG;
-  if (c->wg_dtype != TGRAD_C64 && c->wg_dtype != TGRAD_C32H) return TGRAD_ERR_INVALID_ARG;
+  if (c->wg_dtype != TGRAD_C64 && c->wg_dtype != TGRAD_C32H && c->wg_dtype != TGRAD_C32B) return TGRAD_ERR_INVALID_ARG;
   if (!(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f) || !(c->eps >= 0.f))
     return TGRAD_ERR_INVALID_ARG;
   if (c->jacobi_max_sweeps < 0 || c->jacobi_tol < 0.f) return TGRAD_ERR_INVALID_ARG;
@@ -265,8 +265,9 @@ tgrad_status tail_dispatch(int op, const TailPlan& tp, void* ptr, const TailPara
 }
 
 tgrad_status tail_any(const tgrad_state* s, int op, void* ptr, const TailParams& p, cudaStream_t st) {
-  return s->cfg.wg_dtype == TGRAD_C64 ? tail_dispatch<StoreC64>(op, s->tail, ptr, p, st)
-                                      : tail_dispatch<StoreC32H>(op, s->tail, ptr, p, st);
+  return s->cfg.wg_dtype == TGRAD_C64    ? tail_dispatch<StoreC64>(op, s->tail, ptr, p, st)
+         : s->cfg.wg_dtype == TGRAD_C32H ? tail_dispatch<StoreC32H>(op, s->tail, ptr, p, st)
+                                         : tail_dispatch<StoreC32B>(op, s->tail, ptr, p, st);
 }
 
 template <int RAT, int KS, int NTW, int TW>
@@ -865,7 +866,9 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
 }
 
 tgrad_status do_refresh(tgrad_state* s, void* d_grad, cudaStream_t st) {
-  return s->cfg.wg_dtype == TGRAD_C64 ? refresh_impl<StoreC64>(s, d_grad, st) : refresh_impl<StoreC32H>(s, d_grad, st);
+  return s->cfg.wg_dtype == TGRAD_C64    ? refresh_impl<StoreC64>(s, d_grad, st)
+         : s->cfg.wg_dtype == TGRAD_C32H ? refresh_impl<StoreC32H>(s, d_grad, st)
+                                         : refresh_impl<StoreC32B>(s, d_grad, st);
 }
 
 tgrad_status mode_product(bool conj_t, const cf* in, cf* out, const cf* U, uint64_t O, int M, int K, uint64_t C,
@@ -1032,6 +1035,8 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
     TG_GRAM_ATTR(StoreC64, true, false); TG_GRAM_ATTR(StoreC64, true, true);
     TG_GRAM_ATTR(StoreC32H, false, false); TG_GRAM_ATTR(StoreC32H, false, true);
     TG_GRAM_ATTR(StoreC32H, true, false); TG_GRAM_ATTR(StoreC32H, true, true);
+    TG_GRAM_ATTR(StoreC32B, false, false); TG_GRAM_ATTR(StoreC32B, false, true);
+    TG_GRAM_ATTR(StoreC32B, true, false); TG_GRAM_ATTR(StoreC32B, true, true);
 #undef TG_GRAM_ATTR
     if (!ok) { delete st; return TGRAD_ERR_CUDA; }
   }
@@ -1298,7 +1303,7 @@ tgrad_status select_noalloc_impl(const void* d_grad, uint32_t n, uint32_t k, uin
 extern "C" tgrad_status tgrad_select_topk_noalloc(const void* d_grad, int64_t numel, int64_t k, int32_t wg_dtype,
                                                   uint32_t* d_omega, void* d_values, void* cuda_stream) {
   if (numel < 1 || k < 0 || k > numel) return TGRAD_ERR_INVALID_ARG;
-  if (wg_dtype != TGRAD_C64 && wg_dtype != TGRAD_C32H) return TGRAD_ERR_INVALID_ARG;
+  if (wg_dtype != TGRAD_C64 && wg_dtype != TGRAD_C32H && wg_dtype != TGRAD_C32B) return TGRAD_ERR_INVALID_ARG;
   if ((uint64_t)numel > kNaMaxNumel) return TGRAD_ERR_TOO_LARGE;
   if (!d_grad || (k > 0 && (!d_omega || !d_values))) return TGRAD_ERR_INVALID_ARG;
   // the kernels read the gradient with vector loads and write index / value pairs: same rule as the other calls
@@ -1309,7 +1314,9 @@ extern "C" tgrad_status tgrad_select_topk_noalloc(const void* d_grad, int64_t nu
   tgrad_status r = noalloc_scratch(&sc, &sm);
   if (r != TGRAD_OK) return r;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  return wg_dtype == TGRAD_C64
-             ? select_noalloc_impl<StoreC64>(d_grad, (uint32_t)numel, (uint32_t)k, d_omega, static_cast<cf*>(d_values), sc, sm, st)
-             : select_noalloc_impl<StoreC32H>(d_grad, (uint32_t)numel, (uint32_t)k, d_omega, static_cast<cf*>(d_values), sc, sm, st);
+  if (wg_dtype == TGRAD_C64)
+    return select_noalloc_impl<StoreC64>(d_grad, (uint32_t)numel, (uint32_t)k, d_omega, static_cast<cf*>(d_values), sc, sm, st);
+  if (wg_dtype == TGRAD_C32H)
+    return select_noalloc_impl<StoreC32H>(d_grad, (uint32_t)numel, (uint32_t)k, d_omega, static_cast<cf*>(d_values), sc, sm, st);
+  return select_noalloc_impl<StoreC32B>(d_grad, (uint32_t)numel, (uint32_t)k, d_omega, static_cast<cf*>(d_values), sc, sm, st);
 }

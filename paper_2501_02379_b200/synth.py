@@ -51,6 +51,7 @@ class Workload:
     noise: str = "normal"             # normal | student_t2 | laplace
     noise_scale: float = 0.0          # std (normal), scale b (laplace), x sigma_sig (student)
     half_storage: bool = False        # W, G stored as interleaved fp16 pairs
+    bf16_storage: bool = False        # ... or as interleaved bfloat16 pairs
     lr: float = 1e-3
 
     @property
@@ -240,6 +241,18 @@ def to_half_pairs(x: np.ndarray) -> np.ndarray:
 def from_half_pairs(h: np.ndarray) -> np.ndarray:
     """interleaved fp16 pairs (..., 2) -> complex64 (exact widening)."""
     return np.ascontiguousarray(h.astype(np.float32)).view(np.complex64)[..., 0]
+
+
+def to_bf16_pairs(x: np.ndarray) -> np.ndarray:
+    """complex64 -> interleaved bfloat16 (re, im) pairs as uint16 bit patterns, shape (..., 2); nearest, ties to even."""
+    u = np.ascontiguousarray(x).view(np.float32).reshape(x.shape + (2,)).view(np.uint32).astype(np.uint64)
+    bias = ((u >> np.uint64(16)) & np.uint64(1)) + np.uint64(0x7FFF)
+    return ((u + bias) >> np.uint64(16)).astype(np.uint16)
+
+
+def from_bf16_pairs(b: np.ndarray) -> np.ndarray:
+    """interleaved bfloat16 bit patterns (..., 2) -> complex64 (exact widening)."""
+    return np.ascontiguousarray((b.astype(np.uint32) << np.uint32(16)).view(np.float32)).view(np.complex64)[..., 0]
 
 
 def quantised_ties(shape, levels: int, seed: int) -> np.ndarray:

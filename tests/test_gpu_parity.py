@@ -180,6 +180,17 @@ def test_half_storage_small(name):
     print("half", name, p.report)
 
 
+@pytest.mark.parametrize("name", ["ragged4", "odd32", "small3"])
+def test_bf16_storage_small(name):
+    # bfloat16-stored W and G (the other reading of the mixed recipe's "half precision"): general kernels
+    import dataclasses
+    wl = dataclasses.replace(synth.WORKLOADS[name], bf16_storage=True)
+    p = Pair(wl)
+    for t in range(wl.T + 2):
+        p.step(t)
+    print("bf16", name, p.report)
+
+
 def test_auto_refresh_matches_explicit():
     wl = synth.WORKLOADS["small4"]
     src = synth.GradientSource(wl)

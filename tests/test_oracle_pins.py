@@ -608,6 +608,17 @@ def test_composition_lr_us_takes_the_sparse_part_from_the_lowrank_residual():
     assert np.max(np.abs(wa.reshape(-1)[mask] - wb.reshape(-1)[mask])) < 1e-6
 
 
+def test_bfloat16_rounding_matches_torch():
+    x = (np.random.default_rng(50).standard_normal(50000) * 3.7).astype(np.float32)
+    x[:4] = [1 + 2.0 ** -8, 1 + 2.0 ** -8 + 2.0 ** -20, 1 + 3 * 2.0 ** -8, -1 - 2.0 ** -8]     # ties go to even
+    want = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+    assert np.array_equal(orc.round_to_bfloat16(x), want)
+    assert orc.round_to_bfloat16(x)[:4].tolist() == [1.0, 1.0078125, 1.015625, -1.0]
+    cfg = orc.OracleConfig(shape=(2,), ranks=(1,), k=0, T=1, bf16_storage=True)
+    w = orc._store_w(np.array([1 + 2.0 ** -9 + 1j * (1 + 2.0 ** -6)]), cfg)
+    assert w[0] == complex(1.0, 1 + 2.0 ** -6)
+
+
 # ---- state size: the paper's worked example --------------------------------------------------
 
 def test_state_size_matches_paper_example():
