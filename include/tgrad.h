@@ -20,8 +20,8 @@
  *    G = -grad and W <- W + eta*Gtilde(G); the library evaluates the same
  *    stages on grad and subtracts, which is bit-identical.
  *  - Pointers named d_* are DEVICE pointers, everything else is host memory.
- *  - The library never allocates or frees device memory and never creates
- *    streams.  The caller owns: the weight, the gradient, one persistent
+ *  - The library never allocates or frees device memory and, but for the
+ *    side streams of tgrad_step_batched, never creates streams.  The caller owns: the weight, the gradient, one persistent
  *    block (Omega, U^(n), moments, status words, a split copy of U^(N-1)
  *    laid out for the compression kernel) and one workspace block
  *    (scratch; contents need not survive between calls, but the same
@@ -188,7 +188,13 @@ tgrad_status tgrad_refresh_subspace(tgrad_state* st, void* d_grad, void* cuda_st
 
 /* Batched variants over a list of layers: semantically n independent calls
  * (the tensors of an FNO's spectral layers are independent).  Arrays are HOST
- * arrays of handles / device pointers. */
+ * arrays of handles / device pointers.
+ * tgrad_step_batched runs the tensors' kernel chains side by side: it forks
+ * them onto up to four streams that the library creates per device at the
+ * first batched call (the one exception to "creates no streams") and joins
+ * them back into the given stream, so for the caller the call orders like
+ * any other work on that stream.  The states must have distinct workspaces,
+ * and d_weights / d_grads must not overlap between tensors. */
 tgrad_status tgrad_step_batched(tgrad_state* const* states, void* const* d_weights, void* const* d_grads,
                                 int32_t n_tensors, void* cuda_stream);
 tgrad_status tgrad_refresh_subspace_batched(tgrad_state* const* states, void* const* d_grads, int32_t n_tensors,
@@ -207,6 +213,15 @@ tgrad_status tgrad_export_state(tgrad_state* st, int32_t what, void* host_dst, s
 tgrad_status tgrad_import_state(tgrad_state* st, int32_t what, const void* host_src, size_t bytes,
                                 void* cuda_stream);
 tgrad_status tgrad_set_step(tgrad_state* st, int64_t t);
+
+/* Optional diagnostics of the last step, not part of the timed path (synchronises the stream).  d_grad must be the
+ * gradient that step was given.  out[0] = ||G||_F;  out[1] = ||G_S||_F / ||G||_F, the share of the gradient the
+ * sparse part took;  out[2] = || X - P_U X ||_F / ||G||_F, the part the low-rank compression lost, X being what the
+ * low-rank part was given (the residual of the sparse part in Algorithm 1's order, the gradient otherwise) -- with
+ * orthonormal factors this is sqrt(||X||^2 - ||core||^2), the reconstruction error Section 2.2 reports for its
+ * decompositions;  out[3] = max over modes and entries of |U^(n)H U^(n) - I|.
+ * TGRAD_ERR_BAD_STATE before the first step. */
+tgrad_status tgrad_diagnostics(tgrad_state* st, const void* d_grad, void* cuda_stream, double* out);
 
 /* Frees the host handle only. */
 tgrad_status tgrad_destroy_state(tgrad_state* st);

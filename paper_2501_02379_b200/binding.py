@@ -63,7 +63,7 @@ EXPORTS = [
     "tgrad_state_bytes", "tgrad_init_state", "tgrad_step", "tgrad_refresh_subspace", "tgrad_step_batched",
     "tgrad_refresh_subspace_batched", "tgrad_query_status", "tgrad_export_state", "tgrad_import_state",
     "tgrad_set_step", "tgrad_destroy_state", "tgrad_status_string", "tgrad_launch_count",
-    "tgrad_set_stage_timing", "tgrad_get_stage_times", "tgrad_select_topk_noalloc",
+    "tgrad_set_stage_timing", "tgrad_get_stage_times", "tgrad_select_topk_noalloc", "tgrad_diagnostics",
 ]
 
 
@@ -95,6 +95,7 @@ def lib() -> C.CDLL:
         l.tgrad_set_stage_timing.argtypes = [vp, C.c_int32]
         l.tgrad_get_stage_times.argtypes = [vp, vp, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
         l.tgrad_select_topk_noalloc.argtypes = [vp, C.c_int64, C.c_int64, C.c_int32, vp, vp, vp]
+        l.tgrad_diagnostics.argtypes = [vp, vp, vp, C.POINTER(C.c_double)]
         for name in EXPORTS:
             if name not in ("tgrad_status_string", "tgrad_launch_count"):
                 getattr(l, name).restype = C.c_int
@@ -245,6 +246,12 @@ class TgradState:
 
     def set_step(self, t: int):
         _check(lib().tgrad_set_step(self.handle, int(t)), "tgrad_set_step")
+
+    def diagnostics(self, grad, stream=None):
+        """(||G||_F, sparse share, low-rank reconstruction error relative to ||G||_F, orthonormality defect) of the last step."""
+        out = (C.c_double * 4)()
+        _check(lib().tgrad_diagnostics(self.handle, grad.data_ptr(), _stream_ptr(stream), out), "tgrad_diagnostics")
+        return tuple(float(out[i]) for i in range(4))
 
     def set_stage_timing(self, on: bool):
         _check(lib().tgrad_set_stage_timing(self.handle, 1 if on else 0), "tgrad_set_stage_timing")

@@ -37,7 +37,7 @@ struct Layout {
   uint32_t nslab, E;          // slabs of the trailing two modes, entries per slab
   // workspace block
   size_t w_ns, w_gs, w_core, w_nl, w_bufa, w_bufb, w_sel, w_hist, w_blk, w_gram[TGRAD_MAX_NDIM], w_jac[TGRAD_MAX_NDIM],
-      w_v[TGRAD_MAX_NDIM], w_log[TGRAD_MAX_NDIM], w_lam[TGRAD_MAX_NDIM], w_partial, w_hooi0, w_hooi1, w_ident, w_rbuf, w_total;
+      w_v[TGRAD_MAX_NDIM], w_log[TGRAD_MAX_NDIM], w_lam[TGRAD_MAX_NDIM], w_partial, w_hooi0, w_hooi1, w_ident, w_rbuf, w_diag, w_total;
   uint32_t hooi_smem;         // shared memory of the compression kernel when one trailing factor is replaced by the identity
   bool jac_fast[TGRAD_MAX_NDIM];    // eigensolver with the matrix in shared memory and a rotation log
   uint64_t numel, P, tsize;   // entries, core entries, entries of the tail-contracted tensor
@@ -201,6 +201,7 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
     L.w_ident = o; o = align_up(o + (size_t)(mx * mx) * 8);
   }
   // low-rank-first composition: G - P_U(G) at full size, from which a refresh selects Omega
+  L.w_diag = o; o = align_up(o + 8 * sizeof(double));          // scalars of the diagnostics call
   L.w_rbuf = o;
   if (c->composition == 1) o = align_up(o + (size_t)numel * (c->wg_dtype == TGRAD_C64 ? 8 : 4));
   L.w_total = o;
@@ -738,6 +739,37 @@ __global__ void lowrank_at_omega_kernel(cf* __restrict__ g_s, const uint32_t* __
   g_s[j] = v;
 }
 
+// ---- diagnostics (not on the timed path) ----
+// *acc += sum |x_i|^2 over n complex entries of storage S, in double
+template <class S>
+__global__ void diag_sumsq_kernel(const void* __restrict__ x, uint64_t n, double* __restrict__ acc) {
+  __shared__ double sh[8];
+  double sum = 0.0;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    const cf v = S::load(x, i);
+    sum += (double)v.x * v.x + (double)v.y * v.y;
+  }
+  for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = sum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += sh[w];
+    atomicAdd(acc, t);
+  }
+}
+// *defect = max(*defect, max_{a,b} |(U^H U - I)[a][b]|) for an n x r factor (the maximum of non-negative floats is
+// the maximum of their bit patterns)
+__global__ void diag_ortho_kernel(const cf* __restrict__ U, int n, int r, unsigned int* __restrict__ defect) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= r * r) return;
+  const int a = idx / r, b = idx - a * r;
+  cf acc = make_float2(0.f, 0.f);
+  for (int i = 0; i < n; ++i) cfma_conj(acc, U[(size_t)i * r + b], U[(size_t)i * r + a]);
+  if (a == b) acc.x -= 1.f;
+  atomicMax(defect, __float_as_uint(fmaxf(fabsf(acc.x), fabsf(acc.y))));
+}
+
 __global__ void identity_kernel(cf* __restrict__ m, int n) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx < n * n) m[idx] = make_float2((idx / n) == (idx % n) ? 1.f : 0.f, 0.f);
@@ -977,6 +1009,32 @@ tgrad_status do_step(tgrad_state* s, void* d_weight, void* d_grad, cudaStream_t 
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// Side streams of the batched step, one set per device, created at the first batched call on that device and kept
+// for the life of the process.
+constexpr int kBatchStreams = 4, kBatchDevices = 64;
+struct BatchStreams {
+  std::mutex mu;
+  bool ready = false;
+  cudaStream_t side[kBatchStreams];
+  cudaEvent_t fork, join[kBatchStreams];
+};
+BatchStreams g_batch[kBatchDevices];
+BatchStreams* batch_streams() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kBatchDevices) return nullptr;
+  BatchStreams* b = &g_batch[dev];
+  std::lock_guard<std::mutex> lock(b->mu);
+  if (!b->ready) {
+    bool ok = cudaEventCreateWithFlags(&b->fork, cudaEventDisableTiming) == cudaSuccess;
+    for (int j = 0; ok && j < kBatchStreams; ++j)
+      ok = cudaStreamCreateWithFlags(&b->side[j], cudaStreamNonBlocking) == cudaSuccess &&
+           cudaEventCreateWithFlags(&b->join[j], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return nullptr;          // fall back to the caller's stream alone
+    b->ready = true;
+  }
+  return b;
+}
+
 }  // namespace
 
 extern "C" {
@@ -1076,9 +1134,27 @@ tgrad_status tgrad_step_batched(tgrad_state* const* states, void* const* d_weigh
     if (!states[i]->have_subspace && !(states[i]->cfg.auto_refresh && states[i]->t % states[i]->cfg.T == 0))
       return TGRAD_ERR_BAD_STATE;
   }
-  for (int i = 0; i < n_tensors; ++i)
-    TG_TRY(do_step(states[i], d_weights[i], d_grads[i], static_cast<cudaStream_t>(cuda_stream)));
-  return TGRAD_OK;
+  cudaStream_t user = static_cast<cudaStream_t>(cuda_stream);
+  // The chains of small tensors are bound by launch and dependency latency, not by the GPU, and the tensors are
+  // independent: fork them onto the library's side streams and join them back into the caller's stream.  Work
+  // enqueued on the caller's stream before this call happens before all of it, work enqueued after it happens after.
+  BatchStreams* bs = (n_tensors > 1) ? batch_streams() : nullptr;
+  if (!bs) {
+    for (int i = 0; i < n_tensors; ++i) TG_TRY(do_step(states[i], d_weights[i], d_grads[i], user));
+    return TGRAD_OK;
+  }
+  std::lock_guard<std::mutex> lock(bs->mu);
+  if (cudaEventRecord(bs->fork, user) != cudaSuccess) return TGRAD_ERR_CUDA;
+  const int lanes = n_tensors < kBatchStreams ? n_tensors : kBatchStreams;
+  for (int j = 0; j < lanes; ++j)
+    if (cudaStreamWaitEvent(bs->side[j], bs->fork, 0) != cudaSuccess) return TGRAD_ERR_CUDA;
+  tgrad_status result = TGRAD_OK;
+  for (int i = 0; i < n_tensors && result == TGRAD_OK; ++i) result = do_step(states[i], d_weights[i], d_grads[i], bs->side[i % lanes]);
+  for (int j = 0; j < lanes; ++j) {           // join even after an error, so that nothing is left running unordered
+    if (cudaEventRecord(bs->join[j], bs->side[j]) != cudaSuccess || cudaStreamWaitEvent(user, bs->join[j], 0) != cudaSuccess)
+      return TGRAD_ERR_CUDA;
+  }
+  return result;
 }
 
 tgrad_status tgrad_refresh_subspace_batched(tgrad_state* const* states, void* const* d_grads, int32_t n_tensors,
@@ -1168,6 +1244,44 @@ tgrad_status tgrad_import_state(tgrad_state* st, int32_t what, const void* host_
   }
   if (what == TGRAD_WHAT_OMEGA || what >= TGRAD_WHAT_FACTOR_BASE) st->have_subspace = true;
   if (what >= TGRAD_WHAT_FACTOR_BASE) { st->tabs_stale = true; st->basis_valid = true; }
+  return TGRAD_OK;
+}
+
+tgrad_status tgrad_diagnostics(tgrad_state* st, const void* d_grad, void* cuda_stream, double* out) {
+  if (!st || !d_grad || !out) return TGRAD_ERR_INVALID_ARG;
+  if (!aligned16(d_grad)) return TGRAD_ERR_INVALID_ARG;
+  if (!st->have_subspace || st->t < 1) return TGRAD_ERR_BAD_STATE;
+  const tgrad_config& c = st->cfg; const Layout& L = st->L;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  double* acc = reinterpret_cast<double*>(st->dw + L.w_diag);
+  if (cudaMemsetAsync(acc, 0, 8 * sizeof(double), stream) != cudaSuccess) return TGRAD_ERR_CUDA;
+  const unsigned gsz = (unsigned)(st->sm_count * 8);
+  if (c.wg_dtype == TGRAD_C64) diag_sumsq_kernel<StoreC64><<<gsz, 256, 0, stream>>>(d_grad, L.numel, acc + 0);
+  else if (c.wg_dtype == TGRAD_C32H) diag_sumsq_kernel<StoreC32H><<<gsz, 256, 0, stream>>>(d_grad, L.numel, acc + 0);
+  else diag_sumsq_kernel<StoreC32B><<<gsz, 256, 0, stream>>>(d_grad, L.numel, acc + 0);
+  TG_LAUNCH_CHECK();
+  if (c.k > 0) { diag_sumsq_kernel<StoreC64><<<64, 256, 0, stream>>>(st->dw + L.w_gs, (uint64_t)c.k, acc + 1); TG_LAUNCH_CHECK(); }
+  diag_sumsq_kernel<StoreC64><<<64, 256, 0, stream>>>(st->dw + L.w_core, L.P, acc + 2); TG_LAUNCH_CHECK();
+  for (int n = 0; n < c.ndim; ++n) {
+    const int r = c.ranks[n];
+    diag_ortho_kernel<<<(r * r + 127) / 128, 128, 0, stream>>>(reinterpret_cast<const cf*>(st->dp + L.p_factor[n]), (int)c.dims[n], r,
+                                                              reinterpret_cast<unsigned int*>(acc + 3));
+    TG_LAUNCH_CHECK();
+  }
+  double host[4];
+  if (cudaMemcpyAsync(host, acc, sizeof(host), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return TGRAD_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return TGRAD_ERR_CUDA;
+  const double g2 = host[0], s2 = host[1], l2 = host[2];
+  unsigned int bits; memcpy(&bits, &host[3], sizeof(bits));
+  float defect; memcpy(&defect, &bits, sizeof(defect));
+  // what the low-rank part was given: the residual of the sparse part in Algorithm 1's order (the sparse values were
+  // gathered from the gradient itself there), the gradient otherwise
+  const double x2 = (c.composition == 0) ? (g2 - s2 > 0 ? g2 - s2 : 0.0) : g2;
+  const double gn = std::sqrt(g2);
+  out[0] = gn;
+  out[1] = gn > 0 ? std::sqrt(s2) / gn : 0.0;
+  out[2] = gn > 0 ? std::sqrt(x2 - l2 > 0 ? x2 - l2 : 0.0) / gn : 0.0;
+  out[3] = (double)defect;
   return TGRAD_OK;
 }
 

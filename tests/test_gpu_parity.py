@@ -191,6 +191,26 @@ def test_bf16_storage_small(name):
     print("bf16", name, p.report)
 
 
+@pytest.mark.parametrize("composition", ["us_lr", "sum"])
+def test_diagnostics_against_the_definitions(composition):
+    wl = synth.WORKLOADS["ragged4"]
+    p = Pair(wl, composition=composition)
+    p.step(0)
+    g = p.src.gradient(1)
+    g_dev = to_device(g, False)
+    p.step(1)
+    gn, share, lost, defect = p.gst.diagnostics(g_dev)
+    g128 = g.astype(np.complex128)
+    us = p.ost.factors
+    gs = g128.reshape(-1)[p.ost.omega.astype(np.int64)]
+    x = orc.residual(g, p.ost.omega).astype(np.complex128) if composition == "us_lr" else g128
+    want_lost = np.linalg.norm(x - orc.tucker_reconstruct(orc.tucker_compress(x, us), us)) / np.linalg.norm(g128)
+    assert abs(gn - np.linalg.norm(g128)) <= 1e-6 * gn
+    assert abs(share - np.linalg.norm(gs) / np.linalg.norm(g128)) <= 1e-6
+    assert abs(lost - want_lost) <= 1e-4 * max(want_lost, 1e-3)
+    assert abs(defect - max(H.ortho_defect(u) for u in us)) <= 2e-7 and defect < 1e-5
+
+
 def test_auto_refresh_matches_explicit():
     wl = synth.WORKLOADS["small4"]
     src = synth.GradientSource(wl)
