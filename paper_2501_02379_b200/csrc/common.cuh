@@ -28,11 +28,6 @@ struct StoreC64 {
   static constexpr int kBytes = 8;
   __device__ static __forceinline__ cf widen(const elem& e) { return e; }
   __device__ static __forceinline__ cf narrow(cf v) { return v; }
-  static constexpr int kVec = 2;         // entries per 16-byte load
-  __device__ static __forceinline__ void load16(const void* p, size_t vi, cf (&out)[kVec]) {
-    const float4 q = reinterpret_cast<const float4*>(p)[vi];
-    out[0] = make_float2(q.x, q.y); out[1] = make_float2(q.z, q.w);
-  }
   __device__ static __forceinline__ cf load(const void* p, size_t i) { return reinterpret_cast<const float2*>(p)[i]; }
   __device__ static __forceinline__ void store(void* p, size_t i, cf v) { reinterpret_cast<float2*>(p)[i] = v; }
 };
@@ -41,13 +36,6 @@ struct StoreC32H {
   static constexpr int kBytes = 4;
   __device__ static __forceinline__ cf widen(const elem& e) { return __half22float2(e); }
   __device__ static __forceinline__ cf narrow(cf v) { return __half22float2(__floats2half2_rn(v.x, v.y)); }
-  static constexpr int kVec = 4;
-  __device__ static __forceinline__ void load16(const void* p, size_t vi, cf (&out)[kVec]) {
-    const uint4 q = reinterpret_cast<const uint4*>(p)[vi];
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) out[e] = __half22float2(*reinterpret_cast<const __half2*>(&w[e]));
-  }
   __device__ static __forceinline__ cf load(const void* p, size_t i) {
     return __half22float2(reinterpret_cast<const __half2*>(p)[i]);
   }
@@ -61,13 +49,6 @@ struct StoreC32B {
   static constexpr int kBytes = 4;
   __device__ static __forceinline__ cf widen(const elem& e) { return __bfloat1622float2(e); }
   __device__ static __forceinline__ cf narrow(cf v) { return __bfloat1622float2(__floats2bfloat162_rn(v.x, v.y)); }
-  static constexpr int kVec = 4;
-  __device__ static __forceinline__ void load16(const void* p, size_t vi, cf (&out)[kVec]) {
-    const uint4 q = reinterpret_cast<const uint4*>(p)[vi];
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) out[e] = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
-  }
   __device__ static __forceinline__ cf load(const void* p, size_t i) {
     return __bfloat1622float2(reinterpret_cast<const __nv_bfloat162*>(p)[i]);
   }

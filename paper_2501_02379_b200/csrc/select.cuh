@@ -101,50 +101,34 @@ __global__ void __launch_bounds__(512) sel_hist_kernel(const void* __restrict__ 
   const uint32_t prefix = st->prefix;
   const uint32_t hi_mask = (pass == 0) ? 0u : (0xffffffffu << (shift + bits));
   bool bad = false;
-  // one entry into the shared histogram; every lane of the warp calls this together
-  auto tally = [&](bool valid, cf v, uint32_t i) {
-    const uint32_t key = valid ? sel_key(v, i, kp) : 0u;
-    // a NaN or an infinity among the magnitudes (the random strategy does not look at them)
-    if (valid && pass == 0 && kp.strategy != 1 && (mag_key(v) & 0x7f800000u) == 0x7f800000u) bad = true;
-    const bool in = valid && (key & hi_mask) == prefix;
-    const uint32_t d = (key >> shift) & (nb - 1u);
-    // warp-aggregated shared atomics: gradients crowd into a few exponent bins
-    const unsigned act = __ballot_sync(0xffffffffu, in);
-    if (in) {
-      const unsigned peers = __match_any_sync(act, d);
-      if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&sh[d], (uint32_t)__popc(peers));
-    }
-  };
-  // 16-byte loads (two complex64 or four 16-bit entries), two per thread and iteration so that they are in flight together
-  constexpr int VEC = S::kVec, UN = 2;
-  const uint64_t nvec = (uint64_t)n / VEC;
+  constexpr int UN = 4;                       // entries per thread and iteration: their loads are issued together
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x * UN;
-  // block-uniform loop bound, so every warp stays converged for the warp votes
-  for (uint64_t b0 = (uint64_t)blockIdx.x * blockDim.x * UN; b0 < nvec; b0 += stride) {
-    cf v[UN][VEC];
+  // block-uniform loop bound, so every warp stays converged for the warp votes below
+  for (uint64_t b0 = (uint64_t)blockIdx.x * blockDim.x * UN; b0 < n; b0 += stride) {
+    uint32_t keys[UN];
     bool valid[UN];
 #pragma unroll
     for (int j = 0; j < UN; ++j) {
-      const uint64_t vi = b0 + (uint64_t)j * blockDim.x + threadIdx.x;
-      valid[j] = vi < nvec;
-      if (valid[j]) S::load16(g, vi, v[j]);
-      else {
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) v[j][e] = make_float2(0.f, 0.f);
-      }
+      const uint64_t i = b0 + (uint64_t)j * blockDim.x + threadIdx.x;
+      valid[j] = i < n;
+      cf v = make_float2(0.f, 0.f);
+      if (valid[j]) v = S::load(g, i);
+      keys[j] = valid[j] ? sel_key(v, (uint32_t)i, kp) : 0u;
+      // a NaN or an infinity among the magnitudes (the random strategy does not look at them)
+      if (pass == 0 && kp.strategy != 1 && (mag_key(v) & 0x7f800000u) == 0x7f800000u) bad = true;
     }
 #pragma unroll
     for (int j = 0; j < UN; ++j) {
-      const uint64_t vi = b0 + (uint64_t)j * blockDim.x + threadIdx.x;
-#pragma unroll
-      for (int e = 0; e < VEC; ++e) tally(valid[j], v[j][e], (uint32_t)(vi * VEC + e));
+      const uint32_t key = keys[j];
+      bool in = valid[j] && (key & hi_mask) == prefix;
+      uint32_t d = (key >> shift) & (nb - 1u);
+      // warp-aggregated shared atomics: gradients crowd into a few exponent bins
+      unsigned act = __ballot_sync(0xffffffffu, in);
+      if (in) {
+        unsigned peers = __match_any_sync(act, d);
+        if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&sh[d], (uint32_t)__popc(peers));
+      }
     }
-  }
-  // the last n mod VEC entries
-  if (blockIdx.x == 0 && threadIdx.x < 32) {
-    const uint32_t i = (uint32_t)(nvec * VEC) + threadIdx.x;
-    const bool valid = i < n;
-    tally(valid, valid ? S::load(g, i) : make_float2(0.f, 0.f), i);
   }
   __syncthreads();
   for (uint32_t i = threadIdx.x; i < nb; i += blockDim.x) {
@@ -209,17 +193,12 @@ __global__ void __launch_bounds__(kChunkThreads) sel_count_kernel(const void* __
   const uint32_t thr = st->thr;
   const uint32_t base = blockIdx.x * (uint32_t)kChunk;
   uint32_t cg = 0, ce = 0;
-  // 16-byte loads in coalesced order: only totals matter here (a chunk starts on a 16-byte boundary)
-  constexpr int VEC = S::kVec;
-  for (int r = 0; r < kChunk / (kChunkThreads * VEC); ++r) {
-    const uint32_t i0 = base + (r * kChunkThreads + threadIdx.x) * VEC;
-    if (i0 + VEC <= n) {
-      cf v[VEC];
-      S::load16(g, i0 / VEC, v);
-#pragma unroll
-      for (int e = 0; e < VEC; ++e) { const uint32_t key = sel_key(v[e], i0 + e, kp); cg += key > thr; ce += key == thr; }
-    } else {
-      for (uint32_t i = i0; i < n && i < i0 + VEC; ++i) { const uint32_t key = sel_key(S::load(g, i), i, kp); cg += key > thr; ce += key == thr; }
+  // coalesced order here: only totals matter
+  for (int r = 0; r < kChunk / kChunkThreads; ++r) {
+    uint32_t i = base + r * kChunkThreads + threadIdx.x;
+    if (i < n) {
+      uint32_t key = sel_key(S::load(g, i), i, kp);
+      cg += key > thr; ce += key == thr;
     }
   }
   for (int o = 16; o; o >>= 1) { cg += __shfl_xor_sync(0xffffffffu, cg, o); ce += __shfl_xor_sync(0xffffffffu, ce, o); }
