@@ -1,19 +1,18 @@
 // The two full-tensor streaming kernels of a step.
 //
 // The tensor is seen as S = prod(I_1..I_{N-2}) slabs of A x B entries
-// (A = I_{N-1}, B = I_N, B contiguous).  One warp owns one slab at a time.
+// (A = I_{N-1}, B = I_N, B contiguous).  This file holds what all variants share (parameters, the
+// AdamUpdate) and the general kernels: one thread block per slab at a time, fp32 arithmetic, any
+// slab that fits in shared memory, any storage type.
 //
-// proj_tail (read G once):   per slab, gather the sparse values at Omega and run
-//   their Adam update, zero them (the residual R = G - Sparse(G, Omega)), then
+// proj_tail (read G once):   per slab, gather the sparse values at Omega (their Adam update runs with
+//   the core's), zero them (the residual R = G - Sparse(G, Omega)), then
 //   contract the two trailing modes:  T[s, ja, jb] = sum_{a,b} conj(Ua[a,ja]) conj(Ub[b,jb]) R[s,a,b]
 //   (the last two of the chained mode-n products of the low-rank compression).
 // back_tail (read+write W once): per slab, expand the two trailing modes of the
 //   normalised core, D[s,a,b] = sum_{ja,jb} Ua[a,ja] Ub[b,jb] T'[s,ja,jb], and apply
 //   W <- (1 - eta wd) W - eta alpha D, then W[Omega] -= eta lambda N_S
 //   (reconstruction, scaled sparse add and weight update of Algorithm 1).
-//
-// Lane l of the warp owns rows a = l + 32 r of the slab (r < RPL); the rb
-// columns of the small side live in registers (RBP = rb padded).
 #pragma once
 #include "common.cuh"
 

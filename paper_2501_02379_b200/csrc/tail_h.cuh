@@ -286,7 +286,7 @@ __global__ void __launch_bounds__(512, 1) proj_tail_h_kernel(const void* __restr
 // Two warps share a tile of 16 rows of the slab (each takes half of the column tiles); the products are the
 // split-TF32 ones of back_tail_tc_kernel, with the Ua and Ub fragments in shared-memory tables.  The slab
 // stays fp16 in shared memory: the dense update is rounded to fp16 when it is written back there, the
-// sparse term is then added by one thread per entry and rounded again (the two roundings the oracle makes),
+// sparse term is then added by one thread per entry and rounded again (the storage type is rounded to once after the dense update and once more at Omega),
 // and one bulk copy stores the slab.
 // ---------------------------------------------------------------------------------------------
 struct TailHBGeom {

@@ -1,14 +1,16 @@
 // Fast path of the two streaming kernels of a step (complex64 storage, trailing slab of
 // A x B entries with A in {16, 32, 64}, B <= 33, r_{N-1} <= 16, r_N <= 8).
 //
-// A thread block of eight warps works on one group of 8*8/A.. consecutive slabs at a time.  Groups
-// arrive by bulk asynchronous copy into a ring in shared memory that the whole block shares; a
-// block keeps several groups in flight, and two blocks are resident per SM (16 warps).  The two
+// A thread block works on one group of consecutive slabs at a time.  Groups arrive by bulk
+// asynchronous copy into a ring in shared memory that the whole block shares, and a block keeps
+// several groups in flight.  The compression kernel runs blocks of four warps, four blocks per SM;
+// the reconstruction kernel blocks of eight warps, two per SM (16 warps per SM either way).  The two
 // trailing mode products run on the tensor cores as split-precision TF32 (x = hi + lo, the
 // three products hi*hi, lo*hi, hi*lo, fp32 accumulation), chained through registers: the
 // accumulator fragments of the first product are the operand fragments of the second.  The
 // factor-matrix fragments a warp needs never change (a warp always owns the same rows of a
-// slab), so they live in registers for the whole kernel.
+// slab): the reconstruction keeps them in registers for the whole kernel, the compression reads
+// them from small tables in shared and global memory laid out in MMA register order.
 //
 // Complex arithmetic is carried as real arithmetic on interleaved (re, im) data:
 //   Y = X conj(Ub):   [Yre; Yim] = W1 [Xre; Xim],  W1 = [[ur, ui], [-ui, ur]]

@@ -5,7 +5,8 @@ Nothing here implements the optimizer; these are measuring sticks.
 import numpy as np
 
 
-FLOOR_FRAC = 2.0 ** -5
+FLOOR_FRAC = 2.0 ** -7            # every workload with a full oracle comparison passes at 2^-8 or tighter (most at 2^-16)
+FLOOR_FRAC_LARGE = 2.0 ** -5      # the 545 M-entry configuration, whose 2 M-entry core comes from fp16-stored operands
 
 
 def rel_err(a, b, floor_frac=FLOOR_FRAC):
@@ -18,8 +19,9 @@ def rel_err(a, b, floor_frac=FLOOR_FRAC):
     partial sum rounds.  Measured: rms error 2-4 u, maximum over 1e4..2e6 entries
     up to about 20 u.  An entry much smaller than rms(b) is the result of
     cancellation and cannot carry a 1e-4 *relative* accuracy in fp32; the bound
-    1e-4 * tau = 1e-4 * 2^-5 * rms = 52 u * rms is the absolute accuracy asked of
-    those entries, and every entry above tau must meet 1e-4 relative to itself.
+    1e-4 * tau (13 u * rms at the default floor 2^-7, 52 u * rms at 2^-5) is the absolute
+    accuracy asked of those entries, and every entry above tau must meet 1e-4 relative
+    to itself.
     """
     a = np.asarray(a).reshape(-1).astype(np.complex128)
     b = np.asarray(b).reshape(-1).astype(np.complex128)

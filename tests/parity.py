@@ -15,7 +15,7 @@ from paper_2501_02379_b200 import binding as B
 from paper_2501_02379_b200 import synth
 from tests import helpers as H
 
-TOL_FLOAT = 1e-4       # max relative error, entries measured against max(|ref|, 2^-5 rms(ref)); see helpers.rel_err
+TOL_FLOAT = 1e-4       # max relative error, entries measured against max(|ref|, 2^-7 rms(ref)); see helpers.rel_err
 TOL_FRO = 5e-6         # and the whole array: ||a - b||_F / ||b||_F (split-TF32 products carry 2^-21 relative error
                        # each, and an entry passes through up to 2 N of them)
 TOL_ANGLE = 1e-3       # largest principal-angle sine of a refreshed factor
@@ -192,7 +192,7 @@ class Pair:
             if name in ("m_s", "v_s") and c.composition != "lr_us":       # (low rank first: the sparse values are differences too)
                 assert e3 <= TOL_FLOAT, f"{name}: max relative error {e3} at the 1e-3 rms floor"
             elif a.size <= (1 << 22):
-                self._note_min(name + "_floor_log2", H.tightest_floor_log2(a, b, TOL_FLOAT))
+                self._note_min(name + "_floor_log2", H.tightest_floor_log2(a, b, TOL_FLOAT, lo=7))
                 self._note(name + "_below_1e-3", H.below_floor_fraction(b))
             f = H.fro_err(a, b)
             self._note(name + "_fro", f)
@@ -374,7 +374,7 @@ class SampledChecker:
         # compressed gradient: every entry
         core = st.export(B.WHAT_CORE)
         want_core = full_core_by_slices(r, self.factors)
-        e = H.rel_err(core, want_core); self._note("core", e); assert e <= TOL_FLOAT, ("core", e)
+        e = H.rel_err(core, want_core, H.FLOOR_FRAC_LARGE); self._note("core", e); assert e <= TOL_FLOAT, ("core", e)
         f = H.fro_err(core, want_core); self._note("core_fro", f); assert f <= TOL_FRO, ("core", f)
         self._note("core@1e-3", H.rel_err(core, want_core, H.FLOOR_CONTRACT))
         del r
