@@ -89,7 +89,9 @@ __global__ void sel_init_kernel(SelState* st, uint32_t k) {
 
 // Histogram of the current digit over all entries whose higher bits equal the
 // prefix chosen so far.
-template <class S>
+// TOPK: the key is the magnitude (the strategy of Algorithm 1 and of the five benchmark configurations): built in, so
+// that this path carries nothing of the random strategies.
+template <class S, bool TOPK>
 __global__ void __launch_bounds__(512) sel_hist_kernel(const void* __restrict__ g, uint32_t n, int pass,
                                                       const SelState* __restrict__ st, uint32_t* __restrict__ hist,
                                                       int* __restrict__ flags, SelKey kp) {
@@ -113,9 +115,9 @@ __global__ void __launch_bounds__(512) sel_hist_kernel(const void* __restrict__ 
       valid[j] = i < n;
       cf v = make_float2(0.f, 0.f);
       if (valid[j]) v = S::load(g, i);
-      keys[j] = valid[j] ? sel_key(v, (uint32_t)i, kp) : 0u;
+      keys[j] = valid[j] ? (TOPK ? mag_key(v) : sel_key(v, (uint32_t)i, kp)) : 0u;
       // a NaN or an infinity among the magnitudes (the random strategy does not look at them)
-      if (pass == 0 && kp.strategy != 1 && (mag_key(v) & 0x7f800000u) == 0x7f800000u) bad = true;
+      if (pass == 0 && (TOPK || kp.strategy != 1) && (mag_key(v) & 0x7f800000u) == 0x7f800000u) bad = true;
     }
 #pragma unroll
     for (int j = 0; j < UN; ++j) {
@@ -184,7 +186,7 @@ __global__ void __launch_bounds__(1024) sel_pick_kernel(const uint32_t* __restri
 }
 
 // Per block of kChunk consecutive entries: how many keys lie above / at the threshold.
-template <class S>
+template <class S, bool TOPK>
 __global__ void __launch_bounds__(kChunkThreads) sel_count_kernel(const void* __restrict__ g, uint32_t n,
                                                                   const SelState* __restrict__ st,
                                                                   uint32_t* __restrict__ blk_gt,
@@ -197,7 +199,7 @@ __global__ void __launch_bounds__(kChunkThreads) sel_count_kernel(const void* __
   for (int r = 0; r < kChunk / kChunkThreads; ++r) {
     uint32_t i = base + r * kChunkThreads + threadIdx.x;
     if (i < n) {
-      uint32_t key = sel_key(S::load(g, i), i, kp);
+      uint32_t key = TOPK ? mag_key(S::load(g, i)) : sel_key(S::load(g, i), i, kp);
       cg += key > thr; ce += key == thr;
     }
   }
@@ -251,7 +253,7 @@ __global__ void __launch_bounds__(1024) sel_scan_kernel(uint32_t* __restrict__ b
 // fewer than take_eq equal keys precede it.  Its slot is the number of selected
 // entries before it, so Omega comes out strictly ascending.  The selected values
 // are saved to g_s (fp32 complex) for the residual/restore passes of the refresh.
-template <class S>
+template <class S, bool TOPK>
 __global__ void __launch_bounds__(kChunkThreads) sel_compact_kernel(const void* __restrict__ g, uint32_t n,
                                                                     const SelState* __restrict__ st,
                                                                     const uint32_t* __restrict__ blk_gt,
@@ -268,7 +270,7 @@ __global__ void __launch_bounds__(kChunkThreads) sel_compact_kernel(const void* 
 #pragma unroll
   for (int e = 0; e < EPT; ++e) {
     uint32_t i = base + e;
-    if (i < n) { v[e] = S::load(g, i); key[e] = sel_key(v[e], i, kp); } else { v[e] = make_float2(0.f, 0.f); key[e] = 0u; }
+    if (i < n) { v[e] = S::load(g, i); key[e] = TOPK ? mag_key(v[e]) : sel_key(v[e], i, kp); } else { v[e] = make_float2(0.f, 0.f); key[e] = 0u; }
     bool valid = i < n;
     cnt += (valid && key[e] > thr) ? 1u : 0u;
     cnt += (valid && key[e] == thr) ? 0x10000u : 0u;

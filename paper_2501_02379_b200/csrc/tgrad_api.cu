@@ -583,14 +583,19 @@ tgrad_status select_omega(tgrad_state* s, const void* x, cudaStream_t st) {
   sel_init_kernel<<<1, 1, 0, st>>>(sel, k); TG_LAUNCH_CHECK();
   uint64_t want = ((uint64_t)n + 511) / 512;
   int hgrid = (int)(want < (uint64_t)s->sm_count * 8 ? want : (uint64_t)s->sm_count * 8);
+  const bool topk = c.sparse_strategy == 0;
   for (int pass = 0; pass < 3; ++pass) {
-    sel_hist_kernel<S><<<hgrid, 512, 0, st>>>(x, n, pass, sel, hist + pass * kSelMaxBins, flags, kp);
+    if (topk) sel_hist_kernel<S, true><<<hgrid, 512, 0, st>>>(x, n, pass, sel, hist + pass * kSelMaxBins, flags, kp);
+    else sel_hist_kernel<S, false><<<hgrid, 512, 0, st>>>(x, n, pass, sel, hist + pass * kSelMaxBins, flags, kp);
     TG_LAUNCH_CHECK();
     sel_pick_kernel<<<1, 1024, 0, st>>>(hist + pass * kSelMaxBins, pass, sel); TG_LAUNCH_CHECK();
   }
-  sel_count_kernel<S><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, kp); TG_LAUNCH_CHECK();
+  if (topk) sel_count_kernel<S, true><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, kp);
+  else sel_count_kernel<S, false><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, kp);
+  TG_LAUNCH_CHECK();
   sel_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, L.nblk); TG_LAUNCH_CHECK();
-  sel_compact_kernel<S><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, omega, g_s, k, kp);
+  if (topk) sel_compact_kernel<S, true><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, omega, g_s, k, kp);
+  else sel_compact_kernel<S, false><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, omega, g_s, k, kp);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
@@ -1402,13 +1407,13 @@ tgrad_status select_noalloc_impl(const void* d_grad, uint32_t n, uint32_t k, uin
   const uint64_t want = ((uint64_t)n + 511) / 512;
   const int hgrid = (int)(want < (uint64_t)sm * 8 ? want : (uint64_t)sm * 8);
   for (int pass = 0; pass < 3; ++pass) {
-    sel_hist_kernel<S><<<hgrid, 512, 0, st>>>(d_grad, n, pass, &sc->sel, sc->hist + pass * kSelMaxBins, sc->flags, kp);
+    sel_hist_kernel<S, true><<<hgrid, 512, 0, st>>>(d_grad, n, pass, &sc->sel, sc->hist + pass * kSelMaxBins, sc->flags, kp);
     TG_LAUNCH_CHECK();
     sel_pick_kernel<<<1, 1024, 0, st>>>(sc->hist + pass * kSelMaxBins, pass, &sc->sel); TG_LAUNCH_CHECK();
   }
-  sel_count_kernel<S><<<nblk, kChunkThreads, 0, st>>>(d_grad, n, &sc->sel, blk_gt, blk_eq, kp); TG_LAUNCH_CHECK();
+  sel_count_kernel<S, true><<<nblk, kChunkThreads, 0, st>>>(d_grad, n, &sc->sel, blk_gt, blk_eq, kp); TG_LAUNCH_CHECK();
   sel_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, nblk); TG_LAUNCH_CHECK();
-  sel_compact_kernel<S><<<nblk, kChunkThreads, 0, st>>>(d_grad, n, &sc->sel, blk_gt, blk_eq, d_omega, d_values, k, kp);
+  sel_compact_kernel<S, true><<<nblk, kChunkThreads, 0, st>>>(d_grad, n, &sc->sel, blk_gt, blk_eq, d_omega, d_values, k, kp);
   TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
