@@ -71,6 +71,14 @@ __device__ __forceinline__ void split_f16(float x, __half& hi, __half& lo) {
   lo = __float2half_rn(x - __half2float(hi));
 }
 
+// x = hi + lo / 2048 with hi, lo in fp16: lo carries the 11 bits below hi's at hi's own scale, so that neither part
+// nears the subnormal range before x itself does.
+constexpr float kF16LoScale = 2048.f, kF16LoInv = 1.f / 2048.f;
+__device__ __forceinline__ void split_f16_scaled(float x, __half& hi, __half& lo) {
+  hi = __float2half_rn(x);
+  lo = __float2half_rn((x - __half2float(hi)) * kF16LoScale);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Compression of the two trailing modes (half storage), fused with the sparse gather and the residual.
 //   stage 1 (fp16 m16n8k16), warp = tile of 8 rows a:
@@ -332,23 +340,29 @@ __global__ void __launch_bounds__(512, 1) back_tail_h_kernel(void* __restrict__ 
   const uint32_t E = p.E, nslab = p.nslab, gstride = gridDim.x;
   const int mtile = warp >> 1, am = 16 * mtile, r0 = am + gq, r1 = r0 + 8;
   const int nbh = (nbt + 1) / 2, nb0 = (warp & 1) ? nbh : 0, nb1 = (warp & 1) ? nbt : nbh;   // this warp's column tiles
-  float4* ubf = reinterpret_cast<float4*>(smem + G.off_ub);     // [nbt][RBT][2][32]
+  uint4* ubf = reinterpret_cast<uint4*>(smem + G.off_ub);       // [nbt][RBT][32]: fp16 pairs (b0.hi, b1.hi, b0.lo, b1.lo)
   float4* uaf = reinterpret_cast<float4*>(smem + G.off_ua);     // [A/16][KS2][hi|lo][32]
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + G.off_bar);
   unsigned char* wb = static_cast<unsigned char*>(w);
 
-  // Ub as stage-2 operand fragments (see back_tail_tc_kernel): per column tile, jb tile and lane
+  // Ub as stage-2 operand fragments of the fp16 m16n8k16 shape, per column tile, jb tile and lane (g, t):
+  //   n = g <-> (b, c), b = 16 (nb>>2) + (nb&3) + 4 (g>>1), c = g & 1;  k = 2t, 2t+1 <-> (jb, re), (jb+1, re),
+  //   k = 2t+8, 2t+9 <-> (jb, im), (jb+1, im), jb = 8 jt + 2t;
+  //   W3[(jb,re)][(b,re)] = ur, [(b,im)] = ui;  W3[(jb,im)][(b,re)] = -ui, [(b,im)] = ur.
+  // Each value as hi + lo / 2048 with hi and lo in fp16 (22 bits together; |u| <= 1).
   for (int idx = tid; idx < nbt * RBT * 32; idx += nthr) {
     const int nb = idx / (RBT * 32), rem = idx - nb * (RBT * 32), jt = rem >> 5, ln = rem & 31, g_ = ln >> 2, t_ = ln & 3;
     const int bq = 16 * (nb >> 2) + (nb & 3) + 4 * (g_ >> 1), jb = 8 * jt + 2 * t_;
     const bool odd = g_ & 1;
-    cf va = (bq < B && jb < rb) ? p.Ub[bq * rb + jb] : make_float2(0.f, 0.f);
-    cf vb = (bq < B && jb + 1 < rb) ? p.Ub[bq * rb + jb + 1] : make_float2(0.f, 0.f);
-    cf ah, al, bh, bl;
-    split_tf32(va.x, ah.x, al.x); split_tf32(va.y, ah.y, al.y);
-    split_tf32(vb.x, bh.x, bl.x); split_tf32(vb.y, bh.y, bl.y);
-    ubf[((nb * RBT + jt) * 2 + 0) * 32 + ln] = odd ? make_float4(ah.y, bh.y, al.y, bl.y) : make_float4(ah.x, bh.x, al.x, bl.x);
-    ubf[((nb * RBT + jt) * 2 + 1) * 32 + ln] = odd ? make_float4(ah.x, bh.x, al.x, bl.x) : make_float4(-ah.y, -bh.y, -al.y, -bl.y);
+    const cf va = (bq < B && jb < rb) ? p.Ub[bq * rb + jb] : make_float2(0.f, 0.f);
+    const cf vb = (bq < B && jb + 1 < rb) ? p.Ub[bq * rb + jb + 1] : make_float2(0.f, 0.f);
+    const float re0 = odd ? va.y : va.x, re1 = odd ? vb.y : vb.x;         // rows (jb, re), (jb+1, re) of column n
+    const float im0 = odd ? va.x : -va.y, im1 = odd ? vb.x : -vb.y;       // rows (jb, im), (jb+1, im)
+    __half h[4], l[4];
+    split_f16_scaled(re0, h[0], l[0]); split_f16_scaled(re1, h[1], l[1]);
+    split_f16_scaled(im0, h[2], l[2]); split_f16_scaled(im1, h[3], l[3]);
+    ubf[idx] = make_uint4(h2_bits(__halves2half2(h[0], h[1])), h2_bits(__halves2half2(h[2], h[3])),
+                          h2_bits(__halves2half2(l[0], l[1])), h2_bits(__halves2half2(l[2], l[3])));
   }
   // Ua as stage-1 operand fragments: rows am + g and am + g + 8, ja = 4 ks + t: (u0.x, u1.x, u0.y, u1.y) hi, then lo
   for (int idx = tid; idx < (A / 16) * KS2 * 32; idx += nthr) {
@@ -437,34 +451,38 @@ __global__ void __launch_bounds__(512, 1) back_tail_h_kernel(void* __restrict__ 
           mma_tf32(d1[1][jt], uh.x, uh.y, uh.z, uh.w, til, trl);
         }
       }
-      float yh[2][RBT][4], yl[2][RBT][4];
+      // Y' as fp16 m16n8k16 A fragments, hi and lo (scaled by 2048): a0 = (row g; jb, jb+1; re), a1 = (row g+8; re),
+      // a2 = (row g; im), a3 = (row g+8; im) -- the accumulator pairs of stage 1 as they are.  Y' is built from the
+      // Adam-normalised core through factors with orthonormal columns, so its entries are far inside the fp16 range.
+      uint32_t yh[RBT][4], yl[RBT][4];
 #pragma unroll
-      for (int c = 0; c < 2; ++c)
+      for (int jt = 0; jt < RBT; ++jt)
 #pragma unroll
-        for (int jt = 0; jt < RBT; ++jt)
+        for (int c = 0; c < 2; ++c)
 #pragma unroll
-          for (int i = 0; i < 4; ++i) split_tf32(d1[c][jt][i], yh[c][jt][i], yl[c][jt][i]);
-      // ---- stage 2, one column tile at a time, applied to the slab right away ----
+          for (int hrow = 0; hrow < 2; ++hrow) {
+            const float v0 = d1[c][jt][2 * hrow], v1 = d1[c][jt][2 * hrow + 1];
+            const __half2 hh = __floats2half2_rn(v0, v1);
+            const float2 back = __half22float2(hh);
+            yh[jt][2 * c + hrow] = h2_bits(hh);
+            yl[jt][2 * c + hrow] = h2_bits(__floats2half2_rn((v0 - back.x) * kF16LoScale, (v1 - back.y) * kF16LoScale));
+          }
+      // ---- stage 2, one column tile at a time, applied to the slab right away: three fp16 products per jb tile
+      //      (hi hi, lo hi, hi lo), the two small ones summed and scaled back by 1/2048 ----
       constexpr int NB_UNROLL = NBT ? (NBT + 1) / 2 : 1;
 #pragma unroll NB_UNROLL
       for (int nb = nb0; nb < nb1; ++nb) {
-        float dh[4], dl[4], dx[4];
+        float dh[4] = {0.f, 0.f, 0.f, 0.f}, dl[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int jt = 0; jt < RBT; ++jt) {
-          const float4 fr = ubf[((nb * RBT + jt) * 2 + 0) * 32 + lane], fi = ubf[((nb * RBT + jt) * 2 + 1) * 32 + lane];
-          if (jt == 0) {
-            mma_tf32_z(dh, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.x, fr.y);
-            mma_tf32_z(dl, yl[0][jt][0], yl[0][jt][2], yl[0][jt][1], yl[0][jt][3], fr.x, fr.y);
-            mma_tf32_z(dx, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.z, fr.w);
-          } else {
-            mma_tf32(dh, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.x, fr.y);
-            mma_tf32(dl, yl[0][jt][0], yl[0][jt][2], yl[0][jt][1], yl[0][jt][3], fr.x, fr.y);
-            mma_tf32(dx, yh[0][jt][0], yh[0][jt][2], yh[0][jt][1], yh[0][jt][3], fr.z, fr.w);
-          }
-          mma_tf32(dh, yh[1][jt][0], yh[1][jt][2], yh[1][jt][1], yh[1][jt][3], fi.x, fi.y);
-          mma_tf32(dl, yl[1][jt][0], yl[1][jt][2], yl[1][jt][1], yl[1][jt][3], fi.x, fi.y);
-          mma_tf32(dx, yh[1][jt][0], yh[1][jt][2], yh[1][jt][1], yh[1][jt][3], fi.z, fi.w);
+          const uint4 f = ubf[(nb * RBT + jt) * 32 + lane];
+          mma_f16(dh, yh[jt][0], yh[jt][1], yh[jt][2], yh[jt][3], f.x, f.y);
+          mma_f16(dl, yl[jt][0], yl[jt][1], yl[jt][2], yl[jt][3], f.x, f.y);
+          mma_f16(dl, yh[jt][0], yh[jt][1], yh[jt][2], yh[jt][3], f.z, f.w);
         }
+        float dx[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { dl[i] *= kF16LoInv; dx[i] = 0.f; }
         // d0 + i d1 = D[r0][b], d2 + i d3 = D[r1][b] with b = 16 (nb>>2) + (nb&3) + 4 t
         const int bo = 16 * (nb >> 2) + (nb & 3) + 4 * t;
         if (bo < B) {
