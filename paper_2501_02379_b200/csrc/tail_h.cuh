@@ -300,7 +300,7 @@ __global__ void __launch_bounds__(512, 1) proj_tail_h_kernel(const void* __restr
 struct TailHBGeom {
   int nwarps, nbuf, nbt, ks2;
   uint32_t slab_bytes, buf_stride;
-  uint32_t off_ub, off_ua, off_bar, total;
+  uint32_t off_ub, off_ua, off_ex, off_bar, total;
 };
 __host__ inline bool tail_hb_geom(int A, int B, int ra, int rb, TailHBGeom& g) {
   if (A % 16 || A < 16 || A > 128) return false;
@@ -312,11 +312,14 @@ __host__ inline bool tail_hb_geom(int A, int B, int ra, int rb, TailHBGeom& g) {
   g.slab_bytes = (uint32_t)A * B * 4;
   if (g.slab_bytes % 16) return false;
   g.buf_stride = (g.slab_bytes + 127) & ~127u;
-  const uint32_t ub = (uint32_t)g.nbt * rbt * 2 * 32 * 16, ua = (uint32_t)(A / 16) * g.ks2 * 2 * 32 * 16;
+  // operand tables in fp16 MMA register order (hi and lo parts), and the exchange buffer of the warp pairs
+  const uint32_t ub = (uint32_t)g.nbt * rbt * 32 * 16, ua = (uint32_t)(A / 16) * rat * 2 * 32 * 16;
+  const uint32_t ex = (uint32_t)g.nwarps * 32 * 32;
   g.nbuf = 3;
   g.off_ub = 3 * g.buf_stride;
   g.off_ua = g.off_ub + ub;
-  g.off_bar = g.off_ua + ua;
+  g.off_ex = g.off_ua + ua;
+  g.off_bar = g.off_ex + ex;
   g.total = g.off_bar + 256;
   return g.total <= 227u * 1024u;
 }
@@ -341,7 +344,8 @@ __global__ void __launch_bounds__(512, 1) back_tail_h_kernel(void* __restrict__ 
   const int mtile = warp >> 1, am = 16 * mtile, r0 = am + gq, r1 = r0 + 8;
   const int nbh = (nbt + 1) / 2, nb0 = (warp & 1) ? nbh : 0, nb1 = (warp & 1) ? nbt : nbh;   // this warp's column tiles
   uint4* ubf = reinterpret_cast<uint4*>(smem + G.off_ub);       // [nbt][RBT][32]: fp16 pairs (b0.hi, b1.hi, b0.lo, b1.lo)
-  float4* uaf = reinterpret_cast<float4*>(smem + G.off_ua);     // [A/16][KS2][hi|lo][32]
+  uint4* uaf = reinterpret_cast<uint4*>(smem + G.off_ua);       // [A/16][RAT][hi|lo][32]
+  uint4* exch = reinterpret_cast<uint4*>(smem + G.off_ex);      // [warps][32][2]: Y' fragments handed to the partner warp
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + G.off_bar);
   unsigned char* wb = static_cast<unsigned char*>(w);
 
@@ -364,17 +368,23 @@ __global__ void __launch_bounds__(512, 1) back_tail_h_kernel(void* __restrict__ 
     ubf[idx] = make_uint4(h2_bits(__halves2half2(h[0], h[1])), h2_bits(__halves2half2(h[2], h[3])),
                           h2_bits(__halves2half2(l[0], l[1])), h2_bits(__halves2half2(l[2], l[3])));
   }
-  // Ua as stage-1 operand fragments: rows am + g and am + g + 8, ja = 4 ks + t: (u0.x, u1.x, u0.y, u1.y) hi, then lo
-  for (int idx = tid; idx < (A / 16) * KS2 * 32; idx += nthr) {
-    const int mt = idx / (KS2 * 32), rem = idx - mt * (KS2 * 32), ks = rem >> 5, ln = rem & 31;
-    const int ja = 4 * ks + (ln & 3), q0 = 16 * mt + (ln >> 2), q1 = q0 + 8;
-    cf v0 = (ja < ra) ? p.Ua[q0 * ra + ja] : make_float2(0.f, 0.f);
-    cf v1 = (ja < ra) ? p.Ua[q1 * ra + ja] : make_float2(0.f, 0.f);
-    cf h0, l0, h1, l1;
-    split_tf32(v0.x, h0.x, l0.x); split_tf32(v0.y, h0.y, l0.y);
-    split_tf32(v1.x, h1.x, l1.x); split_tf32(v1.y, h1.y, l1.y);
-    uaf[((mt * KS2 + ks) * 2 + 0) * 32 + ln] = make_float4(h0.x, h1.x, h0.y, h1.y);
-    uaf[((mt * KS2 + ks) * 2 + 1) * 32 + ln] = make_float4(l0.x, l1.x, l0.y, l1.y);
+  // Ua as stage-1 operand fragments of the fp16 m16n8k16 shape, per row tile, step ks and lane (g, t): rows
+  // q0 = 16 mt + g and q0 + 8; k = 2t, 2t+1 <-> (ja, re), (ja+1, re), k = 2t+8, 2t+9 <-> (ja, im), (ja+1, im),
+  // ja = 8 ks + 2t:  a0 = re(q0), a1 = re(q0+8), a2 = im(q0), a3 = im(q0+8), each a pair over (ja, ja+1); hi, then lo
+  for (int idx = tid; idx < (A / 16) * RAT * 32; idx += nthr) {
+    const int mt = idx / (RAT * 32), rem = idx - mt * (RAT * 32), ks = rem >> 5, ln = rem & 31;
+    const int ja = 8 * ks + 2 * (ln & 3), q0 = 16 * mt + (ln >> 2), q1 = q0 + 8;
+    const cf z = make_float2(0.f, 0.f);
+    const cf u00 = (ja < ra) ? p.Ua[q0 * ra + ja] : z, u01 = (ja + 1 < ra) ? p.Ua[q0 * ra + ja + 1] : z;
+    const cf u10 = (ja < ra) ? p.Ua[q1 * ra + ja] : z, u11 = (ja + 1 < ra) ? p.Ua[q1 * ra + ja + 1] : z;
+    const float v[8] = {u00.x, u01.x, u10.x, u11.x, u00.y, u01.y, u10.y, u11.y};
+    __half h[8], l[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) split_f16_scaled(v[e], h[e], l[e]);
+    uaf[((mt * RAT + ks) * 2 + 0) * 32 + ln] = make_uint4(h2_bits(__halves2half2(h[0], h[1])), h2_bits(__halves2half2(h[2], h[3])),
+                                                          h2_bits(__halves2half2(h[4], h[5])), h2_bits(__halves2half2(h[6], h[7])));
+    uaf[((mt * RAT + ks) * 2 + 1) * 32 + ln] = make_uint4(h2_bits(__halves2half2(l[0], l[1])), h2_bits(__halves2half2(l[2], l[3])),
+                                                          h2_bits(__halves2half2(l[4], l[5])), h2_bits(__halves2half2(l[6], l[7])));
   }
   if (tid == 0) {
     for (int i = 0; i < nbuf; ++i) mbar_init(&bars[i], 1);
@@ -404,17 +414,22 @@ __global__ void __launch_bounds__(512, 1) back_tail_h_kernel(void* __restrict__ 
   for (uint32_t it = 0; it < nmine; ++it) {
     const uint32_t s = blockIdx.x + it * gstride;
     if (tid == 0) bulk_wait_read<1>();          // the store of two iterations ago has read its buffer
-    // T' fragments for stage 1 (in flight while the slab arrives): T'[ja = 4 ks + t][jb = 8 jt + gq]
-    cf tv[KS2][RBT];
+    // T' fragments for stage 1 (in flight while the slab arrives): T'[ja = 8 ks + 2t + e][jb = 8 jt + gq], e = 0, 1,
+    // for the jb tiles this warp computes: with two jb tiles the two warps of a row tile take one each
+    constexpr int NJ = (RBT == 2) ? 1 : RBT;          // jb tiles whose stage 1 this warp computes
+    const int jt0 = (RBT == 2) ? (warp & 1) : 0;
+    cf tv[RAT][NJ][2];
     {
       const cf* tin = p.t + (size_t)s * ra * rb;
 #pragma unroll
-      for (int ks = 0; ks < KS2; ++ks)
+      for (int ks = 0; ks < RAT; ++ks)
 #pragma unroll
-        for (int jt = 0; jt < RBT; ++jt) {
-          const int ja = 4 * ks + t, jb = 8 * jt + gq;
-          tv[ks][jt] = (ja < ra && jb < rb) ? __ldg(tin + (size_t)ja * rb + jb) : make_float2(0.f, 0.f);
-        }
+        for (int j = 0; j < NJ; ++j)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int ja = 8 * ks + 2 * t + e, jb = 8 * (jt0 + j) + gq;
+            tv[ks][j][e] = (ja < ra && jb < rb) ? __ldg(tin + (size_t)ja * rb + jb) : make_float2(0.f, 0.f);
+          }
     }
     const bool ok = mbar_wait_bounded(&bars[buf], phase);
     if (__syncthreads_or(!ok)) {
@@ -427,46 +442,76 @@ __global__ void __launch_bounds__(512, 1) back_tail_h_kernel(void* __restrict__ 
     }
     uint32_t* ws = reinterpret_cast<uint32_t*>(smem + (size_t)buf * G.buf_stride);     // half2 words [A][B]
     {
-      // ---- stage 1: Y'[a][(c, jb)] for rows r0 and r1 ----
-      float d1[2][RBT][4];
+      // ---- stage 1: Y'[a][(c, jb)] for rows r0 and r1, fp16 m16n8k16 on two-term splits of both operands
+      //      (re tile: B = (Tr | -Ti), im tile: B = (Ti | Tr); hi hi into one accumulator, lo hi and hi lo, which
+      //      carry the factor 2048, into another) ----
+      float d1[2][NJ][4];
 #pragma unroll
-      for (int c = 0; c < 2; ++c)
+      for (int j = 0; j < NJ; ++j) {
+        float eh[2][4], el[2][4];
 #pragma unroll
-        for (int jt = 0; jt < RBT; ++jt)
+        for (int c = 0; c < 2; ++c)
 #pragma unroll
-          for (int i = 0; i < 4; ++i) d1[c][jt][i] = 0.f;
+          for (int i = 0; i < 4; ++i) { eh[c][i] = 0.f; el[c][i] = 0.f; }
 #pragma unroll
-      for (int ks = 0; ks < KS2; ++ks) {
-        const float4 uh = uaf[((mtile * KS2 + ks) * 2 + 0) * 32 + lane], ul = uaf[((mtile * KS2 + ks) * 2 + 1) * 32 + lane];
-#pragma unroll
-        for (int jt = 0; jt < RBT; ++jt) {
-          float trh, trl, tih, til;
-          split_tf32(tv[ks][jt].x, trh, trl); split_tf32(tv[ks][jt].y, tih, til);
-          // A = (Ua[r0].re, Ua[r1].re, Ua[r0].im, Ua[r1].im);  re tile: B = (Tr, -Ti);  im tile: B = (Ti, Tr)
-          mma_tf32(d1[0][jt], uh.x, uh.y, uh.z, uh.w, trh, -tih);
-          mma_tf32(d1[0][jt], ul.x, ul.y, ul.z, ul.w, trh, -tih);
-          mma_tf32(d1[0][jt], uh.x, uh.y, uh.z, uh.w, trl, -til);
-          mma_tf32(d1[1][jt], uh.x, uh.y, uh.z, uh.w, tih, trh);
-          mma_tf32(d1[1][jt], ul.x, ul.y, ul.z, ul.w, tih, trh);
-          mma_tf32(d1[1][jt], uh.x, uh.y, uh.z, uh.w, til, trl);
+        for (int ks = 0; ks < RAT; ++ks) {
+          const uint4 uh = uaf[((mtile * RAT + ks) * 2 + 0) * 32 + lane], ul = uaf[((mtile * RAT + ks) * 2 + 1) * 32 + lane];
+          const cf t0 = tv[ks][j][0], t1 = tv[ks][j][1];
+          const __half2 rh = __floats2half2_rn(t0.x, t1.x), ih = __floats2half2_rn(t0.y, t1.y);
+          const float2 rb_ = __half22float2(rh), ib_ = __half22float2(ih);
+          const __half2 rl = __floats2half2_rn((t0.x - rb_.x) * kF16LoScale, (t1.x - rb_.y) * kF16LoScale);
+          const __half2 il = __floats2half2_rn((t0.y - ib_.x) * kF16LoScale, (t1.y - ib_.y) * kF16LoScale);
+          const uint32_t trh = h2_bits(rh), tih = h2_bits(ih), trl = h2_bits(rl), til = h2_bits(il);
+          const uint32_t nih = tih ^ 0x80008000u, nil = til ^ 0x80008000u;        // -Ti
+          mma_f16(eh[0], uh.x, uh.y, uh.z, uh.w, trh, nih);
+          mma_f16(el[0], ul.x, ul.y, ul.z, ul.w, trh, nih);
+          mma_f16(el[0], uh.x, uh.y, uh.z, uh.w, trl, nil);
+          mma_f16(eh[1], uh.x, uh.y, uh.z, uh.w, tih, trh);
+          mma_f16(el[1], ul.x, ul.y, ul.z, ul.w, tih, trh);
+          mma_f16(el[1], uh.x, uh.y, uh.z, uh.w, til, trl);
         }
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) d1[c][j][i] = eh[c][i] + el[c][i] * kF16LoInv;
       }
       // Y' as fp16 m16n8k16 A fragments, hi and lo (scaled by 2048): a0 = (row g; jb, jb+1; re), a1 = (row g+8; re),
       // a2 = (row g; im), a3 = (row g+8; im) -- the accumulator pairs of stage 1 as they are.  Y' is built from the
       // Adam-normalised core through factors with orthonormal columns, so its entries are far inside the fp16 range.
-      uint32_t yh[RBT][4], yl[RBT][4];
+      uint32_t ymh[NJ][4], yml[NJ][4];                 // of the jb tiles this warp computed
 #pragma unroll
-      for (int jt = 0; jt < RBT; ++jt)
+      for (int j = 0; j < NJ; ++j)
 #pragma unroll
         for (int c = 0; c < 2; ++c)
 #pragma unroll
           for (int hrow = 0; hrow < 2; ++hrow) {
-            const float v0 = d1[c][jt][2 * hrow], v1 = d1[c][jt][2 * hrow + 1];
+            const float v0 = d1[c][j][2 * hrow], v1 = d1[c][j][2 * hrow + 1];
             const __half2 hh = __floats2half2_rn(v0, v1);
             const float2 back = __half22float2(hh);
-            yh[jt][2 * c + hrow] = h2_bits(hh);
-            yl[jt][2 * c + hrow] = h2_bits(__floats2half2_rn((v0 - back.x) * kF16LoScale, (v1 - back.y) * kF16LoScale));
+            ymh[j][2 * c + hrow] = h2_bits(hh);
+            yml[j][2 * c + hrow] = h2_bits(__floats2half2_rn((v0 - back.x) * kF16LoScale, (v1 - back.y) * kF16LoScale));
           }
+      uint32_t yh[RBT][4], yl[RBT][4];
+      if (RBT == 2) {
+        // hand this warp's jb tile to the partner warp of the row tile and take the partner's (one named barrier per
+        // pair of warps; the block barrier further down keeps the next iteration's writes behind these reads)
+        exch[(warp * 32 + lane) * 2 + 0] = make_uint4(ymh[0][0], ymh[0][1], ymh[0][2], ymh[0][3]);
+        exch[(warp * 32 + lane) * 2 + 1] = make_uint4(yml[0][0], yml[0][1], yml[0][2], yml[0][3]);
+        asm volatile("barrier.sync %0, 64;" ::"r"(1 + mtile) : "memory");
+        const uint4 oh = exch[((warp ^ 1) * 32 + lane) * 2 + 0], ol = exch[((warp ^ 1) * 32 + lane) * 2 + 1];
+        const uint32_t oth[4] = {oh.x, oh.y, oh.z, oh.w}, otl[4] = {ol.x, ol.y, ol.z, ol.w};
+        const bool second = (warp & 1) != 0;           // this warp computed jb tile 1
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          yh[0][i] = second ? oth[i] : ymh[0][i]; yh[RBT - 1][i] = second ? ymh[0][i] : oth[i];
+          yl[0][i] = second ? otl[i] : yml[0][i]; yl[RBT - 1][i] = second ? yml[0][i] : otl[i];
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < NJ; ++j)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) { yh[j][i] = ymh[j][i]; yl[j][i] = yml[j][i]; }
+      }
       // ---- stage 2, one column tile at a time, applied to the slab right away: three fp16 products per jb tile
       //      (hi hi, lo hi, hi lo), the two small ones summed and scaled back by 1/2048 ----
       constexpr int NB_UNROLL = NBT ? (NBT + 1) / 2 : 1;
