@@ -4,8 +4,9 @@
 // A slab arrives by one bulk asynchronous copy as it is stored (fp16), and stays fp16 in shared memory.
 // fp16 values are exact fp16 MMA operands, so the first trailing-mode product needs no splitting of the
 // streamed operand at all: Y = X conj(Ub) is two m16n8k16 MMAs per step (Ub = hi + lo in fp16, X exact),
-// at twice the K per instruction of the TF32 shape.  The second product (over the slab rows) and the
-// reconstruction run as split-precision TF32 like the fp32-storage kernels.
+// at twice the K per instruction of the TF32 shape.  The second product of the compression (over the slab rows, whose
+// operand carries the gradient's scale) runs as split-precision TF32 like the fp32-storage kernels; the two products
+// of the reconstruction run as fp16 MMAs on two-term splits (see back_tail_h_kernel).
 //
 // A block has one warp per tile of 8 slab rows (A/8 warps, at most 16) and works on one slab at a time
 // from a ring of bulk copies; one block per SM.
@@ -231,11 +232,11 @@ __global__ void __launch_bounds__(512, 1) proj_tail_h_kernel(const void* __restr
     if (it < nmine) {
       const uint32_t* xs = reinterpret_cast<const uint32_t*>(smem + (size_t)buf * G.buf_stride);
       const uint32_t* xrow = xs + (size_t)(8 * warp + gq) * B;
-      float d[RBT][4];
+      float d[RBT][4], dlo[RBT][4];        // the hi and lo parts of Ub accumulate apart: two short chains instead of one
 #pragma unroll
       for (int jt = 0; jt < RBT; ++jt)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) d[jt][i] = 0.f;
+        for (int i = 0; i < 4; ++i) { d[jt][i] = 0.f; dlo[jt][i] = 0.f; }
       for (int ks = 0; ks < ks16; ++ks) {
         const int c1_ = 32 * (ks >> 2) + 8 * t + (ks & 3), c2_ = c1_ + 4;
         const uint32_t x1 = c1_ < B ? xrow[c1_] : 0u, x2 = c2_ < B ? xrow[c2_] : 0u;
@@ -243,9 +244,13 @@ __global__ void __launch_bounds__(512, 1) proj_tail_h_kernel(const void* __restr
         for (int jt = 0; jt < RBT; ++jt) {
           const uint4 h = u1tab[((ks * RBT + jt) * 2 + 0) * 32 + lane], l = u1tab[((ks * RBT + jt) * 2 + 1) * 32 + lane];
           mma_f16(d[jt], h.x, h.y, h.z, h.w, x1, x2);
-          mma_f16(d[jt], l.x, l.y, l.z, l.w, x1, x2);
+          mma_f16(dlo[jt], l.x, l.y, l.z, l.w, x1, x2);
         }
       }
+#pragma unroll
+      for (int jt = 0; jt < RBT; ++jt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) d[jt][i] += dlo[jt][i];
       // d0 = Yre[a][jb], d1 = Yre[a+1][jb], d2 = Yim[a][jb], d3 = Yim[a+1][jb], a = 8 warp + 2t, jb = 8 jt + gq
       cf* ys = ysb + (size_t)(it & 1) * A * ldy;
 #pragma unroll
@@ -261,7 +266,7 @@ __global__ void __launch_bounds__(512, 1) proj_tail_h_kernel(const void* __restr
       const int steps = (A / 4) / ksplit;
       for (int unit = warp; unit < units; unit += nwarps) {
         const int tile = unit / ksplit, kh = unit - tile * ksplit, mt = tile / RBT, nt = tile - mt * RBT;
-        float tot[4] = {0.f, 0.f, 0.f, 0.f}, acc[4] = {0.f, 0.f, 0.f, 0.f};
+        float tot[4] = {0.f, 0.f, 0.f, 0.f}, acc[4] = {0.f, 0.f, 0.f, 0.f}, acl[4] = {0.f, 0.f, 0.f, 0.f}, acx[4] = {0.f, 0.f, 0.f, 0.f};
         for (int q = 0; q < steps; ++q) {
           const int a = 4 * (kh * steps + q) + t;
           const cf y = ys[a * ldy + 8 * nt + gq], u = uas[a * ldu + 8 * mt + gq];
@@ -269,16 +274,17 @@ __global__ void __launch_bounds__(512, 1) proj_tail_h_kernel(const void* __restr
           split_tf32(y.x, yh0, yl0); split_tf32(y.y, yh1, yl1);
           split_tf32(u.x, urh, url); split_tf32(u.y, uih, uil);
           // rows (re, ja): (ur | ui); rows (im, ja): (-ui | ur)
+          // the three products keep their own accumulators: three independent chains
           mma_tf32(acc, urh, -uih, uih, urh, yh0, yh1);
-          mma_tf32(acc, url, -uil, uil, url, yh0, yh1);
-          mma_tf32(acc, urh, -uih, uih, urh, yl0, yl1);
-          if ((q & 7) == 7) {      // the tensor core's accumulator adds truncate: keep its chains short
+          mma_tf32(acl, url, -uil, uil, url, yh0, yh1);
+          mma_tf32(acx, urh, -uih, uih, urh, yl0, yl1);
+          if ((q & 15) == 15) {    // the tensor core's accumulator adds truncate: keep its chains short
 #pragma unroll
-            for (int i = 0; i < 4; ++i) { tot[i] += acc[i]; acc[i] = 0.f; }
+            for (int i = 0; i < 4; ++i) { tot[i] += acc[i] + (acl[i] + acx[i]); acc[i] = 0.f; acl[i] = 0.f; acx[i] = 0.f; }
           }
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) tot[i] += acc[i];
+        for (int i = 0; i < 4; ++i) tot[i] += acc[i] + (acl[i] + acx[i]);
         *reinterpret_cast<float4*>(pw + (size_t)unit * 128 + lane * 4) = make_float4(tot[0], tot[1], tot[2], tot[3]);
       }
     }
@@ -291,8 +297,11 @@ __global__ void __launch_bounds__(512, 1) proj_tail_h_kernel(const void* __restr
 
 // ---------------------------------------------------------------------------------------------
 // Reconstruction of the two trailing modes (half storage), fused with the weight update and the sparse add.
-// Two warps share a tile of 16 rows of the slab (each takes half of the column tiles); the products are the
-// split-TF32 ones of back_tail_tc_kernel, with the Ua and Ub fragments in shared-memory tables.  The slab
+// Two warps share a tile of 16 rows of the slab: each computes the first product for one of the two jb tiles and
+// hands its fragments to the other, and each takes half of the column tiles of the second product.  Both products
+// run as fp16 m16n8k16 MMAs on two-term fp16 splits of both operands (x = hi + lo / 2048; hi hi, lo hi, hi lo: 22
+// bits, the accuracy of the split-TF32 products at half the instructions): the operands here are the factor
+// matrices (|u| <= 1) and the expansion of the Adam-normalised core, both far inside the fp16 range.  The slab
 // stays fp16 in shared memory: the dense update is rounded to fp16 when it is written back there, the
 // sparse term is then added by one thread per entry and rounded again (the storage type is rounded to once after the dense update and once more at Omega),
 // and one bulk copy stores the slab.
