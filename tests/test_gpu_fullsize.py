@@ -65,6 +65,20 @@ def test_cfg4_full_oracle_steps_across_a_scheduled_refresh():
     _schedule_run("cfg4", [0])
 
 
+@pytest.mark.parametrize("kw", [dict(hooi_iters=1), dict(composition="lr_us"),
+                                dict(composition="sum", strategy="probk", seed=77)],
+                         ids=["hooi", "lr_us", "sum_probk"])
+def test_cfg3_variants_full_oracle_steps(kw):
+    # the options beyond Algorithm 1's defaults at the size of the benchmark configuration: one refinement sweep of the
+    # factors; low rank first (Omega from G - P_U(G)); both parts on the gradient with probability-k selection (whose
+    # 34.6 M keys must come out bit-identical on both sides).  A refresh step and a plain step each, every output compared.
+    wl = synth.WORKLOADS["cfg3"]
+    p = Pair(wl, **kw)
+    p.step(0)
+    p.step(1)
+    print("cfg3", kw, {k: v for k, v in p.report.items() if k in ("angle", "core", "m_s", "w@1e-3", "omega_boundary_entries")})
+
+
 def test_cfg5_whole_slabs_and_full_core():
     wl = synth.WORKLOADS["cfg5"]
     t0 = time.time()
