@@ -210,6 +210,8 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, 4) proj_tail_tc_kernel(const vo
     }
   }
 
+  // the last column's factor row for the FMA path of an odd KS: Ub[B-1][gq]
+  const cf ulast = ((KS & 1) && gq < rb) ? p.Ub[(size_t)(B - 1) * rb + gq] : make_float2(0.f, 0.f);
   if (tid == 0) {
     for (int i = 0; i < nbuf; ++i) mbar_init(&bars[i], 1);
     fence_mbar_init();
@@ -312,8 +314,11 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, 4) proj_tail_tc_kernel(const vo
       // stage 1 for the warp's NTW row tiles together: one Ub fragment load serves them all
       const float* xrow = xg + (size_t)q * (2 * E) + (size_t)(8 * wt + gq) * twoB;
       float dh[NTW][4], dl[NTW][4], dx[NTW][4];
+      // An odd KS means a last k-step that holds the column b = B - 1 alone (a quarter of an MMA's K range): that
+      // column is added with fp32 FMAs below instead, on the accumulator entries this lane owns.
+      constexpr int KSM = (KS & 1) ? KS - 1 : KS;
 #pragma unroll
-      for (int ks = 0; ks < KS; ++ks) {
+      for (int ks = 0; ks < KSM; ++ks) {
         // Where a lane's float offset f lies past the row (the table holds zeros there) it reads the row's last
         // entry instead: finite data, no predicate.  KS odd means B = 4 (KS - 1) + 1: every step but the last is
         // whole, the last holds b = B - 1 alone.  KS == 8 means 16 <= B <= 32: the first four steps are whole.
@@ -344,8 +349,16 @@ __global__ void __launch_bounds__(32 * PJ_WARPS, 4) proj_tail_tc_kernel(const vo
       for (int nt = 0; nt < NTW; ++nt) {
         // Y fragments: [0] Yre[a][jb], [1] Yre[a+1][jb], [2] Yim[a][jb], [3] Yim[a+1][jb], a = 8 tile + 2t, jb = gq
         float yh[4], yl[4];
+        float ex[4] = {0.f, 0.f, 0.f, 0.f};
+        if (KS & 1) {
+          // Y[a][jb] += x[a][B-1] conj(Ub[B-1][jb]) for a = 8 tile + 2t, + 1 and jb = gq
+          const float* xa = xg + (size_t)q * (2 * E) + (size_t)(8 * (wt + nt * tw) + 2 * t) * twoB + (twoB - 2);
+          const float2 x0 = *reinterpret_cast<const float2*>(xa), x1 = *reinterpret_cast<const float2*>(xa + twoB);
+          ex[0] = fmaf(x0.x, ulast.x, x0.y * ulast.y); ex[1] = fmaf(x1.x, ulast.x, x1.y * ulast.y);
+          ex[2] = fmaf(x0.y, ulast.x, -x0.x * ulast.y); ex[3] = fmaf(x1.y, ulast.x, -x1.x * ulast.y);
+        }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) split_tf32(dh[nt][i] + (dl[nt][i] + dx[nt][i]), yh[i], yl[i]);
+        for (int i = 0; i < 4; ++i) split_tf32((dh[nt][i] + ex[i]) + (dl[nt][i] + dx[nt][i]), yh[i], yl[i]);
 #pragma unroll
         for (int mt = 0; mt < RAT; ++mt) {
           // (x, y, -y) of u0.hi, u1.hi, u0.lo, u1.lo with u0 = Ua[a][ja], u1 = Ua[a+1][ja]
