@@ -43,6 +43,12 @@ constexpr int SUB_THREADS = 1024;
 constexpr int SUB_MAX_N = 256;            // rows of Q that fit beside the small matrices in shared memory
 constexpr int SUB_MAX_R = 80;
 constexpr int SUB_MAX_IT = 12;            // outer iterations (each up to SUB_MAX_DEG multiplications by A) before giving up
+// Unsigned key that orders like the float, with every NaN below -inf.
+__device__ __forceinline__ uint32_t sub_order_key(float x) {
+  const uint32_t u = __float_as_uint(x);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return 0u;
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
 constexpr int SUB_MAX_DEG = 7;            // highest degree of the polynomial filter
 constexpr float SUB_MAX_GROWTH = 1e6f;    // cap on the filter's amplification of the largest eigenvalue (fp32 range of a column)
 constexpr float SUB_TOL = 1e-4f;          // bound on the sine of the largest angle to the invariant subspace
@@ -586,10 +592,12 @@ __global__ void __launch_bounds__(SUB_THREADS, 1) subspace_kernel(SubspaceParams
       // ---- Ritz values in descending order (ties: lower index first) ----
       for (int i = tid; i < R; i += SUB_THREADS) theta[i] = Hm[(size_t)i * ld + i].x;
       __syncthreads();
+      // (compared through sub_order_key: a strict total order even with NaN among the values, so that the ranks
+      // are a permutation and every order[] entry is written)
       for (int i = tid; i < R; i += SUB_THREADS) {
-        const float li = theta[i];
+        const uint32_t li = sub_order_key(theta[i]);
         int rk = 0;
-        for (int j = 0; j < R; ++j) { const float lj = theta[j]; rk += (lj > li) || (lj == li && j < i); }
+        for (int j = 0; j < R; ++j) { const uint32_t lj = sub_order_key(theta[j]); rk += (lj > li) || (lj == li && j < i); }
         order[rk] = i;
       }
       __syncthreads();

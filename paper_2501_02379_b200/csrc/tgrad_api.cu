@@ -11,6 +11,7 @@
 #include "../../include/tgrad.h"
 #include "common.cuh"
 #include "gram.cuh"
+#include "gram_tc.cuh"
 #include "jacobi.cuh"
 #include "modeprod.cuh"
 #include "select.cuh"
@@ -113,6 +114,33 @@ void plan_gram(const tgrad_config* c, int n, int sm, uint32_t& chunks, uint32_t&
   plan_gram_dims((int)c->dims[n], O, C, sm, chunks, cps, splits);
 }
 
+// Plan of the tcgen05 Gram kernel for a tensor seen as [O][In][C] with entries of `ebytes` bytes; ok = false when the
+// shape does not suit it (rows that are not 16-byte multiples or too short for 128-byte tiles, a short contraction
+// that wants the split-precision products, fewer than 64 or more than 256 rows) and the mma.sync kernel runs instead.
+struct GramTcPlan { bool ok; int rows, stages, mtiles, splits; uint32_t tiles_per_o, tiles_total, per; };
+constexpr int kGramTcMaxBlocks = 148;     // upper bound of splits x row tiles, whatever the device: sizes the scratch
+GramTcPlan plan_gram_tc(int In, uint64_t O, uint64_t C, int ebytes, int sm) {
+  GramTcPlan pl; memset(&pl, 0, sizeof(pl));
+  const uint64_t run = C * (uint64_t)ebytes;           // bytes of one row's contiguous run
+  if (In < GT_MIN_ROWS || In > GT_MAX_ROWS || run % 16 != 0 || run < 512 || O * C < 16384) return pl;
+  const uint64_t per_o = (run + GT_ROW_BYTES - 1) / GT_ROW_BYTES, total = O * per_o;
+  if (O >= (1ull << 31) || 2 * C >= (1ull << 32) || total >= (1ull << 32) || (uint64_t)In * run >= (1ull << 40)) return pl;
+  pl.rows = (In + 15) / 16 * 16;
+  pl.mtiles = pl.rows > 128 ? 2 : 1;
+  const size_t stage = (size_t)2 * pl.rows * GT_ROW_BYTES;
+  pl.stages = (int)((size_t)(200 << 10) / stage);
+  if (pl.stages > GT_MAX_STAGES) pl.stages = GT_MAX_STAGES;
+  if (sm > kGramTcMaxBlocks) sm = kGramTcMaxBlocks;
+  uint64_t want = (uint64_t)(sm / pl.mtiles);
+  if (want < 1) want = 1;
+  if (want > total) want = total;
+  const uint64_t per = (total + want - 1) / want;
+  pl.tiles_per_o = (uint32_t)per_o; pl.tiles_total = (uint32_t)total; pl.per = (uint32_t)per;
+  pl.splits = (int)((total + per - 1) / per);
+  pl.ok = true;
+  return pl;
+}
+
 // The configuration the kernels see.  A matrix (N = 2, where the Tucker decomposition is the matrix SVD) is handled as
 // the 3-way tensor I_1 x 1 x I_2 with ranks (r_1, 1, r_2): the unit mode's factor is the 1 x 1 identity, so every
 // stage computes exactly what Algorithm 1 computes for the matrix.  map[n] = internal mode of the caller's mode n.
@@ -182,6 +210,8 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
     plan_gram(c, n, sm, L.gram_chunks[n], L.gram_cps[n], L.gram_splits[n]);
     size_t pb = sq * L.gram_splits[n];
     if (pb > partial) partial = pb;
+    // the tcgen05 kernel (64..256 rows) writes at most this many partial matrices, whatever tensor it is given
+    if (c->dims[n] >= GT_MIN_ROWS && c->dims[n] <= GT_MAX_ROWS && sq * kGramTcMaxBlocks > partial) partial = sq * kGramTcMaxBlocks;
   }
   L.w_partial = o; o = align_up(o + partial);
   // refinement sweeps: two buffers for the tensor compressed in all modes but one, and an identity matrix that
@@ -458,10 +488,59 @@ tgrad_status build_slab_ptr(tgrad_state* s, cudaStream_t st) {
 tgrad_status mode_product(bool conj_t, const cf* in, cf* out, const cf* U, uint64_t O, int M, int K, uint64_t C,
                           int r_n, int sm_count, cudaStream_t st);
 
+// cuTensorMapEncodeTiled, fetched through the runtime so that the library does not link against the driver.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess) return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+template <class S> struct GramTcFmt;
+template <> struct GramTcFmt<StoreC64> { static constexpr int fmt = 2; static constexpr CUtensorMapDataType dt = CU_TENSOR_MAP_DATA_TYPE_FLOAT32; };
+template <> struct GramTcFmt<StoreC32H> { static constexpr int fmt = 0; static constexpr CUtensorMapDataType dt = CU_TENSOR_MAP_DATA_TYPE_FLOAT16; };
+template <> struct GramTcFmt<StoreC32B> { static constexpr int fmt = 1; static constexpr CUtensorMapDataType dt = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16; };
+
+// The same on the tcgen05 kernel: a rank-3 tensor map (2C reals, In rows, O blocks) over this GPU's own memory.
+template <class S>
+tgrad_status launch_gram_tc(tgrad_state* s, const void* x, int In, uint64_t O, uint64_t C, const GramTcPlan& pl, cf* A,
+                            cudaStream_t st) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return TGRAD_ERR_CUDA;
+  constexpr int fmt = GramTcFmt<S>::fmt;
+  const uint64_t real_bytes = S::kBytes / 2;
+  CUtensorMap tm;
+  const cuuint64_t dims[3] = {2 * C, (cuuint64_t)In, O};
+  const cuuint64_t strides[2] = {C * S::kBytes, (cuuint64_t)In * C * S::kBytes};
+  const cuuint32_t box[3] = {(cuuint32_t)(GT_ROW_BYTES / real_bytes), (cuuint32_t)pl.rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  if (enc(&tm, GramTcFmt<S>::dt, 3, const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return TGRAD_ERR_CUDA;
+  GramTcParams gp;
+  gp.In = In; gp.rows = pl.rows; gp.stages = pl.stages; gp.tiles_per_o = pl.tiles_per_o; gp.tiles_total = pl.tiles_total;
+  gp.tiles_per_split = pl.per; gp.group_tiles = 32; gp.partial = reinterpret_cast<cf*>(s->dw + s->L.w_partial);
+  gp.flags = reinterpret_cast<int*>(s->dp + s->L.p_flags);
+  size_t smem = gram_tc_smem(pl.rows, pl.stages);
+  if (smem < ((size_t)120 << 10)) smem = (size_t)120 << 10;   // one block per SM: each takes all of the tensor memory
+  gram_tc_kernel<fmt><<<dim3(pl.splits, pl.mtiles), GT_THREADS, smem, st>>>(tm, gp); TG_LAUNCH_CHECK();
+  gram_reduce_kernel<<<(In * In + GRR_E - 1) / GRR_E, GRR_E * GRR_G, 0, st>>>(gp.partial, pl.splits, In, A); TG_LAUNCH_CHECK();
+  return TGRAD_OK;
+}
+
 // A = X_(n) X_(n)^H for a tensor seen as [O][In][C] (storage S), split-K partial sums reduced in a fixed order.
 template <class S>
 tgrad_status launch_gram(tgrad_state* s, const void* x, int In, uint64_t O, uint64_t C, uint32_t chunks, uint32_t cps,
                          int splits, cf* A, cudaStream_t st) {
+  const GramTcPlan pl = plan_gram_tc(In, O, C, S::kBytes, s->sm_count);
+  if (pl.ok && (reinterpret_cast<uintptr_t>(x) & 15) == 0) return launch_gram_tc<S>(s, x, In, O, C, pl, A, st);
   cf* partial = reinterpret_cast<cf*>(s->dw + s->L.w_partial);
   const int T = (In + GR_T - 1) / GR_T;
   dim3 grid(T * T, splits);
@@ -1101,6 +1180,9 @@ tgrad_status tgrad_init_state(const tgrad_config* cfg, void* d_persistent, size_
     TG_GRAM_ATTR(StoreC32B, false, false); TG_GRAM_ATTR(StoreC32B, false, true);
     TG_GRAM_ATTR(StoreC32B, true, false); TG_GRAM_ATTR(StoreC32B, true, true);
 #undef TG_GRAM_ATTR
+    ok = ok && cudaFuncSetAttribute(gram_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemMax - 1024)) == cudaSuccess;
+    ok = ok && cudaFuncSetAttribute(gram_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemMax - 1024)) == cudaSuccess;
+    ok = ok && cudaFuncSetAttribute(gram_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemMax - 1024)) == cudaSuccess;
     if (!ok) { delete st; return TGRAD_ERR_CUDA; }
   }
   if (cfg->dims[0] <= SW_MAX_I && cfg->ranks[0] <= SW_MAX_R &&

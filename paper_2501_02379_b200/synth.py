@@ -111,6 +111,14 @@ WORKLOADS: Dict[str, Workload] = {
                  outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.02),
         Workload("tail19", 101, (5, 6, 16, 19), (3, 3, 4, 3), (1, 50), 3, 5,
                  outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.05),
+        # leading modes with long contiguous rows and 64..256 entries (the tcgen05 Gram kernel): two 128-row tiles of
+        # the Gram matrix, fp16 storage with a row count that is not a multiple of 16, and an odd row count
+        Workload("gram144", 103, (144, 40, 32, 17), (8, 6, 6, 4), (1, 50), 3, 5,
+                 outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.02),
+        Workload("gram96h", 104, (96, 72, 32, 17), (8, 6, 6, 4), (1, 100), 3, 5,
+                 outlier_frac=(1, 200), outlier_scale=20.0, noise_scale=0.02, half_storage=True),
+        Workload("gram75", 105, (75, 64, 32, 16), (6, 8, 6, 4), (1, 50), 3, 5,
+                 outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.02),
         # the matrix case (N = 2)
         Workload("mat2", 102, (96, 80), (12, 10), (1, 50), 3, 7,
                  outlier_frac=(1, 100), outlier_scale=20.0, noise_scale=0.02),

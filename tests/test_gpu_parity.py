@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("name", ["tiny4", "small4", "small5", "ragged4", "small3", "odd4", "odd32", "small5b",
-                                  "half65", "lead200", "lead300", "tail19"])
+                                  "half65", "lead200", "lead300", "tail19", "gram144", "gram96h", "gram75"])
 def test_trajectory_small(name):
     wl = synth.WORKLOADS[name]
     p = Pair(wl)
@@ -180,11 +180,11 @@ def test_half_storage_small(name):
     print("half", name, p.report)
 
 
-@pytest.mark.parametrize("name", ["ragged4", "odd32", "small3"])
+@pytest.mark.parametrize("name", ["ragged4", "odd32", "small3", "gram96h"])
 def test_bf16_storage_small(name):
     # bfloat16-stored W and G (the other reading of the mixed recipe's "half precision"): general kernels
     import dataclasses
-    wl = dataclasses.replace(synth.WORKLOADS[name], bf16_storage=True)
+    wl = dataclasses.replace(synth.WORKLOADS[name], bf16_storage=True, half_storage=False)
     p = Pair(wl)
     for t in range(wl.T + 2):
         p.step(t)
