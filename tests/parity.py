@@ -18,6 +18,7 @@ from tests import helpers as H
 TOL_FLOAT = 1e-4       # max relative error, entries measured against max(|ref|, 2^-7 rms(ref)); see helpers.rel_err
 TOL_FRO = 5e-6         # and the whole array: ||a - b||_F / ||b||_F (split-TF32 products carry 2^-21 relative error
                        # each, and an entry passes through up to 2 N of them)
+TOL_GRAM = 2e-4        # largest entry error of a Gram matrix over its largest diagonal entry
 TOL_ANGLE = 1e-3       # largest principal-angle sine of a refreshed factor
 TOL_ORTHO = 1e-5       # max |U^H U - I|
 
@@ -113,6 +114,18 @@ class Pair:
         lr_first = self.ocfg.composition == "lr_us"
         if not lr_first:
             assert np.array_equal(om, self.ost.omega), "Omega differs from the oracle"
+        if self.ocfg.composition == "us_lr" and self.ocfg.hooi_iters == 0 and self.ocfg.strategy == "topk":
+            # the Gram matrices themselves, entry by entry, against the definition R_(n) R_(n)^H in complex128
+            # (fp32 storage: TF32 inputs on the long contractions, hence 2e-4 of the largest diagonal entry)
+            res = orc.residual(g, self.ost.omega).astype(np.complex128)
+            for n in range(len(self.wl.shape)):
+                want = orc.mode_gram(res, n)
+                got = self.gst.export(B.WHAT_GRAM_BASE + n).astype(np.complex128)
+                scale = float(np.abs(np.diag(want)).max())
+                if scale > 0:
+                    e = float(np.abs(got - want).max() / scale)
+                    self._note("gram", e)
+                    assert e <= TOL_GRAM, f"mode {n}: Gram matrix off by {e} of its largest diagonal entry"
         us = self.gst.factors()
         for n, (ug, uo) in enumerate(zip(us, self.ost.factors)):
             ang = H.max_sin_angle(ug, uo)
