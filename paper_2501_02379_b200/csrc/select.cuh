@@ -1,7 +1,7 @@
 // Magnitude top-k selection of the sparse index set Omega
 // (SparseIndices with the top-k strategy, Section 2.2 "Unstructured sparse
-// gradient tensor"): radix select on the fp32 bit pattern of |g|^2, then an
-// ordered compaction that writes Omega ascending.  Ties at the threshold key
+// gradient tensor"): radix select on the fp32 bit pattern of |g|^2 (first digit on the tensor, the other two on a
+// copy of the threshold bucket's keys), then an ordered compaction that writes Omega ascending.  Ties at the threshold key
 // go to the lower flat index.  Everything is integer work after the key, and
 // no result depends on the order in which atomics land.
 #pragma once
@@ -14,6 +14,14 @@ struct SelState {
   uint32_t krem;     // rank still to resolve inside the current prefix bucket
   uint32_t thr;      // final threshold key (valid after the last pass)
   uint32_t take_eq;  // how many entries with key == thr belong to Omega
+  // After the first pass only the keys of the threshold bucket matter.  When they fit the candidate buffer they are
+  // copied there (one more pass over the tensor, which also counts, per block of kChunk entries, the keys above the
+  // bucket), the second and third digit are found on the copy, and the per-block counts are completed from it: three
+  // passes over the tensor (histogram, copy, compaction) instead of five.
+  uint32_t cand_cap;    // capacity of the candidate buffer in keys (0: never used)
+  uint32_t use_cand;    // decided by the first pick
+  uint32_t cand_total;  // keys in the buffer
+  uint32_t pad;
 };
 
 // What the entries are ranked by (SparseIndices of Algorithm 1 with one of the sparsification strategies of
@@ -83,8 +91,9 @@ constexpr int kSelMaxBins = 2048;
 constexpr int kChunk = 2048;        // elements per compaction block
 constexpr int kChunkThreads = 256;  // 8 consecutive elements per thread
 
-__global__ void sel_init_kernel(SelState* st, uint32_t k) {
+__global__ void sel_init_kernel(SelState* st, uint32_t k, uint32_t cand_cap) {
   st->prefix = 0u; st->krem = k; st->thr = 0u; st->take_eq = 0u;
+  st->cand_cap = cand_cap; st->use_cand = 0u; st->cand_total = 0u; st->pad = 0u;
 }
 
 // Histogram of the current digit over all entries whose higher bits equal the
@@ -96,6 +105,7 @@ __global__ void __launch_bounds__(512) sel_hist_kernel(const void* __restrict__ 
                                                       const SelState* __restrict__ st, uint32_t* __restrict__ hist,
                                                       int* __restrict__ flags, SelKey kp) {
   __shared__ uint32_t sh[kSelMaxBins];
+  if (pass > 0 && st->use_cand) return;        // the later digits come from the candidate buffer
   const int bits = sel_bits(pass), shift = sel_shift(pass);
   const uint32_t nb = 1u << bits;
   for (uint32_t i = threadIdx.x; i < nb; i += blockDim.x) sh[i] = 0u;
@@ -181,6 +191,7 @@ __global__ void __launch_bounds__(1024) sel_pick_kernel(const uint32_t* __restri
       st->prefix = np;
       st->krem = krem - prev;
       if (pass == 2) { st->thr = np; st->take_eq = krem - prev; }
+      if (pass == 0) st->use_cand = (cur - prev <= st->cand_cap) ? 1u : 0u;      // cur - prev: keys in the bucket
     }
   }
 }
@@ -192,6 +203,7 @@ __global__ void __launch_bounds__(kChunkThreads) sel_count_kernel(const void* __
                                                                   uint32_t* __restrict__ blk_gt,
                                                                   uint32_t* __restrict__ blk_eq, SelKey kp) {
   __shared__ uint32_t sg[kChunkThreads / 32], se[kChunkThreads / 32];
+  if (st->use_cand) return;                    // counted from the candidate buffer instead
   const uint32_t thr = st->thr;
   const uint32_t base = blockIdx.x * (uint32_t)kChunk;
   uint32_t cg = 0, ce = 0;
@@ -211,6 +223,104 @@ __global__ void __launch_bounds__(kChunkThreads) sel_count_kernel(const void* __
     for (int w = 0; w < kChunkThreads / 32; ++w) { a += sg[w]; b += se[w]; }
     blk_gt[blockIdx.x] = a; blk_eq[blockIdx.x] = b;
   }
+}
+
+// The pass that copies the threshold bucket: per block of kChunk entries, the keys whose first digit is the chosen
+// one go to a run of the candidate buffer (the block reserves it with one atomic add: where a run lies depends on the
+// order the blocks arrive in, what it holds does not, and nothing downstream looks at more than the multiset of keys of
+// a run), and the keys with a larger first digit are counted.
+template <class S, bool TOPK>
+__global__ void __launch_bounds__(kChunkThreads) sel_gather_kernel(const void* __restrict__ g, uint32_t n, SelState* st,
+                                                                   uint32_t* __restrict__ blk_gt, uint32_t* __restrict__ blk_eq,
+                                                                   uint32_t* __restrict__ cand, uint32_t* __restrict__ cand_start,
+                                                                   uint32_t* __restrict__ cand_cnt, SelKey kp) {
+  __shared__ uint32_t sg[kChunkThreads / 32], sc[kChunkThreads / 32], run_base;
+  if (!st->use_cand) return;
+  constexpr int EPT = kChunk / kChunkThreads;
+  const uint32_t d0 = st->prefix >> sel_shift(0);
+  const uint32_t base = blockIdx.x * (uint32_t)kChunk;
+  const int t = threadIdx.x;
+  uint32_t mine[EPT];
+  uint32_t cg = 0, cc = 0;
+#pragma unroll
+  for (int r = 0; r < EPT; ++r) {
+    const uint32_t i = base + r * kChunkThreads + t;
+    uint32_t key = 0u; bool in = false;
+    if (i < n) {
+      key = TOPK ? mag_key(S::load(g, i)) : sel_key(S::load(g, i), i, kp);
+      const uint32_t d = key >> sel_shift(0);
+      cg += d > d0; in = d == d0;
+    }
+    mine[r] = key;
+    cc |= in ? (1u << r) : 0u;               // which of this thread's entries are candidates
+  }
+  const uint32_t nc = __popc(cc);
+  uint32_t ig = cg, ic = nc;
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t vg = __shfl_up_sync(0xffffffffu, ig, o), vc = __shfl_up_sync(0xffffffffu, ic, o);
+    if ((t & 31) >= o) { ig += vg; ic += vc; }
+  }
+  if ((t & 31) == 31) { sg[t >> 5] = ig; sc[t >> 5] = ic; }
+  __syncthreads();
+  uint32_t woff = 0, tot_g = 0, tot_c = 0;
+  for (int w = 0; w < kChunkThreads / 32; ++w) { if (w < (t >> 5)) woff += sc[w]; tot_g += sg[w]; tot_c += sc[w]; }
+  if (t == 0) {
+    run_base = tot_c ? atomicAdd(&st->cand_total, tot_c) : 0u;
+    blk_gt[blockIdx.x] = tot_g; blk_eq[blockIdx.x] = 0u;
+  }
+  __syncthreads();
+  const uint32_t rb = run_base;
+  if (t == 0) { cand_start[blockIdx.x] = rb; cand_cnt[blockIdx.x] = tot_c; }
+  uint32_t pos = rb + woff + ic - nc;
+#pragma unroll
+  for (int r = 0; r < EPT; ++r)
+    if (cc & (1u << r)) cand[pos++] = mine[r];
+}
+
+// Histogram of the current digit over the candidate keys whose higher bits equal the prefix chosen so far.
+__global__ void __launch_bounds__(512) sel_hist_keys_kernel(const uint32_t* __restrict__ cand, int pass,
+                                                           const SelState* __restrict__ st, uint32_t* __restrict__ hist) {
+  __shared__ uint32_t sh[kSelMaxBins];
+  if (!st->use_cand) return;
+  const int bits = sel_bits(pass), shift = sel_shift(pass);
+  const uint32_t nb = 1u << bits, n = st->cand_total;
+  for (uint32_t i = threadIdx.x; i < nb; i += blockDim.x) sh[i] = 0u;
+  __syncthreads();
+  const uint32_t prefix = st->prefix;
+  const uint32_t hi_mask = 0xffffffffu << (shift + bits);
+  const uint32_t stride = gridDim.x * blockDim.x;
+  for (uint32_t b0 = blockIdx.x * blockDim.x; b0 < n; b0 += stride) {      // block-uniform bound: warps stay converged
+    const uint32_t i = b0 + threadIdx.x;
+    const uint32_t key = i < n ? cand[i] : 0u;
+    const bool in = i < n && (key & hi_mask) == prefix;
+    const uint32_t d = (key >> shift) & (nb - 1u);
+    const unsigned act = __ballot_sync(0xffffffffu, in);
+    if (in) {
+      const unsigned peers = __match_any_sync(act, d);
+      if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&sh[d], (uint32_t)__popc(peers));
+    }
+  }
+  __syncthreads();
+  for (uint32_t i = threadIdx.x; i < nb; i += blockDim.x) {
+    const uint32_t c = sh[i];
+    if (c) atomicAdd(&hist[i], c);
+  }
+}
+
+// Per block of kChunk entries: the keys above / at the final threshold = those above the bucket (counted by the
+// copying pass) + those of the block's run of candidates above / at it.  One thread per block.
+__global__ void __launch_bounds__(256) sel_count_cand_kernel(const uint32_t* __restrict__ cand,
+                                                            const uint32_t* __restrict__ cand_start,
+                                                            const uint32_t* __restrict__ cand_cnt,
+                                                            const SelState* __restrict__ st, uint32_t* __restrict__ blk_gt,
+                                                            uint32_t* __restrict__ blk_eq, uint32_t nblk) {
+  if (!st->use_cand) return;
+  const uint32_t b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= nblk) return;
+  const uint32_t thr = st->thr, s0 = cand_start[b], c = cand_cnt[b];
+  uint32_t cg = 0, ce = 0;
+  for (uint32_t j = 0; j < c; ++j) { const uint32_t key = cand[s0 + j]; cg += key > thr; ce += key == thr; }
+  blk_gt[b] += cg; blk_eq[b] = ce;
 }
 
 // In-place exclusive scan of the per-block counts (single block).

@@ -195,7 +195,7 @@ tgrad_status compute_layout(const tgrad_config* c, Layout& L, int sm) {
   L.w_sel = o; o = align_up(o + sizeof(SelState));
   L.w_hist = o; o = align_up(o + 3 * kSelMaxBins * 4);
   L.nblk = (uint32_t)((numel + kChunk - 1) / kChunk);
-  L.w_blk = o; o = align_up(o + (size_t)2 * L.nblk * 4);
+  L.w_blk = o; o = align_up(o + (size_t)4 * L.nblk * 4);      // per block: keys above / at the threshold, start and length of its run of candidates
   size_t partial = 0;
   for (int n = 0; n < N; ++n) {
     size_t sq = (size_t)c->dims[n] * c->dims[n] * 8;
@@ -658,20 +658,35 @@ tgrad_status select_omega(tgrad_state* s, const void* x, cudaStream_t st) {
   SelKey kp;
   kp.seed_lo = (uint32_t)(c.seed & 0xffffffffull); kp.seed_hi = (uint32_t)(c.seed >> 32);
   kp.epoch = (uint32_t)(s->t / c.T); kp.strategy = c.sparse_strategy;
+  // candidate keys of the threshold bucket: in the two buffers of the compressed tensor, which nothing uses while
+  // Omega is being selected; runs of candidates per block of kChunk entries behind the per-block counts
+  uint32_t* cand = reinterpret_cast<uint32_t*>(s->dw + L.w_bufa);
+  uint64_t cap64 = (uint64_t)(L.w_bufb + L.tsize * 8 - L.w_bufa) / 4;
+  if (cap64 > n / 4) cap64 = n / 4;
+  uint32_t* cand_start = blk_eq + L.nblk;
+  uint32_t* cand_cnt = cand_start + L.nblk;
   if (cudaMemsetAsync(hist, 0, 3 * kSelMaxBins * 4, st) != cudaSuccess) return TGRAD_ERR_CUDA;
-  sel_init_kernel<<<1, 1, 0, st>>>(sel, k); TG_LAUNCH_CHECK();
+  sel_init_kernel<<<1, 1, 0, st>>>(sel, k, (uint32_t)cap64); TG_LAUNCH_CHECK();
   uint64_t want = ((uint64_t)n + 511) / 512;
   int hgrid = (int)(want < (uint64_t)s->sm_count * 8 ? want : (uint64_t)s->sm_count * 8);
   const bool topk = c.sparse_strategy == 0;
   for (int pass = 0; pass < 3; ++pass) {
+    // passes 1 and 2: one of the two histogram kernels returns at once (decided on the device by the first pick)
     if (topk) sel_hist_kernel<S, true><<<hgrid, 512, 0, st>>>(x, n, pass, sel, hist + pass * kSelMaxBins, flags, kp);
     else sel_hist_kernel<S, false><<<hgrid, 512, 0, st>>>(x, n, pass, sel, hist + pass * kSelMaxBins, flags, kp);
     TG_LAUNCH_CHECK();
+    if (pass > 0) { sel_hist_keys_kernel<<<2 * s->sm_count, 512, 0, st>>>(cand, pass, sel, hist + pass * kSelMaxBins); TG_LAUNCH_CHECK(); }
     sel_pick_kernel<<<1, 1024, 0, st>>>(hist + pass * kSelMaxBins, pass, sel); TG_LAUNCH_CHECK();
+    if (pass == 0) {
+      if (topk) sel_gather_kernel<S, true><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, cand, cand_start, cand_cnt, kp);
+      else sel_gather_kernel<S, false><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, cand, cand_start, cand_cnt, kp);
+      TG_LAUNCH_CHECK();
+    }
   }
   if (topk) sel_count_kernel<S, true><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, kp);
   else sel_count_kernel<S, false><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, kp);
   TG_LAUNCH_CHECK();
+  sel_count_cand_kernel<<<(L.nblk + 255) / 256, 256, 0, st>>>(cand, cand_start, cand_cnt, sel, blk_gt, blk_eq, L.nblk); TG_LAUNCH_CHECK();
   sel_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, L.nblk); TG_LAUNCH_CHECK();
   if (topk) sel_compact_kernel<S, true><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, omega, g_s, k, kp);
   else sel_compact_kernel<S, false><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, omega, g_s, k, kp);
@@ -1485,7 +1500,7 @@ tgrad_status select_noalloc_impl(const void* d_grad, uint32_t n, uint32_t k, uin
   uint32_t* blk_eq = sc->blk + nblk;
   // the histograms and the flag word must start at zero; everything else is overwritten before it is read
   if (cudaMemsetAsync(sc->flags, 0, sizeof(sc->flags) + sizeof(sc->hist), st) != cudaSuccess) return TGRAD_ERR_CUDA;
-  sel_init_kernel<<<1, 1, 0, st>>>(&sc->sel, k); TG_LAUNCH_CHECK();
+  sel_init_kernel<<<1, 1, 0, st>>>(&sc->sel, k, 0u); TG_LAUNCH_CHECK();
   const uint64_t want = ((uint64_t)n + 511) / 512;
   const int hgrid = (int)(want < (uint64_t)sm * 8 ? want : (uint64_t)sm * 8);
   for (int pass = 0; pass < 3; ++pass) {
