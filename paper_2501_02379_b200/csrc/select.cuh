@@ -115,7 +115,6 @@ __global__ void __launch_bounds__(512) sel_hist_kernel(const void* __restrict__ 
   bool bad = false;
   constexpr int UN = 4;                       // entries per thread and iteration: their loads are issued together
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x * UN;
-  // block-uniform loop bound, so every warp stays converged for the warp votes below
   for (uint64_t b0 = (uint64_t)blockIdx.x * blockDim.x * UN; b0 < n; b0 += stride) {
     uint32_t keys[UN];
     bool valid[UN];
@@ -134,12 +133,9 @@ __global__ void __launch_bounds__(512) sel_hist_kernel(const void* __restrict__ 
       const uint32_t key = keys[j];
       bool in = valid[j] && (key & hi_mask) == prefix;
       uint32_t d = (key >> shift) & (nb - 1u);
-      // warp-aggregated shared atomics: gradients crowd into a few exponent bins
-      unsigned act = __ballot_sync(0xffffffffu, in);
-      if (in) {
-        unsigned peers = __match_any_sync(act, d);
-        if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&sh[d], (uint32_t)__popc(peers));
-      }
+      // plain shared-memory atomics: measured three times faster than aggregating equal digits within the warp first
+      // (match.any + ballot per entry), although gradients crowd into a few exponent bins
+      if (in) atomicAdd(&sh[d], 1u);
     }
   }
   __syncthreads();
@@ -289,16 +285,12 @@ __global__ void __launch_bounds__(512) sel_hist_keys_kernel(const uint32_t* __re
   const uint32_t prefix = st->prefix;
   const uint32_t hi_mask = 0xffffffffu << (shift + bits);
   const uint32_t stride = gridDim.x * blockDim.x;
-  for (uint32_t b0 = blockIdx.x * blockDim.x; b0 < n; b0 += stride) {      // block-uniform bound: warps stay converged
+  for (uint32_t b0 = blockIdx.x * blockDim.x; b0 < n; b0 += stride) {
     const uint32_t i = b0 + threadIdx.x;
     const uint32_t key = i < n ? cand[i] : 0u;
     const bool in = i < n && (key & hi_mask) == prefix;
     const uint32_t d = (key >> shift) & (nb - 1u);
-    const unsigned act = __ballot_sync(0xffffffffu, in);
-    if (in) {
-      const unsigned peers = __match_any_sync(act, d);
-      if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&sh[d], (uint32_t)__popc(peers));
-    }
+    if (in) atomicAdd(&sh[d], 1u);
   }
   __syncthreads();
   for (uint32_t i = threadIdx.x; i < nb; i += blockDim.x) {
