@@ -26,6 +26,7 @@ __device__ __forceinline__ void cfma_conj(cf& acc, cf a, cf b) {
 struct StoreC64 {
   typedef float2 elem;
   static constexpr int kBytes = 8;
+  static constexpr bool kBf16 = false;
   __device__ static __forceinline__ cf widen(const elem& e) { return e; }
   __device__ static __forceinline__ cf narrow(cf v) { return v; }
   __device__ static __forceinline__ cf load(const void* p, size_t i) { return reinterpret_cast<const float2*>(p)[i]; }
@@ -34,6 +35,7 @@ struct StoreC64 {
 struct StoreC32H {
   typedef __half2 elem;
   static constexpr int kBytes = 4;
+  static constexpr bool kBf16 = false;
   __device__ static __forceinline__ cf widen(const elem& e) { return __half22float2(e); }
   __device__ static __forceinline__ cf narrow(cf v) { return __half22float2(__floats2half2_rn(v.x, v.y)); }
   __device__ static __forceinline__ cf load(const void* p, size_t i) {
@@ -47,6 +49,7 @@ struct StoreC32H {
 struct StoreC32B {
   typedef __nv_bfloat162 elem;
   static constexpr int kBytes = 4;
+  static constexpr bool kBf16 = true;
   __device__ static __forceinline__ cf widen(const elem& e) { return __bfloat1622float2(e); }
   __device__ static __forceinline__ cf narrow(cf v) { return __bfloat1622float2(__floats2bfloat162_rn(v.x, v.y)); }
   __device__ static __forceinline__ cf load(const void* p, size_t i) {

@@ -136,6 +136,41 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
     auto widen = [](const Elem& e) -> cf {
       return S::widen(e);
     };
+    if (HALF) {
+      // 16-bit storage: a stored (re, im) pair is one packed operand register of the m16n8k16 shape (k = 2c, 2c + 1),
+      // so the tiles are contracted as stored, exactly, eight entries per instruction; y = (-im, re) is a swap of
+      // the halves and a sign flip
+      const uint32_t (*Ua)[GR_LD] = reinterpret_cast<const uint32_t (*)[GR_LD]>(Xa);
+      const uint32_t (*Ub)[GR_LD] = reinterpret_cast<const uint32_t (*)[GR_LD]>(XB);
+#pragma unroll
+      for (int ks = 0; ks < GR_KT / 8; ++ks) {
+        const int kc = ks * 8 + t;
+        uint32_t a[2][4];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          const int r = wm * 32 + mt * 16 + gq;
+          a[mt][0] = Ua[r][kc]; a[mt][1] = Ua[r + 8][kc]; a[mt][2] = Ua[r][kc + 4]; a[mt][3] = Ua[r + 8][kc + 4];
+        }
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          if (!FULL && !nok[nt]) continue;
+          const int r = wn * 32 + nt * 8 + gq;
+          const uint32_t b0 = Ub[r][kc], b1 = Ub[r][kc + 4];
+          const uint32_t y0 = ((b0 >> 16) ^ 0x8000u) | (b0 << 16), y1 = ((b1 >> 16) ^ 0x8000u) | (b1 << 16);
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            if (!FULL && !mok[mt]) continue;
+            if (S::kBf16) {
+              mma_bf16(are[mt][nt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], b0, b1);
+              mma_bf16(aim[mt][nt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], y0, y1);
+            } else {
+              mma_f16(are[mt][nt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], b0, b1);
+              mma_f16(aim[mt][nt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], y0, y1);
+            }
+          }
+        }
+      }
+    } else
 #pragma unroll
     for (int ks = 0; ks < GR_KT / 4; ++ks) {
       const int kc = ks * 4 + t;
