@@ -15,7 +15,10 @@
 //     accumulators in tensor memory: Re in columns [0, I_n), Im in [256, 256 + I_n); when 2 I_n <= 256, one
 //     instruction of N = 2 I_n with Im at column I_n) and commits the stage back to the loader.
 // 16-bit storage is contracted exactly (kind::f16, fp16 or bfloat16 operands as stored, products exact in fp32).
-// Grid = (split of the contraction range, 128-row tile of A).  The tensor core adds into its fp32 accumulator with
+// Grid = splits of the contraction range; a launch computes the first 128 rows of A for the rows it is given.  A
+// matrix of more than 128 rows takes two launches: rows 0..127 against all columns (B = all rows, all 512 columns of
+// tensor memory), then the same kernel on the rows from 128 on alone (A is Hermitian: their columns below 128 are
+// the first launch's), which loads and multiplies half as much.  The tensor core adds into its fp32 accumulator with
 // truncation, which biases a long chain (measured: 6e-5 of the diagonal after 676 instructions), so the chain is cut
 // into groups of tiles: after each group four more warps move the accumulators out of tensor memory and add them,
 // with ordinary fp32 adds, into the block's own partial[split][a][b] (entries on and above the diagonal's 16-column
@@ -43,14 +46,17 @@ constexpr uint32_t GT_WAIT_LIMIT = 1u << 22;      // polls of a wait, and
 constexpr uint64_t GT_WAIT_NS = 1000000000ull;     // its limit in nanoseconds of the global timer
 
 struct GramTcParams {
-  int In;                    // rows of the unfolding
+  int In;                    // rows of this launch: rows row0 .. row0 + In of the unfolding
   int rows;                  // In rounded up to a multiple of 16: rows of a tile
+  int row0;                  // first row
+  int a_min;                 // rows of A below this one belong to another launch and are not written
+  int ld;                    // rows (= columns) of the whole Gram matrix
   int stages;
   uint32_t tiles_per_o;      // 128-byte tiles per run of C entries
   uint32_t tiles_total;      // O * tiles_per_o
   uint32_t tiles_per_split;
   uint32_t group_tiles;      // tiles accumulated in tensor memory before the sums move to the partial matrix
-  cf* partial;               // [splits][In][In]
+  cf* partial;               // [splits][ld][ld]
   int* flags;
 };
 
@@ -93,7 +99,6 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gram_tc_kernel(const __grid_con
   const uint32_t t1 = min(t0 + P.tiles_per_split, P.tiles_total);
   const uint32_t n = t1 > t0 ? t1 - t0 : 0;
   const uint32_t F = P.group_tiles;
-  const int mtile = blockIdx.y;
   const bool single = 2 * P.rows <= 256;                // Re and Im columns from one instruction, two accumulator sets
   const int im_col = single ? P.rows : GT_IM_COL;
   const uint32_t nbuf = single ? 2 : 1;
@@ -119,7 +124,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gram_tc_kernel(const __grid_con
         if (!gt_wait(&empty[s], ph ^ 1, failed)) { atomicOr(P.flags, 4); *failed = 1; break; }
         mbar_expect_tx(&full[s], tile_bytes);
         const uint32_t t = t0 + it, o = t / P.tiles_per_o, kt = t - o * P.tiles_per_o;
-        tma_load_3d(tiles0 + s * stage_bytes, &tmap, (int)(kt * BOXK), 0, (int)o, &full[s]);
+        tma_load_3d(tiles0 + s * stage_bytes, &tmap, (int)(kt * BOXK), P.row0, (int)o, &full[s]);
       }
       if (*failed) {
         // loads still in flight must land before the block's shared memory is given up
@@ -142,7 +147,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gram_tc_kernel(const __grid_con
         if (!gt_wait(&ready[s], ph, failed)) { atomicOr(P.flags, 4); *failed = 1; break; }
         tc_fence_after_sync();
         const uint32_t xs = tiles0 + s * stage_bytes, d = tmem + b * 256u;
-        const uint64_t da = umma_desc_k128(xs + (uint32_t)mtile * 128u * GT_ROW_BYTES);
+        const uint64_t da = umma_desc_k128(xs);
         const uint64_t dx = umma_desc_k128(xs), dy = umma_desc_k128(xs + tile_bytes);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks) {                 // 32 bytes of every row per instruction
@@ -195,11 +200,11 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gram_tc_kernel(const __grid_con
   } else {
     // ---- drain: tensor memory -> partial[split][a][b], one group of tiles at a time ----
     const int q = warp & 3;                              // the 32 lanes of tensor memory this warp may read
-    const int a = mtile * 128 + q * 32 + lane;
-    cf* out = P.partial + (size_t)blockIdx.x * P.In * P.In + (size_t)a * P.In;
-    const int c_first = (mtile * 128 + q * 32) & ~15;    // pieces left of the diagonal are not needed
+    const int a = q * 32 + lane;                         // row of the tile; row0 + a of the Gram matrix
+    cf* out = P.partial + (size_t)blockIdx.x * P.ld * P.ld + (size_t)(P.row0 + a) * P.ld + P.row0;
+    const int c_first = (q * 32) & ~15;                  // pieces left of the diagonal are not needed
     const uint32_t ngroups = (n + F - 1) / F;
-    const bool even = (P.In & 1) == 0;                   // rows of the partial matrix start on 16-byte boundaries
+    const bool even = ((P.ld | P.row0) & 1) == 0;        // the 16-column pieces start on 16-byte boundaries
     float4* stg = reinterpret_cast<float4*>(tiles_p + (size_t)stages * stage_bytes) + (warp - 6) * 256;
     for (uint32_t g = 0; g < ngroups; ++g) {
       const uint32_t b = g % nbuf;
@@ -227,14 +232,14 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gram_tc_kernel(const __grid_con
             const int row = 4 * i + (lane >> 3), u = lane & 7;
             float4 v = stg[row * 8 + (u ^ (row & 7))];
             const int ar = a - lane + row;
-            if (ar < P.In && c0 + 2 * u < P.In) {
-              float4* dst = reinterpret_cast<float4*>(out + (ptrdiff_t)(row - lane) * P.In + c0) + u;
+            if (ar < P.In && P.row0 + ar >= P.a_min && c0 + 2 * u < P.In) {
+              float4* dst = reinterpret_cast<float4*>(out + (ptrdiff_t)(row - lane) * P.ld + c0) + u;
               if (g != 0) { const float4 w = *dst; v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w; }
               *dst = v;
             }
           }
           __syncwarp();
-        } else if (a < P.In) {
+        } else if (a < P.In && P.row0 + a >= P.a_min) {
 #pragma unroll
           for (int j = 0; j < 16; ++j)
             if (c0 + j < P.In) {

@@ -117,21 +117,31 @@ void plan_gram(const tgrad_config* c, int n, int sm, uint32_t& chunks, uint32_t&
 // Plan of the tcgen05 Gram kernel for a tensor seen as [O][In][C] with entries of `ebytes` bytes; ok = false when the
 // shape does not suit it (rows that are not 16-byte multiples or too short for 128-byte tiles, a short contraction
 // that wants the split-precision products, fewer than 64 or more than 256 rows) and the mma.sync kernel runs instead.
-struct GramTcPlan { bool ok; int rows, stages, mtiles, splits; uint32_t tiles_per_o, tiles_total, per; };
-constexpr int kGramTcMaxBlocks = 148;     // upper bound of splits x row tiles, whatever the device: sizes the scratch
+struct GramTcLaunch { int In, rows, row0, a_min, stages; };
+struct GramTcPlan { bool ok; int nlaunch, splits; GramTcLaunch l[2]; uint32_t tiles_per_o, tiles_total, per; };
+constexpr int kGramTcMaxBlocks = 148;     // upper bound of the splits, whatever the device: sizes the scratch
 GramTcPlan plan_gram_tc(int In, uint64_t O, uint64_t C, int ebytes, int sm) {
   GramTcPlan pl; memset(&pl, 0, sizeof(pl));
   const uint64_t run = C * (uint64_t)ebytes;           // bytes of one row's contiguous run
   if (In < GT_MIN_ROWS || In > GT_MAX_ROWS || run % 16 != 0 || run < 512 || O * C < 16384) return pl;
   const uint64_t per_o = (run + GT_ROW_BYTES - 1) / GT_ROW_BYTES, total = O * per_o;
   if (O >= (1ull << 31) || 2 * C >= (1ull << 32) || total >= (1ull << 32) || (uint64_t)In * run >= (1ull << 40)) return pl;
-  pl.rows = (In + 15) / 16 * 16;
-  pl.mtiles = pl.rows > 128 ? 2 : 1;
-  const size_t stage = (size_t)2 * pl.rows * GT_ROW_BYTES;
-  pl.stages = (int)((size_t)(200 << 10) / stage);
-  if (pl.stages > GT_MAX_STAGES) pl.stages = GT_MAX_STAGES;
+  const int rows = (In + 15) / 16 * 16;
+  pl.nlaunch = rows > 128 ? 2 : 1;
+  pl.l[0].In = In; pl.l[0].rows = rows; pl.l[0].row0 = 0; pl.l[0].a_min = 0;
+  if (pl.nlaunch == 2) {
+    // the rows from 128 on; at least 64 of them, so that the A operand's 128 rows stay inside a stage
+    int row0 = 128;
+    if (In - row0 < GT_MIN_ROWS) row0 = (In - GT_MIN_ROWS) & ~1;
+    pl.l[1].In = In - row0; pl.l[1].rows = (In - row0 + 15) / 16 * 16; pl.l[1].row0 = row0; pl.l[1].a_min = 128;
+  }
+  for (int i = 0; i < pl.nlaunch; ++i) {
+    const size_t stage = (size_t)2 * pl.l[i].rows * GT_ROW_BYTES;
+    int st = (int)((size_t)(200 << 10) / stage);
+    pl.l[i].stages = st > GT_MAX_STAGES ? GT_MAX_STAGES : st;
+  }
   if (sm > kGramTcMaxBlocks) sm = kGramTcMaxBlocks;
-  uint64_t want = (uint64_t)(sm / pl.mtiles);
+  uint64_t want = (uint64_t)sm;
   if (want < 1) want = 1;
   if (want > total) want = total;
   const uint64_t per = (total + want - 1) / want;
@@ -516,21 +526,25 @@ tgrad_status launch_gram_tc(tgrad_state* s, const void* x, int In, uint64_t O, u
   if (!enc) return TGRAD_ERR_CUDA;
   constexpr int fmt = GramTcFmt<S>::fmt;
   const uint64_t real_bytes = S::kBytes / 2;
-  CUtensorMap tm;
-  const cuuint64_t dims[3] = {2 * C, (cuuint64_t)In, O};
-  const cuuint64_t strides[2] = {C * S::kBytes, (cuuint64_t)In * C * S::kBytes};
-  const cuuint32_t box[3] = {(cuuint32_t)(GT_ROW_BYTES / real_bytes), (cuuint32_t)pl.rows, 1};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  if (enc(&tm, GramTcFmt<S>::dt, 3, const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return TGRAD_ERR_CUDA;
   GramTcParams gp;
-  gp.In = In; gp.rows = pl.rows; gp.stages = pl.stages; gp.tiles_per_o = pl.tiles_per_o; gp.tiles_total = pl.tiles_total;
+  gp.ld = In; gp.tiles_per_o = pl.tiles_per_o; gp.tiles_total = pl.tiles_total;
   gp.tiles_per_split = pl.per; gp.group_tiles = 32; gp.partial = reinterpret_cast<cf*>(s->dw + s->L.w_partial);
   gp.flags = reinterpret_cast<int*>(s->dp + s->L.p_flags);
-  size_t smem = gram_tc_smem(pl.rows, pl.stages);
-  if (smem < ((size_t)120 << 10)) smem = (size_t)120 << 10;   // one block per SM: each takes all of the tensor memory
-  gram_tc_kernel<fmt><<<dim3(pl.splits, pl.mtiles), GT_THREADS, smem, st>>>(tm, gp); TG_LAUNCH_CHECK();
+  for (int i = 0; i < pl.nlaunch; ++i) {
+    const GramTcLaunch& l = pl.l[i];
+    CUtensorMap tm;
+    const cuuint64_t dims[3] = {2 * C, (cuuint64_t)In, O};
+    const cuuint64_t strides[2] = {C * S::kBytes, (cuuint64_t)In * C * S::kBytes};
+    const cuuint32_t box[3] = {(cuuint32_t)(GT_ROW_BYTES / real_bytes), (cuuint32_t)l.rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    if (enc(&tm, GramTcFmt<S>::dt, 3, const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return TGRAD_ERR_CUDA;
+    gp.In = l.In; gp.rows = l.rows; gp.row0 = l.row0; gp.a_min = l.a_min; gp.stages = l.stages;
+    size_t smem = gram_tc_smem(l.rows, l.stages);
+    if (smem < ((size_t)120 << 10)) smem = (size_t)120 << 10;   // one block per SM: each takes all of the tensor memory
+    gram_tc_kernel<fmt><<<pl.splits, GT_THREADS, smem, st>>>(tm, gp); TG_LAUNCH_CHECK();
+  }
   gram_reduce_kernel<<<(In * In + GRR_E - 1) / GRR_E, GRR_E * GRR_G, 0, st>>>(gp.partial, pl.splits, In, A); TG_LAUNCH_CHECK();
   return TGRAD_OK;
 }
