@@ -583,10 +583,11 @@ tgrad_status solve_modes(tgrad_state* s, const int* modes, int nm, bool warm, cu
   SubspaceParams sp; memset(&sp, 0, sizeof(sp));
   size_t sub_bytes = 0;
   int nslow = 0;
-  // no mode's factor is written yet (the eigensolvers below read these words)
-  if (cudaMemsetAsync(flags + SUB_DONE, 0, TGRAD_MAX_NDIM * sizeof(int), st) != cudaSuccess) return TGRAD_ERR_CUDA;
   for (int i = 0; i < nm; ++i) {
     const int m = modes[i];
+    // this mode's factor is not written yet (the eigensolvers below read the word); only this call's modes are
+    // touched: another group of modes may be in flight on another stream
+    if (cudaMemsetAsync(flags + SUB_DONE + m, 0, sizeof(int), st) != cudaSuccess) return TGRAD_ERR_CUDA;
     const int In = (int)c.dims[m];
     cf* A = reinterpret_cast<cf*>(s->dw + L.w_gram[m]);
     {
@@ -943,6 +944,30 @@ tgrad_status hooi_mode_update(tgrad_state* s, int m, const void* d_grad, cudaStr
   return solve_modes(s, &m, 1, true, st);
 }
 
+// One side stream per device on which the eigenvectors of the leading modes are computed while the Gram matrices of
+// the trailing modes are still being accumulated on the caller's stream (the eigensolvers keep one SM per mode busy,
+// the Gram kernels all of them).  Created at the first refresh on the device and kept for the life of the process.
+struct RefreshStreams {
+  std::mutex mu;
+  bool ready = false, failed = false;
+  cudaStream_t side;
+  cudaEvent_t fork, join;
+};
+RefreshStreams g_refresh[64];
+RefreshStreams* refresh_streams() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  RefreshStreams* r = &g_refresh[dev];
+  std::lock_guard<std::mutex> lock(r->mu);
+  if (!r->ready && !r->failed) {
+    const bool ok = cudaStreamCreateWithFlags(&r->side, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&r->fork, cudaEventDisableTiming) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&r->join, cudaEventDisableTiming) == cudaSuccess;
+    r->ready = ok; r->failed = !ok;
+  }
+  return r->ready ? r : nullptr;      // nullptr: everything on the caller's stream
+}
+
 template <class S>
 tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   const tgrad_config& c = s->cfg;
@@ -969,15 +994,33 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   const bool from_stored = c.hooi_iters > 0 && c.warm_refresh && s->basis_valid;
   if (!from_stored) {
     int modes[TGRAD_MAX_NDIM];
-    for (int m = 0; m < N; ++m) {
+    const bool warm = c.warm_refresh && s->basis_valid;
+    auto gram_of = [&](int m) -> tgrad_status {
       uint64_t O = 1, C = 1;
       for (int q = 0; q < m; ++q) O *= c.dims[q];
       for (int q = m + 1; q < N; ++q) C *= c.dims[q];
-      TG_TRY(launch_gram<S>(s, d_grad, (int)c.dims[m], O, C, L.gram_chunks[m], L.gram_cps[m], L.gram_splits[m],
-                            reinterpret_cast<cf*>(s->dw + L.w_gram[m]), st));
-      modes[m] = m;
+      return launch_gram<S>(s, d_grad, (int)c.dims[m], O, C, L.gram_chunks[m], L.gram_cps[m], L.gram_splits[m],
+                            reinterpret_cast<cf*>(s->dw + L.w_gram[m]), st);
+    };
+    for (int m = 0; m < N; ++m) modes[m] = m;
+    const int nlead = N - 2;                       // the leading modes have the larger matrices
+    RefreshStreams* rs = nlead > 0 ? refresh_streams() : nullptr;
+    if (!rs) {
+      for (int m = 0; m < N; ++m) TG_TRY(gram_of(m));
+      TG_TRY(solve_modes(s, modes, N, warm, st));
+    } else {
+      for (int m = 0; m < nlead; ++m) TG_TRY(gram_of(m));
+      std::lock_guard<std::mutex> lock(rs->mu);    // the events are shared by every state on this device
+      if (cudaEventRecord(rs->fork, st) != cudaSuccess || cudaStreamWaitEvent(rs->side, rs->fork, 0) != cudaSuccess)
+        return TGRAD_ERR_CUDA;
+      tgrad_status r = solve_modes(s, modes, nlead, warm, rs->side);
+      for (int m = nlead; m < N && r == TGRAD_OK; ++m) r = gram_of(m);
+      if (r == TGRAD_OK) r = solve_modes(s, modes + nlead, N - nlead, warm, st);
+      // join even after an error, so that nothing is left running unordered
+      if (cudaEventRecord(rs->join, rs->side) != cudaSuccess || cudaStreamWaitEvent(st, rs->join, 0) != cudaSuccess)
+        return TGRAD_ERR_CUDA;
+      TG_TRY(r);
     }
-    TG_TRY(solve_modes(s, modes, N, c.warm_refresh && s->basis_valid, st));
   }
   // Refinement (higher-order orthogonal iteration): per sweep and mode, compress the residual in every other mode
   // with the current factors and take the leading eigenvectors of the mode-n Gram matrix of the result.
