@@ -21,7 +21,8 @@
  *    stages on grad and subtracts, which is bit-identical.
  *  - Pointers named d_* are DEVICE pointers, everything else is host memory.
  *  - The library never allocates or frees device memory and, but for the
- *    side streams of tgrad_step_batched, never creates streams.  The caller owns: the weight, the gradient, one persistent
+ *    side streams of tgrad_step_batched and the one a refresh uses (below),
+ *    never creates streams.  The caller owns: the weight, the gradient, one persistent
  *    block (Omega, U^(n), moments, status words, a split copy of U^(N-1)
  *    laid out for the compression kernel) and one workspace block
  *    (scratch; contents need not survive between calls, but the same
@@ -183,7 +184,15 @@ tgrad_status tgrad_step(tgrad_state* st, void* d_weight, void* d_grad, void* cud
  * eigenvalues of R_(n) R_(n)^H (Jacobi), descending, each column scaled by the
  * unit phase that makes its largest-modulus component real positive.
  * Moments are not touched.  d_grad is modified while the call's work runs and
- * restored at its end. */
+ * restored at its end.
+ * Part of a refresh (the eigenvectors of the leading modes, while the Gram
+ * matrices of the trailing modes are accumulated) runs on one side stream per
+ * device, created at the first refresh on that device and kept for the life of
+ * the process.  It is forked from and joined back into the caller's stream with
+ * events: work enqueued on that stream before the call happens before all of
+ * the refresh, work enqueued after it happens after all of it.  If the stream
+ * cannot be created everything runs on the caller's stream.  The same holds
+ * for a refresh that tgrad_step runs by itself. */
 tgrad_status tgrad_refresh_subspace(tgrad_state* st, void* d_grad, void* cuda_stream);
 
 /* Batched variants over a list of layers: semantically n independent calls
