@@ -24,8 +24,9 @@
 // with ordinary fp32 adds, into the block's own partial[split][a][b] (entries on and above the diagonal's 16-column
 // piece only), while the next group accumulates into the other half of tensor memory (I_n <= 128; larger I_n
 // fill all 512 columns, and the tensor core waits for the drain).  The partials are summed in a fixed order by
-// gram_reduce_kernel: every sum is formed in one order, so the result is deterministic.  Every wait is bounded; a wait that runs out sets the sticky copy-timeout
-// flag, the block drains what it started, frees its tensor memory and returns.
+// gram_reduce_kernel: every sum is formed in one order, so the result is deterministic.  Every wait is bounded; a
+// wait that runs out sets the sticky copy-timeout flag, the block drains what it started, frees its tensor memory
+// and returns.
 #pragma once
 #include <cuda.h>
 #include "common.cuh"
