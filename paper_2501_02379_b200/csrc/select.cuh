@@ -315,21 +315,27 @@ __global__ void __launch_bounds__(256) sel_count_cand_kernel(const uint32_t* __r
   blk_gt[b] += cg; blk_eq[b] = ce;
 }
 
-// In-place exclusive scan of the per-block counts (single block).
+// In-place exclusive scan of the per-block counts (single block; eight consecutive counts per thread and round).
 __global__ void __launch_bounds__(1024) sel_scan_kernel(uint32_t* __restrict__ blk_gt, uint32_t* __restrict__ blk_eq,
                                                        uint32_t nblk) {
+  constexpr int PT = 8;
   __shared__ uint32_t wg[32], we[32];
   __shared__ uint32_t carry_g, carry_e;
   const int t = threadIdx.x;
   if (t == 0) { carry_g = 0; carry_e = 0; }
   __syncthreads();
-  for (uint32_t base = 0; base < nblk; base += 1024) {
-    uint32_t i = base + t;
-    uint32_t g = (i < nblk) ? blk_gt[i] : 0u, e = (i < nblk) ? blk_eq[i] : 0u;
+  for (uint32_t base = 0; base < nblk; base += 1024 * PT) {
+    const uint32_t i0 = base + (uint32_t)t * PT;
+    uint32_t vg[PT], ve[PT], g = 0, e = 0;
+#pragma unroll
+    for (int j = 0; j < PT; ++j) {
+      vg[j] = (i0 + j < nblk) ? blk_gt[i0 + j] : 0u; ve[j] = (i0 + j < nblk) ? blk_eq[i0 + j] : 0u;
+      g += vg[j]; e += ve[j];
+    }
     uint32_t ig = g, ie = e;
     for (int o = 1; o < 32; o <<= 1) {
-      uint32_t vg = __shfl_up_sync(0xffffffffu, ig, o), ve = __shfl_up_sync(0xffffffffu, ie, o);
-      if ((t & 31) >= o) { ig += vg; ie += ve; }
+      uint32_t ug = __shfl_up_sync(0xffffffffu, ig, o), ue = __shfl_up_sync(0xffffffffu, ie, o);
+      if ((t & 31) >= o) { ig += ug; ie += ue; }
     }
     if ((t & 31) == 31) { wg[t >> 5] = ig; we[t >> 5] = ie; }
     __syncthreads();
@@ -342,11 +348,14 @@ __global__ void __launch_bounds__(1024) sel_scan_kernel(uint32_t* __restrict__ b
       wg[t] = ia - a; we[t] = ib - b;
     }
     __syncthreads();
-    uint32_t cg = carry_g, ce = carry_e;
-    uint32_t xg = cg + wg[t >> 5] + ig - g, xe = ce + we[t >> 5] + ie - e;
-    if (i < nblk) { blk_gt[i] = xg; blk_eq[i] = xe; }
+    uint32_t xg = carry_g + wg[t >> 5] + ig - g, xe = carry_e + we[t >> 5] + ie - e;    // exclusive prefix of this thread's run
+#pragma unroll
+    for (int j = 0; j < PT; ++j) {
+      if (i0 + j < nblk) { blk_gt[i0 + j] = xg; blk_eq[i0 + j] = xe; }
+      xg += vg[j]; xe += ve[j];
+    }
     __syncthreads();
-    if (t == 1023) { carry_g = xg + g; carry_e = xe + e; }
+    if (t == 1023) { carry_g = xg; carry_e = xe; }
     __syncthreads();
   }
 }
