@@ -201,23 +201,29 @@ __global__ void __launch_bounds__(kChunkThreads) sel_count_kernel(const void* __
   __shared__ uint32_t sg[kChunkThreads / 32], se[kChunkThreads / 32];
   if (st->use_cand) return;                    // counted from the candidate buffer instead
   const uint32_t thr = st->thr;
-  const uint32_t base = blockIdx.x * (uint32_t)kChunk;
-  uint32_t cg = 0, ce = 0;
-  // coalesced order here: only totals matter
-  for (int r = 0; r < kChunk / kChunkThreads; ++r) {
-    uint32_t i = base + r * kChunkThreads + threadIdx.x;
-    if (i < n) {
-      uint32_t key = TOPK ? mag_key(S::load(g, i)) : sel_key(S::load(g, i), i, kp);
-      cg += key > thr; ce += key == thr;
+  const uint32_t nblk = (n + kChunk - 1) / kChunk;
+  // a block walks over blocks of kChunk entries (the grid is a few blocks per SM, so that the launch costs little
+  // when the kernel has nothing to do)
+  for (uint32_t blk = blockIdx.x; blk < nblk; blk += gridDim.x) {
+    const uint32_t base = blk * (uint32_t)kChunk;
+    uint32_t cg = 0, ce = 0;
+    // coalesced order here: only totals matter
+    for (int r = 0; r < kChunk / kChunkThreads; ++r) {
+      uint32_t i = base + r * kChunkThreads + threadIdx.x;
+      if (i < n) {
+        uint32_t key = TOPK ? mag_key(S::load(g, i)) : sel_key(S::load(g, i), i, kp);
+        cg += key > thr; ce += key == thr;
+      }
     }
-  }
-  for (int o = 16; o; o >>= 1) { cg += __shfl_xor_sync(0xffffffffu, cg, o); ce += __shfl_xor_sync(0xffffffffu, ce, o); }
-  if ((threadIdx.x & 31) == 0) { sg[threadIdx.x >> 5] = cg; se[threadIdx.x >> 5] = ce; }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    uint32_t a = 0, b = 0;
-    for (int w = 0; w < kChunkThreads / 32; ++w) { a += sg[w]; b += se[w]; }
-    blk_gt[blockIdx.x] = a; blk_eq[blockIdx.x] = b;
+    for (int o = 16; o; o >>= 1) { cg += __shfl_xor_sync(0xffffffffu, cg, o); ce += __shfl_xor_sync(0xffffffffu, ce, o); }
+    if ((threadIdx.x & 31) == 0) { sg[threadIdx.x >> 5] = cg; se[threadIdx.x >> 5] = ce; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t a = 0, b = 0;
+      for (int w = 0; w < kChunkThreads / 32; ++w) { a += sg[w]; b += se[w]; }
+      blk_gt[blk] = a; blk_eq[blk] = b;
+    }
+    __syncthreads();
   }
 }
 

@@ -698,8 +698,9 @@ tgrad_status select_omega(tgrad_state* s, const void* x, cudaStream_t st) {
       TG_LAUNCH_CHECK();
     }
   }
-  if (topk) sel_count_kernel<S, true><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, kp);
-  else sel_count_kernel<S, false><<<L.nblk, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, kp);
+  const uint32_t cgrid = L.nblk < (uint32_t)s->sm_count * 8 ? L.nblk : (uint32_t)s->sm_count * 8;
+  if (topk) sel_count_kernel<S, true><<<cgrid, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, kp);
+  else sel_count_kernel<S, false><<<cgrid, kChunkThreads, 0, st>>>(x, n, sel, blk_gt, blk_eq, kp);
   TG_LAUNCH_CHECK();
   sel_count_cand_kernel<<<(L.nblk + 255) / 256, 256, 0, st>>>(cand, cand_start, cand_cnt, sel, blk_gt, blk_eq, L.nblk); TG_LAUNCH_CHECK();
   sel_scan_kernel<<<1, 1024, 0, st>>>(blk_gt, blk_eq, L.nblk); TG_LAUNCH_CHECK();
