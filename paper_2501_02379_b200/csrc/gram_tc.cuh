@@ -53,7 +53,8 @@ struct GramTcParams {
   int a_min;                 // rows of A below this one belong to another launch and are not written
   int ld;                    // rows (= columns) of the whole Gram matrix
   int stages;
-  uint32_t tiles_per_o;      // 128-byte tiles per run of C entries
+  int kt;                    // 128-byte pieces of every row per stage (a tile)
+  uint32_t tiles_per_o;      // tiles per run of C entries
   uint32_t tiles_total;      // O * tiles_per_o
   uint32_t tiles_per_split;
   uint32_t group_tiles;      // tiles accumulated in tensor memory before the sums move to the partial matrix
@@ -62,7 +63,7 @@ struct GramTcParams {
 };
 
 constexpr size_t GT_STAGING = 4 * 32 * 128;     // per drain warp: 32 rows x 16 complex sums
-inline size_t gram_tc_smem(int rows, int stages) { return (size_t)stages * 2 * rows * GT_ROW_BYTES + GT_STAGING + 1024; }
+inline size_t gram_tc_smem(int rows, int stages, int kt) { return (size_t)stages * kt * 2 * rows * GT_ROW_BYTES + GT_STAGING + 1024; }
 
 // wait on an mbarrier phase; gives up when the limit runs out or another thread of the block has given up
 __device__ __forceinline__ bool gt_wait(uint64_t* bar, uint32_t parity, volatile int* failed) {
@@ -94,7 +95,9 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gram_tc_kernel(const __grid_con
   const uint32_t raw = smem_u32(gt_raw);
   const uint32_t tiles0 = (raw + 1023u) & ~1023u;       // swizzled tiles sit on 1,024-byte boundaries
   unsigned char* tiles_p = gt_raw + (tiles0 - raw);
-  const uint32_t tile_bytes = (uint32_t)P.rows * GT_ROW_BYTES, stage_bytes = 2 * tile_bytes;
+  // a stage: KT pieces, each the X half (rows x 128 bytes) followed by its Y half
+  const int KT = P.kt;
+  const uint32_t tile_bytes = (uint32_t)P.rows * GT_ROW_BYTES, piece_bytes = 2 * tile_bytes, stage_bytes = piece_bytes * (uint32_t)KT;
   const int stages = P.stages;
   const uint32_t t0 = blockIdx.x * P.tiles_per_split;
   const uint32_t t1 = min(t0 + P.tiles_per_split, P.tiles_total);
@@ -123,9 +126,11 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gram_tc_kernel(const __grid_con
       for (; it < n; ++it) {
         const int s = it % stages; const uint32_t ph = (it / stages) & 1;
         if (!gt_wait(&empty[s], ph ^ 1, failed)) { atomicOr(P.flags, 4); *failed = 1; break; }
-        mbar_expect_tx(&full[s], tile_bytes);
-        const uint32_t t = t0 + it, o = t / P.tiles_per_o, kt = t - o * P.tiles_per_o;
-        tma_load_3d(tiles0 + s * stage_bytes, &tmap, (int)(kt * BOXK), P.row0, (int)o, &full[s]);
+        mbar_expect_tx(&full[s], tile_bytes * (uint32_t)KT);
+        const uint32_t t = t0 + it, o = t / P.tiles_per_o, kt = (t - o * P.tiles_per_o) * (uint32_t)KT;
+        // (a piece beyond the end of the run starts outside the tensor and arrives as zeros)
+        for (int j = 0; j < KT; ++j)
+          tma_load_3d(tiles0 + s * stage_bytes + j * piece_bytes, &tmap, (int)((kt + j) * BOXK), P.row0, (int)o, &full[s]);
       }
       if (*failed) {
         // loads still in flight must land before the block's shared memory is given up
@@ -147,15 +152,17 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gram_tc_kernel(const __grid_con
         const int s = it % stages; const uint32_t ph = (it / stages) & 1;
         if (!gt_wait(&ready[s], ph, failed)) { atomicOr(P.flags, 4); *failed = 1; break; }
         tc_fence_after_sync();
-        const uint32_t xs = tiles0 + s * stage_bytes, d = tmem + b * 256u;
-        const uint64_t da = umma_desc_k128(xs);
-        const uint64_t dx = umma_desc_k128(xs), dy = umma_desc_k128(xs + tile_bytes);
+        const uint32_t d = tmem + b * 256u;
+        for (int j = 0; j < KT; ++j) {
+          const uint32_t xs = tiles0 + s * stage_bytes + j * piece_bytes;
+          const uint64_t dx = umma_desc_k128(xs), dy = umma_desc_k128(xs + tile_bytes);
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {                 // 32 bytes of every row per instruction
-          const bool acc = in_group != 0 || ks != 0;
-          const uint64_t adv = (uint64_t)(ks * 32 >> 4);
-          umma_ss<TF32>(d, da + adv, dx + adv, idesc, acc);
-          if (!single) umma_ss<TF32>(d + GT_IM_COL, da + adv, dy + adv, idesc, acc);
+          for (int ks = 0; ks < 4; ++ks) {               // 32 bytes of every row per instruction
+            const bool acc = in_group != 0 || j != 0 || ks != 0;
+            const uint64_t adv = (uint64_t)(ks * 32 >> 4);
+            umma_ss<TF32>(d, dx + adv, dx + adv, idesc, acc);
+            if (!single) umma_ss<TF32>(d + GT_IM_COL, dx + adv, dy + adv, idesc, acc);
+          }
         }
         umma_commit(&empty[s]);
         if (++in_group == F || it + 1 == n) { umma_commit(&acc_full[b]); in_group = 0; ++g; }
@@ -169,8 +176,9 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gram_tc_kernel(const __grid_con
     for (uint32_t it = 0; it < n; ++it) {
       const int s = it % stages; const uint32_t ph = (it / stages) & 1;
       if (!gt_wait(&full[s], ph, failed)) { atomicOr(P.flags, 4); *failed = 1; break; }
-      uint4* x = reinterpret_cast<uint4*>(tiles_p + (size_t)s * stage_bytes);
-      uint4* y = reinterpret_cast<uint4*>(tiles_p + (size_t)s * stage_bytes + tile_bytes);
+      for (int pj = 0; pj < KT; ++pj) {
+      uint4* x = reinterpret_cast<uint4*>(tiles_p + (size_t)s * stage_bytes + (size_t)pj * piece_bytes);
+      uint4* y = reinterpret_cast<uint4*>(tiles_p + (size_t)s * stage_bytes + (size_t)pj * piece_bytes + tile_bytes);
       // eight 16-byte pieces per thread in flight: all loads of a batch before its first store (the stores may not
       // overtake loads the compiler cannot prove disjoint)
       for (int c = w; c < nchunks; c += 8 * GT_WORKERS) {
@@ -194,6 +202,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gram_tc_kernel(const __grid_con
           }
           y[c + j * GT_WORKERS] = o;
         }
+      }
       }
       fence_async_smem();
       mbar_arrive(&ready[s]);

@@ -117,8 +117,8 @@ void plan_gram(const tgrad_config* c, int n, int sm, uint32_t& chunks, uint32_t&
 // Plan of the tcgen05 Gram kernel for a tensor seen as [O][In][C] with entries of `ebytes` bytes; ok = false when the
 // shape does not suit it (rows that are not 16-byte multiples or too short for 128-byte tiles, a short contraction
 // that wants the split-precision products, fewer than 64 or more than 256 rows) and the mma.sync kernel runs instead.
-struct GramTcLaunch { int In, rows, row0, a_min, stages; };
-struct GramTcPlan { bool ok; int nlaunch, splits; GramTcLaunch l[2]; uint32_t tiles_per_o, tiles_total, per; };
+struct GramTcLaunch { int In, rows, row0, a_min, stages, kt; uint32_t tiles_per_o, tiles_total, per; int splits; };
+struct GramTcPlan { bool ok; int nlaunch, splits; GramTcLaunch l[2]; };
 constexpr int kGramTcMaxBlocks = 148;     // upper bound of the splits, whatever the device: sizes the scratch
 GramTcPlan plan_gram_tc(int In, uint64_t O, uint64_t C, int ebytes, int sm) {
   GramTcPlan pl; memset(&pl, 0, sizeof(pl));
@@ -135,18 +135,40 @@ GramTcPlan plan_gram_tc(int In, uint64_t O, uint64_t C, int ebytes, int sm) {
     if (In - row0 < GT_MIN_ROWS) row0 = (In - GT_MIN_ROWS) & ~1;
     pl.l[1].In = In - row0; pl.l[1].rows = (In - row0 + 15) / 16 * 16; pl.l[1].row0 = row0; pl.l[1].a_min = 128;
   }
-  for (int i = 0; i < pl.nlaunch; ++i) {
-    const size_t stage = (size_t)2 * pl.l[i].rows * GT_ROW_BYTES;
-    int st = (int)((size_t)(200 << 10) / stage);
-    pl.l[i].stages = st > GT_MAX_STAGES ? GT_MAX_STAGES : st;
-  }
   if (sm > kGramTcMaxBlocks) sm = kGramTcMaxBlocks;
-  uint64_t want = (uint64_t)sm;
-  if (want < 1) want = 1;
-  if (want > total) want = total;
-  const uint64_t per = (total + want - 1) / want;
-  pl.tiles_per_o = (uint32_t)per_o; pl.tiles_total = (uint32_t)total; pl.per = (uint32_t)per;
-  pl.splits = (int)((total + per - 1) / per);
+  for (int i = 0; i < pl.nlaunch; ++i) {
+    GramTcLaunch& l = pl.l[i];
+    // Pieces of 128 bytes per stage and stages, as measured (us per Gram matrix with pieces x stages = 1x4, 2x3, 4x3:
+    // 64 rows of fp32 343 / 244 / 195, 96 rows of fp16 135 / 103 / -, 128 rows of fp32 99 / 123 / -): handing a
+    // stage on costs about the same whatever its size, but more than about 96 KB of tiles in flight is slower again.
+    const size_t piece = (size_t)2 * l.rows * GT_ROW_BYTES;
+    int kt = l.rows <= 64 ? 4 : (l.rows < 128 ? 2 : 1);
+    if ((uint64_t)kt > per_o) kt = (int)per_o;
+    l.kt = kt;
+    int st = (kt == 1 && l.rows <= 128) ? 4 : 3;
+    const int fit = (int)((size_t)(200 << 10) / (piece * kt));
+    if (st > fit) st = fit;
+    if (st > GT_MAX_STAGES) st = GT_MAX_STAGES;
+    if (st < 1) return pl;
+    l.stages = st;
+    const uint64_t tpo = (per_o + kt - 1) / kt, tot = O * tpo;
+    uint64_t want = (uint64_t)(sm < 1 ? 1 : sm);
+    if (want > tot) want = tot;
+    const uint64_t per = (tot + want - 1) / want;
+    l.tiles_per_o = (uint32_t)tpo; l.tiles_total = (uint32_t)tot; l.per = (uint32_t)per;
+    l.splits = (int)((tot + per - 1) / per);
+  }
+  // both launches must write the same number of partial matrices (the reduction sums that many for every entry)
+  if (pl.nlaunch == 2 && pl.l[0].splits != pl.l[1].splits) {
+    const int common = pl.l[0].splits < pl.l[1].splits ? pl.l[0].splits : pl.l[1].splits;
+    for (int i = 0; i < 2; ++i) {
+      GramTcLaunch& l = pl.l[i];
+      const uint64_t per = ((uint64_t)l.tiles_total + common - 1) / common;
+      l.per = (uint32_t)per; l.splits = (int)(((uint64_t)l.tiles_total + per - 1) / per);
+    }
+    if (pl.l[0].splits != pl.l[1].splits) return pl;      // (short contractions only) leave it to the other kernel
+  }
+  pl.splits = pl.l[0].splits;
   pl.ok = true;
   return pl;
 }
@@ -527,8 +549,7 @@ tgrad_status launch_gram_tc(tgrad_state* s, const void* x, int In, uint64_t O, u
   constexpr int fmt = GramTcFmt<S>::fmt;
   const uint64_t real_bytes = S::kBytes / 2;
   GramTcParams gp;
-  gp.ld = In; gp.tiles_per_o = pl.tiles_per_o; gp.tiles_total = pl.tiles_total;
-  gp.tiles_per_split = pl.per; gp.group_tiles = 32; gp.partial = reinterpret_cast<cf*>(s->dw + s->L.w_partial);
+  gp.ld = In; gp.partial = reinterpret_cast<cf*>(s->dw + s->L.w_partial);
   gp.flags = reinterpret_cast<int*>(s->dp + s->L.p_flags);
   for (int i = 0; i < pl.nlaunch; ++i) {
     const GramTcLaunch& l = pl.l[i];
@@ -540,10 +561,12 @@ tgrad_status launch_gram_tc(tgrad_state* s, const void* x, int In, uint64_t O, u
     if (enc(&tm, GramTcFmt<S>::dt, 3, const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return TGRAD_ERR_CUDA;
-    gp.In = l.In; gp.rows = l.rows; gp.row0 = l.row0; gp.a_min = l.a_min; gp.stages = l.stages;
-    size_t smem = gram_tc_smem(l.rows, l.stages);
+    gp.In = l.In; gp.rows = l.rows; gp.row0 = l.row0; gp.a_min = l.a_min; gp.stages = l.stages; gp.kt = l.kt;
+    gp.tiles_per_o = l.tiles_per_o; gp.tiles_total = l.tiles_total; gp.tiles_per_split = l.per;
+    gp.group_tiles = (uint32_t)(32 / l.kt);
+    size_t smem = gram_tc_smem(l.rows, l.stages, l.kt);
     if (smem < ((size_t)120 << 10)) smem = (size_t)120 << 10;   // one block per SM: each takes all of the tensor memory
-    gram_tc_kernel<fmt><<<pl.splits, GT_THREADS, smem, st>>>(tm, gp); TG_LAUNCH_CHECK();
+    gram_tc_kernel<fmt><<<l.splits, GT_THREADS, smem, st>>>(tm, gp); TG_LAUNCH_CHECK();
   }
   gram_reduce_kernel<<<(In * In + GRR_E - 1) / GRR_E, GRR_E * GRR_G, 0, st>>>(gp.partial, pl.splits, In, A); TG_LAUNCH_CHECK();
   return TGRAD_OK;
