@@ -5,7 +5,7 @@
 // With a row as the interleaved real vector x_a = (re, im, re, im, ...) of length 2C,
 //   Re A[a][b] = x_a . x_b,    Im A[a][b] = x_a . y_b,    y_b = (-im, re, -im, re, ...),
 // i.e. one real product D = X [X; Y]^T with K = 2 O C.  The contraction range is cut into tiles of 128 bytes per
-// row.  Per tile:
+// row; a stage of the ring holds 1, 2 or 4 of them (more for fewer rows).  Per piece:
 //   * one thread issues a tiled TMA load of the I_n x 128-byte box (128-byte swizzle, rows beyond I_n and bytes
 //     beyond the run zero-filled) into the X half of a stage;
 //   * four warps make the Y half from it, 16 bytes at a time at the same offset (the swizzle permutes 16-byte pieces
