@@ -198,9 +198,9 @@ tgrad_status tgrad_refresh_subspace(tgrad_state* st, void* d_grad, void* cuda_st
 /* Batched variants over a list of layers: semantically n independent calls
  * (the tensors of an FNO's spectral layers are independent).  Arrays are HOST
  * arrays of handles / device pointers.
- * tgrad_step_batched runs the tensors' kernel chains side by side: it forks
+ * tgrad_step_batched and tgrad_refresh_subspace_batched run the tensors' kernel chains side by side: they fork
  * them onto up to four streams that the library creates per device at the
- * first batched call (the one exception to "creates no streams") and joins
+ * first batched call (an exception to "creates no streams") and join
  * them back into the given stream, so for the caller the call orders like
  * any other work on that stream.  The states must have distinct workspaces,
  * and d_weights / d_grads must not overlap between tensors. */

@@ -1345,8 +1345,25 @@ tgrad_status tgrad_refresh_subspace_batched(tgrad_state* const* states, void* co
   if (n_tensors < 0 || (n_tensors > 0 && (!states || !d_grads))) return TGRAD_ERR_INVALID_ARG;
   for (int i = 0; i < n_tensors; ++i)
     if (!states[i] || !d_grads[i] || !aligned16(d_grads[i])) return TGRAD_ERR_INVALID_ARG;
-  for (int i = 0; i < n_tensors; ++i) TG_TRY(do_refresh(states[i], d_grads[i], static_cast<cudaStream_t>(cuda_stream)));
-  return TGRAD_OK;
+  cudaStream_t user = static_cast<cudaStream_t>(cuda_stream);
+  // as in the batched step: the tensors' refreshes are independent, so they are forked onto the side streams
+  BatchStreams* bs = (n_tensors > 1) ? batch_streams() : nullptr;
+  if (!bs) {
+    for (int i = 0; i < n_tensors; ++i) TG_TRY(do_refresh(states[i], d_grads[i], user));
+    return TGRAD_OK;
+  }
+  std::lock_guard<std::mutex> lock(bs->mu);
+  if (cudaEventRecord(bs->fork, user) != cudaSuccess) return TGRAD_ERR_CUDA;
+  const int lanes = n_tensors < kBatchStreams ? n_tensors : kBatchStreams;
+  for (int j = 0; j < lanes; ++j)
+    if (cudaStreamWaitEvent(bs->side[j], bs->fork, 0) != cudaSuccess) return TGRAD_ERR_CUDA;
+  tgrad_status result = TGRAD_OK;
+  for (int i = 0; i < n_tensors && result == TGRAD_OK; ++i) result = do_refresh(states[i], d_grads[i], bs->side[i % lanes]);
+  for (int j = 0; j < lanes; ++j) {           // join even after an error, so that nothing is left running unordered
+    if (cudaEventRecord(bs->join[j], bs->side[j]) != cudaSuccess || cudaStreamWaitEvent(user, bs->join[j], 0) != cudaSuccess)
+      return TGRAD_ERR_CUDA;
+  }
+  return result;
 }
 
 tgrad_status tgrad_query_status(tgrad_state* st, void* cuda_stream, int32_t* sticky_flags, int64_t* t, int32_t* sweeps) {

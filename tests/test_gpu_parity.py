@@ -308,6 +308,33 @@ def test_batched_matches_single():
         assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("name", ["ragged4", "gram75"])
+def test_batched_refresh_matches_single(name):
+    # five tensors (more than the library has side streams) refreshed one by one and through the batched call: the same
+    # index sets and factors, bit for bit, and the gradients left as they were
+    wl = synth.WORKLOADS[name]
+    gs = [synth.GradientSource(wl, i).gradient(0) for i in range(5)]
+    out = {}
+    for mode in ("single", "batched"):
+        sts = [B.TgradState(B.make_config(wl.shape, wl.ranks, wl.k, wl.T, auto_refresh=False)) for _ in gs]
+        gd = [to_device(g, False) for g in gs]
+        if mode == "single":
+            for st, g in zip(sts, gd):
+                st.refresh_subspace(g)
+        else:
+            B.refresh_subspace_batched(sts, gd)
+        torch.cuda.synchronize()
+        out[mode] = [(st.export(B.WHAT_OMEGA), st.factors()) for st in sts]
+        for st in sts:
+            assert st.query_status()[0] == 0
+        for g, d in zip(gs, gd):
+            assert np.array_equal(from_device(d, False), g)
+    for (oa, fa), (ob, fb) in zip(out["single"], out["batched"]):
+        assert np.array_equal(oa, ob)
+        for ua, ub in zip(fa, fb):
+            assert np.array_equal(ua, ub)
+
+
 def test_nonfinite_sets_flag():
     wl = synth.WORKLOADS["small4"]
     g = synth.GradientSource(wl).gradient(0)
