@@ -48,7 +48,11 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
   constexpr bool HALF = S::kBytes == 4;
   constexpr bool DOSPLIT = SPLIT && !HALF;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, t = lane & 3;
-  const int wm = warp >> 1, wn = warp & 1;           // 2 x 2 warps of 32 x 32
+  // 2 x 2 warps of 32 x 32.  A matrix of at most 32 rows lies in the first warp's quarter alone: the four warps then
+  // all take that quarter and share the contraction range instead (k-step ks goes to warp ks mod 4), and their sums are
+  // added at the end.
+  const bool ksplit = In <= 32;
+  const int wm = ksplit ? 0 : warp >> 1, wn = ksplit ? 0 : warp & 1;
   const int a0 = ta * GR_T, b0 = tb * GR_T;
   const bool diag = ta == tb;
   const uint32_t K32 = O * C;                        // the tensor has fewer than 2^32 entries
@@ -77,15 +81,27 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
     for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
       for (int i = 0; i < 4; ++i) { tre[mt][nt][i] = 0.f; tim[mt][nt][i] = 0.f; }
-  // loader mapping (fixed per thread): lanes along k when rows are runs of k -- a thread keeps one k of
-  // the chunk and walks 16 rows; along the rows when C == 1 -- it keeps one row and walks 16 k
+  // Loader.  Rows of a tile beyond the matrix are never loaded: the tiles are zeroed once, and only the rows that
+  // exist are copied (the copies of a chunk's entries beyond the contraction range write zeros).  Rows are runs of
+  // k (C > 1): a thread keeps one k of the chunk and walks the existing rows, four apart.  C == 1 (the rows of one k
+  // are contiguous): the threads are spread over (existing rows) x (as many k as that leaves room for).
   const bool along_k = C > 1;
-  const int ld_kc = along_k ? (tid % GR_KT) : 0, ld_row = along_k ? (tid / GR_KT) : (tid % GR_T);
-  const int ld_k2 = along_k ? 0 : (tid / GR_T);
+  const int nra = min(GR_T, In - a0), nrb = min(GR_T, In - b0);            // rows of the two tiles that exist
+  const int ld_kc = tid % GR_KT, ld_row = tid / GR_KT;                     // C > 1
+  const int ka = GR_THREADS / nra, kb = GR_THREADS / nrb;                  // C == 1: k per pass (at least 2)
+  const int ra1 = tid % nra, ka0 = tid / nra, rb1 = tid % nrb, kb0 = tid / nrb;
   const unsigned char* gb = static_cast<const unsigned char*>(g);
+  {
+    uint32_t* z = reinterpret_cast<uint32_t*>(gsm);
+    for (int idx = tid; idx < (int)(GR_SMEM / 4); idx += GR_THREADS) z[idx] = 0u;
+    __syncthreads();
+  }
+  auto copy1 = [&](Elem* dst, size_t entry, bool ok) {
+    if (!HALF) cp_async8(dst, ok ? gb + entry * 8 : gb, ok ? 8u : 0u);
+    else cp_async4(dst, ok ? gb + entry * 4 : gb, ok ? 4u : 0u);
+  };
 
-  // chunk ch -> stage st: asynchronous 8-byte copies for fp32 storage (zero-filled outside the tensor),
-  // loads through registers with widening for fp16 storage
+  // chunk ch -> stage st: asynchronous 8-byte (fp32 storage) or 4-byte (16-bit storage) copies
   auto load_chunk = [&](uint32_t ch, int st) {
     const uint32_t kk0 = ch * GR_KT;
     Elem (*xa)[GR_LD] = XA[st];
@@ -95,32 +111,14 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
       const bool kok = kk < K32;
       const uint32_t o = kok ? kk / C : 0, c = kok ? kk - o * C : 0;
       const size_t base = (size_t)o * In * C + c;
-#pragma unroll 4
-      for (int i = 0; i < GR_T / (GR_THREADS / GR_KT); ++i) {
-        const int row = ld_row + i * (GR_THREADS / GR_KT);
-        const bool va = kok && a0 + row < In, vb = kok && b0 + row < In;
-        if (!HALF) {
-          cp_async8(&xa[row][ld_kc], va ? gb + (base + (size_t)(a0 + row) * C) * 8 : gb, va ? 8u : 0u);
-          if (!diag) cp_async8(&xb[row][ld_kc], vb ? gb + (base + (size_t)(b0 + row) * C) * 8 : gb, vb ? 8u : 0u);
-        } else {
-          cp_async4(&xa[row][ld_kc], va ? gb + (base + (size_t)(a0 + row) * C) * 4 : gb, va ? 4u : 0u);
-          if (!diag) cp_async4(&xb[row][ld_kc], vb ? gb + (base + (size_t)(b0 + row) * C) * 4 : gb, vb ? 4u : 0u);
-        }
-      }
+      for (int row = ld_row; row < nra; row += GR_THREADS / GR_KT) copy1(&xa[row][ld_kc], base + (size_t)(a0 + row) * C, kok);
+      if (!diag)
+        for (int row = ld_row; row < nrb; row += GR_THREADS / GR_KT) copy1(&xb[row][ld_kc], base + (size_t)(b0 + row) * C, kok);
     } else {
-#pragma unroll 4
-      for (int i = 0; i < GR_KT / (GR_THREADS / GR_T); ++i) {
-        const int kc = ld_k2 + i * (GR_THREADS / GR_T);
-        const uint32_t kk = kk0 + kc;
-        const bool va = kk < K32 && a0 + ld_row < In, vb = kk < K32 && b0 + ld_row < In;
-        if (!HALF) {
-          cp_async8(&xa[ld_row][kc], va ? gb + ((size_t)kk * In + a0 + ld_row) * 8 : gb, va ? 8u : 0u);
-          if (!diag) cp_async8(&xb[ld_row][kc], vb ? gb + ((size_t)kk * In + b0 + ld_row) * 8 : gb, vb ? 8u : 0u);
-        } else {
-          cp_async4(&xa[ld_row][kc], va ? gb + ((size_t)kk * In + a0 + ld_row) * 4 : gb, va ? 4u : 0u);
-          if (!diag) cp_async4(&xb[ld_row][kc], vb ? gb + ((size_t)kk * In + b0 + ld_row) * 4 : gb, vb ? 4u : 0u);
-        }
-      }
+      if (ka0 < ka)
+        for (int kc = ka0; kc < GR_KT; kc += ka) copy1(&xa[ra1][kc], (size_t)(kk0 + kc) * In + a0 + ra1, kk0 + kc < K32);
+      if (!diag && kb0 < kb)
+        for (int kc = kb0; kc < GR_KT; kc += kb) copy1(&xb[rb1][kc], (size_t)(kk0 + kc) * In + b0 + rb1, kk0 + kc < K32);
     }
     cp_async_commit();
   };
@@ -144,6 +142,7 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
       const uint32_t (*Ub)[GR_LD] = reinterpret_cast<const uint32_t (*)[GR_LD]>(XB);
 #pragma unroll
       for (int ks = 0; ks < GR_KT / 8; ++ks) {
+        if (ksplit && (ks & 3) != warp) continue;
         const int kc = ks * 8 + t;
         uint32_t a[2][4];
 #pragma unroll
@@ -173,6 +172,7 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
     } else
 #pragma unroll
     for (int ks = 0; ks < GR_KT / 4; ++ks) {
+      if (ksplit && (ks & 3) != warp) continue;
       const int kc = ks * 4 + t;
       // A fragments: (row g, re), (row g+8, re), (row g, im), (row g+8, im)
       float ah[2][4], al[2][4];
@@ -214,6 +214,35 @@ __global__ void __launch_bounds__(GR_THREADS, 3) gram_partial_kernel(const void*
             tim[mt][nt][i] += aim[mt][nt][i]; aim[mt][nt][i] = 0.f;
           }
     }
+  }
+  if (ksplit) {
+    // the four warps' sums of the same quarter, added in a fixed order by the first warp (through the tile memory)
+    __syncthreads();
+    float* red = reinterpret_cast<float*>(gsm);          // [warp][re|im][mt][nt][i][lane]: 32 KB
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          red[((((warp * 2 + 0) * 2 + mt) * 4 + nt) * 4 + i) * 32 + lane] = tre[mt][nt][i];
+          red[((((warp * 2 + 1) * 2 + mt) * 4 + nt) * 4 + i) * 32 + lane] = tim[mt][nt][i];
+        }
+    __syncthreads();
+    if (warp != 0) return;
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          float sr = 0.f, si = 0.f;
+          for (int w = 0; w < 4; ++w) {
+            sr += red[((((w * 2 + 0) * 2 + mt) * 4 + nt) * 4 + i) * 32 + lane];
+            si += red[((((w * 2 + 1) * 2 + mt) * 4 + nt) * 4 + i) * 32 + lane];
+          }
+          tre[mt][nt][i] = sr; tim[mt][nt][i] = si;
+        }
   }
   // accumulator (row g | g+8, col 2t | 2t+1) -> partial[split][a][b]
   cf* out = partial + (size_t)blockIdx.y * In * In;
