@@ -1015,6 +1015,7 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   // Starting factors: the leading eigenvectors of the mode-n Gram matrices of the residual (truncated SVDs of the
   // unfoldings).  With refinement sweeps and a warm start, the factors the state holds are the starting point
   // instead (the "warm restart" of the decomposition) and the full-size Gram matrices are not formed at all.
+  bool restored = false;
   const bool from_stored = c.hooi_iters > 0 && c.warm_refresh && s->basis_valid;
   if (!from_stored) {
     int modes[TGRAD_MAX_NDIM];
@@ -1039,6 +1040,14 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
         return TGRAD_ERR_CUDA;
       tgrad_status r = solve_modes(s, modes, nlead, warm, rs->side);
       for (int m = nlead; m < N && r == TGRAD_OK; ++m) r = gram_of(m);
+      // nothing reads the residual any more unless refinement sweeps follow: the gathered values go back into the
+      // gradient now, beside the eigensolvers
+      if (r == TGRAD_OK && k > 0 && comp == 0 && c.hooi_iters == 0) {
+        scatter_restore_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, g_s, k);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        if (cudaPeekAtLastError() != cudaSuccess) r = TGRAD_ERR_CUDA;
+        restored = true;
+      }
       if (r == TGRAD_OK) r = solve_modes(s, modes + nlead, N - nlead, warm, st);
       // join even after an error, so that nothing is left running unordered
       if (cudaEventRecord(rs->join, rs->side) != cudaSuccess || cudaStreamWaitEvent(st, rs->join, 0) != cudaSuccess)
@@ -1050,7 +1059,7 @@ tgrad_status refresh_impl(tgrad_state* s, void* d_grad, cudaStream_t st) {
   // with the current factors and take the leading eigenvectors of the mode-n Gram matrix of the result.
   for (int it = 0; it < c.hooi_iters; ++it)
     for (int m = 0; m < N; ++m) TG_TRY(hooi_mode_update<S>(s, m, d_grad, st));
-  if (k > 0 && comp == 0) { scatter_restore_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, g_s, k); TG_LAUNCH_CHECK(); }
+  if (k > 0 && comp == 0 && !restored) { scatter_restore_kernel<S><<<(k + 255) / 256, 256, 0, st>>>(d_grad, omega, g_s, k); TG_LAUNCH_CHECK(); }
   if (comp == 1) {
     // low rank first: R = G - P_U(G) in a buffer of its own (compression of G down to the core, reconstruction down
     // to the trailing modes, last two modes fused with the subtraction from a copy of G), Omega from R
